@@ -1,0 +1,174 @@
+/*
+ * lookat.h - C ABI of the B200 (sm_100a) LOOKAT library: decode-time attention
+ * whose keys are stored only as product-quantisation codes.
+ *
+ * The four operations follow the paper's statement of the method:
+ *   lookat_fit_codebooks  Section 3.4 "Prototype Learning" (k-means per subspace)
+ *   lookat_encode_keys    Section 3.4 "Encoding" (nearest centroid per subspace)
+ *   lookat_build_lut      Section 3.5 "Precomputation Lookup Tables", Algorithm 1 loop 1
+ *   lookat_attend         Section 3.5 "Lookup and Sum", Algorithm 1 loop 2 + softmax + value sum
+ *
+ * Symbols: B batch, H_q query heads, H_kv KV heads, g = H_q / H_kv, L cached
+ * tokens, d_k / d_v head dims, m subspaces, d_sub = d_k / m, K centroids (<= 256).
+ * Query head hq uses the codebooks, codes and values of KV head hq / g.
+ *
+ * Memory: every data pointer is DEVICE memory owned by the caller unless its
+ * comment says host; the library reads or writes it in stream order on the
+ * context's stream and keeps no reference after the call's work completes.
+ * Arrays are dense, row-major, innermost dimension last.  Pointers must be
+ * aligned to 16 bytes (what cudaMalloc and torch allocations give).
+ * The context owns scratch (chunk partials, a table buffer, k-means sums);
+ * it grows on demand, which allocates: call once at full size before timing.
+ *
+ * Errors: every call returns a lookat_status and launches nothing when it
+ * rejects its arguments.  Calls do not synchronise; asynchronous CUDA errors
+ * surface at the caller's next synchronisation.  There is no CPU fallback.
+ */
+#ifndef LOOKAT_H
+#define LOOKAT_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lookat_ctx lookat_ctx;
+
+typedef enum {
+    LOOKAT_OK = 0,
+    LOOKAT_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, bad shape, out-of-range size */
+    LOOKAT_ERR_UNSUPPORTED = 2,   /* valid but not implemented for this shape */
+    LOOKAT_ERR_CUDA = 3,          /* a CUDA runtime call failed; see lookat_last_error */
+    LOOKAT_ERR_NOMEM = 4,         /* scratch allocation failed */
+    LOOKAT_ERR_TIMEOUT = 5        /* reserved: a bounded device-side wait expired */
+} lookat_status;
+
+typedef struct {
+    int32_t n_q_heads;   /* H_q */
+    int32_t n_kv_heads;  /* H_kv, divides H_q */
+    int32_t d_k;         /* key / query head dim */
+    int32_t d_v;         /* value head dim */
+    int32_t m;           /* subspaces, divides d_k */
+    int32_t K;           /* centroids per subspace, 1..256 (codes are uint8) */
+    float scale;         /* softmax scale; 0 selects 1/sqrt(d_k) (Algorithm 1) */
+} lookat_config;
+
+/* Creates a context bound to CUDA device `device` and to `cuda_stream` (a
+ * cudaStream_t passed as void*; NULL = the default stream).  *out is set only
+ * on success.  Destroy frees the scratch; NULL is accepted. */
+lookat_status lookat_create(const lookat_config *cfg, int device, void *cuda_stream, lookat_ctx **out);
+void lookat_destroy(lookat_ctx *ctx);
+
+/* Host string describing the last error this context returned ("" if none). */
+const char *lookat_last_error(const lookat_ctx *ctx);
+
+/*
+ * Section 3.4, Prototype Learning: for every KV head h and subspace j, a
+ * K-centroid codebook minimising  sum_k min_c || k^(j) - c ||^2  over the
+ * given keys, by `iters` Lloyd iterations (no early stop).
+ *
+ *   keys        fp16 [B][H_kv][n][d_k]; the N = B*n keys of a head are pooled,
+ *               pooled index = b*n + t.  N <= 2^22.
+ *   init        NULL, or fp32 [H_kv][m][K][d_sub] starting centroids.
+ *               NULL: centroid c starts at pooled row (off + c*stride) mod N,
+ *               off = (seed + 0x9E3779B97F4A7C15*(h*m+j+1)) mod 2^64 mod N,
+ *               stride = max(1, N/K).  (The paper fixes no initialisation.)
+ *   codebooks   out, fp32 [H_kv][m][K][d_sub].
+ *   distortion  NULL, or out fp64 [H_kv][m][iters+1]: the objective before
+ *               each update and after the last.
+ * Assignment takes the lowest index among equal minima.  The update is the
+ * exact mean (64-bit fixed-point sums, one fp64 division, rounded to fp32);
+ * an empty cluster keeps its centroid.
+ */
+lookat_status lookat_fit_codebooks(lookat_ctx *ctx, const void *keys, int32_t B, int64_t n,
+                                   int32_t iters, uint64_t seed, const float *init,
+                                   float *codebooks, double *distortion);
+
+/*
+ * Section 3.4, Encoding: code[t][j] = argmin_c || k_t^(j) - C_j[c] ||^2,
+ * lowest index on ties, for n new keys per (batch, KV head), written at token
+ * offset pos of the code cache.
+ *
+ *   keys       fp16 [B][H_kv][n][d_k]
+ *   codebooks  fp32 [H_kv][m][K][d_sub]
+ *   codes      in/out, uint8 [B][H_kv][L_max][m]; rows pos..pos+n-1 are written
+ *   near_ties  NULL, or in/out uint64[1]: incremented once per (key, subspace)
+ *              whose best and second-best distance differ by a relative gap in
+ *              (0, 1e-6) as evaluated in fp64.
+ * Decisions are taken in fp32 and re-taken in fp64 wherever the two best
+ * fp32 distances are within 1e-4 relative, so codes equal the fp64 argmin.
+ * Requires pos >= 0, pos + n <= L_max.
+ */
+lookat_status lookat_encode_keys(lookat_ctx *ctx, const void *keys, int32_t B, int64_t n,
+                                 const float *codebooks, uint8_t *codes, int64_t L_max, int64_t pos,
+                                 unsigned long long *near_ties);
+
+/*
+ * Section 3.5, Precomputation Lookup Tables (Algorithm 1, first loop):
+ *   lut[b][hq][j][c] = sum_i q[b][hq][j*d_sub+i] * C[hq/g][j][c][i]     (unscaled)
+ *
+ *   q    fp16 [B][H_q][d_k]
+ *   lut  out, fp32 [B][H_q][m][K]; products are accumulated in fp64 and
+ *        rounded once.
+ */
+lookat_status lookat_build_lut(lookat_ctx *ctx, const void *q, int32_t B, const float *codebooks,
+                               float *lut);
+
+/*
+ * Section 3.5, Lookup and Sum, and the continuation of Algorithm 1:
+ *   s_t = sum_j lut[j][code[t][j]],  alpha = softmax(s * scale),  o = sum_t alpha_t v_t
+ * over t < seq_len, computed per sequence chunk with a running maximum and a
+ * final merge of the chunk partials.  Keys are never reconstructed.
+ *
+ * Exactly one of `lut` or (`q`, `codebooks`) is given; with lut == NULL the
+ * tables are built first into context scratch.
+ *   codes       uint8 [B][H_kv][L_max][m], every code < K (not checked)
+ *   v           fp16 [B][H_kv][L_max][d_v]
+ *   seq_lens    NULL (all rows use L_max tokens) or int32 [B], 0..L_max
+ *   n_splits    chunks per sequence; 0 = chosen by the library
+ *   out         fp32 [B][H_q][d_v]; a row with seq_len 0 gives zeros
+ *   scores_out  NULL, or fp32 [B][H_q][L_max] raw unscaled s_t for t < seq_len
+ *               (for validation; costs extra writes)
+ */
+lookat_status lookat_attend(lookat_ctx *ctx, const float *lut, const void *q, const float *codebooks,
+                            const uint8_t *codes, const void *v, int32_t B, int64_t L_max,
+                            const int32_t *seq_lens, int32_t n_splits, float *out, float *scores_out);
+
+/*
+ * One decode step driven from HOST buffers (what a serving loop that keeps
+ * its activations on the host calls): copies the step's query, new key and
+ * new value rows to the device, encodes the new key at token `pos`
+ * (Section 3.4), stores the value row there, attends over tokens 0..pos
+ * (Algorithm 1) and copies the output back.  All on the context's stream;
+ * the call returns after the output has arrived (it synchronises the stream).
+ *
+ *   q_host      host fp16 [B][H_q][d_k]          (pinned memory for speed)
+ *   k_new_host  host fp16 [B][H_kv][d_k]
+ *   v_new_host  host fp16 [B][H_kv][d_v]
+ *   codebooks   device fp32 [H_kv][m][K][d_sub]
+ *   codes       device uint8 [B][H_kv][L_max][m]  (row pos is written)
+ *   v           device fp16 [B][H_kv][L_max][d_v] (row pos is written)
+ *   out_host    host fp32 [B][H_q][d_v]
+ * Requires 0 <= pos < L_max.
+ */
+lookat_status lookat_decode_step_host(lookat_ctx *ctx, const void *q_host, const void *k_new_host,
+                                      const void *v_new_host, int32_t B, const float *codebooks,
+                                      uint8_t *codes, void *v, int64_t L_max, int64_t pos,
+                                      int32_t n_splits, float *out_host);
+
+/* Number of kernels this context has launched since it was created. */
+uint64_t lookat_kernel_launches(const lookat_ctx *ctx);
+
+/* Average device time in milliseconds of the attend kernel over the launches
+ * made while timing was enabled (CUDA events on the context's stream).
+ * lookat_set_timing(ctx, 1) resets and starts, (ctx, 0) stops;
+ * lookat_attend_kernel_ms synchronises the events and returns the mean, or
+ * -1 when nothing was timed. */
+void lookat_set_timing(lookat_ctx *ctx, int32_t enabled);
+double lookat_attend_kernel_ms(lookat_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOOKAT_H */

@@ -1,0 +1,255 @@
+"""Thin Python binding of liblookat.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (include/lookat.h)
+and hands it raw device pointers of torch CUDA tensors; no step of the method
+runs in Python or in torch.  There is no CPU path: a missing library or a
+tensor that is not on a CUDA device raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "liblookat.so")
+
+EXPORTS = [
+    "lookat_create", "lookat_destroy", "lookat_last_error", "lookat_fit_codebooks",
+    "lookat_encode_keys", "lookat_build_lut", "lookat_attend", "lookat_decode_step_host",
+    "lookat_kernel_launches", "lookat_set_timing", "lookat_attend_kernel_ms",
+]
+
+STATUS = {0: "LOOKAT_OK", 1: "LOOKAT_ERR_INVALID_ARG", 2: "LOOKAT_ERR_UNSUPPORTED",
+          3: "LOOKAT_ERR_CUDA", 4: "LOOKAT_ERR_NOMEM", 5: "LOOKAT_ERR_TIMEOUT"}
+
+
+class LookatError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS.get(status, status)}: {message}")
+        self.status = status
+
+
+class lookat_config(ctypes.Structure):
+    _fields_ = [("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("m", ctypes.c_int32),
+                ("K", ctypes.c_int32), ("scale", ctypes.c_float)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads liblookat.so (built by paper_2601_10155_b200.build); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} is missing: run `python -m paper_2601_10155_b200.build` (needs nvcc). "
+            "There is no fallback path.")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint64
+    lib.lookat_create.argtypes = [ctypes.POINTER(lookat_config), ctypes.c_int, vp, ctypes.POINTER(vp)]
+    lib.lookat_create.restype = ctypes.c_int
+    lib.lookat_destroy.argtypes = [vp]
+    lib.lookat_destroy.restype = None
+    lib.lookat_last_error.argtypes = [vp]
+    lib.lookat_last_error.restype = ctypes.c_char_p
+    lib.lookat_fit_codebooks.argtypes = [vp, vp, i32, i64, i32, u64, vp, vp, vp]
+    lib.lookat_fit_codebooks.restype = ctypes.c_int
+    lib.lookat_encode_keys.argtypes = [vp, vp, i32, i64, vp, vp, i64, i64, vp]
+    lib.lookat_encode_keys.restype = ctypes.c_int
+    lib.lookat_build_lut.argtypes = [vp, vp, i32, vp, vp]
+    lib.lookat_build_lut.restype = ctypes.c_int
+    lib.lookat_attend.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, vp, i32, vp, vp]
+    lib.lookat_attend.restype = ctypes.c_int
+    lib.lookat_decode_step_host.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i64, i64, i32, vp]
+    lib.lookat_decode_step_host.restype = ctypes.c_int
+    lib.lookat_kernel_launches.argtypes = [vp]
+    lib.lookat_kernel_launches.restype = ctypes.c_uint64
+    lib.lookat_set_timing.argtypes = [vp, i32]
+    lib.lookat_set_timing.restype = None
+    lib.lookat_attend_kernel_ms.argtypes = [vp]
+    lib.lookat_attend_kernel_ms.restype = ctypes.c_double
+    _lib = lib
+    return lib
+
+
+def _dev(t, dtype, name, shape=None):
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor (the library has no CPU path)")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(t.shape)}")
+    return t.data_ptr()
+
+
+def _host(t, dtype, name, shape):
+    if not isinstance(t, torch.Tensor) or t.is_cuda:
+        raise TypeError(f"{name} must be a host tensor")
+    if t.dtype != dtype or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must be contiguous {dtype} of shape {tuple(shape)}")
+    return t.data_ptr()
+
+
+class Lookat:
+    """A library context for one attention shape on one device and stream.
+
+    Method names and argument order are those of the C entry points.
+    """
+
+    def __init__(self, n_q_heads, n_kv_heads, d_k, d_v, m, K=256, scale=0.0, device=0, stream=None):
+        self._lib = load_library()
+        self._h = None
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the LOOKAT library runs on the GPU only")
+        self.cfg = lookat_config(n_q_heads, n_kv_heads, d_k, d_v, m, K, scale)
+        self.device = torch.device("cuda", device)
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        self.stream = stream
+        h = ctypes.c_void_p()
+        st = self._lib.lookat_create(ctypes.byref(self.cfg), device, ctypes.c_void_p(stream.cuda_stream),
+                                     ctypes.byref(h))
+        if st != 0:
+            raise LookatError(st, "lookat_create rejected the configuration or the device")
+        self._h = h
+        self.scale = scale if scale > 0 else 1.0 / math.sqrt(d_k)
+
+    # -- helpers ---------------------------------------------------------------
+    @property
+    def d_sub(self):
+        return self.cfg.d_k // self.cfg.m
+
+    @property
+    def g(self):
+        return self.cfg.n_q_heads // self.cfg.n_kv_heads
+
+    def _check(self, st):
+        if st != 0:
+            raise LookatError(st, self._lib.lookat_last_error(self._h).decode())
+
+    def close(self):
+        if self._h is not None:
+            self._lib.lookat_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the C entry points ------------------------------------------------------
+    def lookat_fit_codebooks(self, keys, iters, seed=0, init=None, codebooks=None, distortion=None,
+                             want_distortion=False):
+        c = self.cfg
+        B, H, n, d_k = keys.shape
+        if codebooks is None:
+            codebooks = torch.empty((c.n_kv_heads, c.m, c.K, self.d_sub), dtype=torch.float32, device=self.device)
+        if distortion is None and want_distortion:
+            distortion = torch.empty((c.n_kv_heads, c.m, iters + 1), dtype=torch.float64, device=self.device)
+        self._check(self._lib.lookat_fit_codebooks(
+            self._h, _dev(keys, torch.float16, "keys", (B, c.n_kv_heads, n, c.d_k)), B, n, iters, seed,
+            _dev(init, torch.float32, "init", (c.n_kv_heads, c.m, c.K, self.d_sub)),
+            _dev(codebooks, torch.float32, "codebooks", (c.n_kv_heads, c.m, c.K, self.d_sub)),
+            _dev(distortion, torch.float64, "distortion", (c.n_kv_heads, c.m, iters + 1))))
+        return (codebooks, distortion) if distortion is not None else codebooks
+
+    def lookat_encode_keys(self, keys, codebooks, codes=None, L_max=None, pos=0, near_ties=None):
+        c = self.cfg
+        B, H, n, d_k = keys.shape
+        if L_max is None:
+            L_max = codes.shape[2] if codes is not None else pos + n
+        if codes is None:
+            codes = torch.zeros((B, c.n_kv_heads, L_max, c.m), dtype=torch.uint8, device=self.device)
+        self._check(self._lib.lookat_encode_keys(
+            self._h, _dev(keys, torch.float16, "keys", (B, c.n_kv_heads, n, c.d_k)), B, n,
+            _dev(codebooks, torch.float32, "codebooks", (c.n_kv_heads, c.m, c.K, self.d_sub)),
+            _dev(codes, torch.uint8, "codes", (B, c.n_kv_heads, L_max, c.m)), L_max, pos,
+            _dev(near_ties, torch.int64, "near_ties", (1,))))
+        return codes
+
+    def lookat_build_lut(self, q, codebooks, lut=None):
+        c = self.cfg
+        B = q.shape[0]
+        if lut is None:
+            lut = torch.empty((B, c.n_q_heads, c.m, c.K), dtype=torch.float32, device=self.device)
+        self._check(self._lib.lookat_build_lut(
+            self._h, _dev(q, torch.float16, "q", (B, c.n_q_heads, c.d_k)), B,
+            _dev(codebooks, torch.float32, "codebooks", (c.n_kv_heads, c.m, c.K, self.d_sub)),
+            _dev(lut, torch.float32, "lut", (B, c.n_q_heads, c.m, c.K))))
+        return lut
+
+    def lookat_attend(self, codes, v, lut=None, q=None, codebooks=None, seq_lens=None, n_splits=0,
+                      out=None, scores_out=None):
+        c = self.cfg
+        B, H, L_max, m = codes.shape
+        if out is None:
+            out = torch.empty((B, c.n_q_heads, c.d_v), dtype=torch.float32, device=self.device)
+        self._check(self._lib.lookat_attend(
+            self._h, _dev(lut, torch.float32, "lut", (B, c.n_q_heads, c.m, c.K)),
+            _dev(q, torch.float16, "q", (B, c.n_q_heads, c.d_k)),
+            _dev(codebooks, torch.float32, "codebooks", (c.n_kv_heads, c.m, c.K, self.d_sub)),
+            _dev(codes, torch.uint8, "codes", (B, c.n_kv_heads, L_max, c.m)),
+            _dev(v, torch.float16, "v", (B, c.n_kv_heads, L_max, c.d_v)), B, L_max,
+            _dev(seq_lens, torch.int32, "seq_lens", (B,)), n_splits,
+            _dev(out, torch.float32, "out", (B, c.n_q_heads, c.d_v)),
+            _dev(scores_out, torch.float32, "scores_out", (B, c.n_q_heads, L_max))))
+        return out
+
+    def lookat_decode_step_host(self, q_host, k_new_host, v_new_host, codebooks, codes, v, pos, out_host,
+                                n_splits=0):
+        c = self.cfg
+        B, H, L_max, m = codes.shape
+        self._check(self._lib.lookat_decode_step_host(
+            self._h, _host(q_host, torch.float16, "q_host", (B, c.n_q_heads, c.d_k)),
+            _host(k_new_host, torch.float16, "k_new_host", (B, c.n_kv_heads, c.d_k)),
+            _host(v_new_host, torch.float16, "v_new_host", (B, c.n_kv_heads, c.d_v)), B,
+            _dev(codebooks, torch.float32, "codebooks", (c.n_kv_heads, c.m, c.K, self.d_sub)),
+            _dev(codes, torch.uint8, "codes", (B, c.n_kv_heads, L_max, c.m)),
+            _dev(v, torch.float16, "v", (B, c.n_kv_heads, L_max, c.d_v)), L_max, pos, n_splits,
+            _host(out_host, torch.float32, "out_host", (B, c.n_q_heads, c.d_v))))
+        return out_host
+
+    def lookat_kernel_launches(self) -> int:
+        return int(self._lib.lookat_kernel_launches(self._h))
+
+    def lookat_set_timing(self, enabled: bool):
+        self._lib.lookat_set_timing(self._h, 1 if enabled else 0)
+
+    def lookat_attend_kernel_ms(self) -> float:
+        return float(self._lib.lookat_attend_kernel_ms(self._h))
+
+
+# ---- byte accounting of the method (Section 3.4 "Compression Ratio", Section 3.1) ----
+def key_bytes_per_token(m: int) -> int:
+    """A compressed key is m uint8 indices."""
+    return m
+
+
+def key_compression_ratio(d_k: int, m: int) -> float:
+    """fp16 key (2*d_k bytes) over its m code bytes."""
+    return 2.0 * d_k / m
+
+
+def lut_entries(m: int, K: int = 256) -> int:
+    return m * K
+
+
+def kv_cache_bytes_fp16(H: int, L: int, d_k: int) -> int:
+    """Uncompressed fp16 KV cache: 2*H*d_k values per token, 2 bytes each."""
+    return 4 * H * L * d_k
+
+
+def attend_bytes_per_token_kvhead(m: int, d_v: int) -> int:
+    """What one attend pass must read per cached token and KV head: m code bytes + fp16 V row."""
+    return m + 2 * d_v

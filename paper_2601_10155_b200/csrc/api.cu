@@ -1,0 +1,435 @@
+// C ABI of liblookat.so: context management, argument validation, dispatch to
+// the kernel launchers.  Every entry point is declared in include/lookat.h.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace lookat {
+
+lookat_status set_error(Ctx *ctx, lookat_status st, const char *fmt, ...)
+{
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+        va_end(ap);
+    }
+    return st;
+}
+
+lookat_status check_launch(Ctx *ctx, const char *what)
+{
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess)
+        return set_error(ctx, LOOKAT_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+    return LOOKAT_OK;
+}
+
+lookat_status ensure(Ctx *ctx, void **ptr, size_t *cap, size_t need_bytes, const char *what)
+{
+    if (need_bytes <= *cap) return LOOKAT_OK;
+    if (*ptr) {
+        cudaStreamSynchronize(ctx->stream);       // earlier work may still use the old buffer
+        cudaFree(*ptr);
+        *ptr = nullptr;
+        *cap = 0;
+    }
+    void *p = nullptr;
+    cudaError_t e = cudaMalloc(&p, need_bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return set_error(ctx, LOOKAT_ERR_NOMEM, "%s: cudaMalloc(%zu) failed: %s", what, need_bytes,
+                         cudaGetErrorString(e));
+    }
+    *ptr = p;
+    *cap = need_bytes;
+    return LOOKAT_OK;
+}
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceGuard {
+    int prev;
+    bool ok;
+    explicit DeviceGuard(int dev) : prev(-1), ok(false)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard()
+    {
+        if (ok && prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+lookat_status need_ptr(Ctx *ctx, const void *p, const char *name)
+{
+    if (!p) return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "%s is NULL", name);
+    if (!aligned16(p)) return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "%s is not 16-byte aligned", name);
+    return LOOKAT_OK;
+}
+
+#define LOOKAT_TRY(expr)                         \
+    do {                                         \
+        lookat_status st__ = (expr);             \
+        if (st__ != LOOKAT_OK) return st__;      \
+    } while (0)
+
+lookat_status attend_impl(Ctx *ctx, const float *lut, const void *q, const float *codebooks,
+                          const uint8_t *codes, const void *v, int32_t B, int64_t L_max,
+                          const int32_t *seq_lens, int64_t uniform_len, int32_t n_splits, float *out,
+                          float *scores_out)
+{
+    const lookat_config &c = ctx->cfg;
+    if (B < 1 || B > 65535) return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "B=%d out of range 1..65535", B);
+    if (L_max < 1 || L_max > (1ll << 30))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "L_max=%lld out of range", (long long)L_max);
+    if (n_splits < 0) return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "n_splits=%d is negative", n_splits);
+    if (lut && (q || codebooks))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "give either lut or (q, codebooks), not both");
+    if (!lut && !(q && codebooks))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "lut is NULL and (q, codebooks) is incomplete");
+    LOOKAT_TRY(need_ptr(ctx, codes, "codes"));
+    LOOKAT_TRY(need_ptr(ctx, v, "v"));
+    LOOKAT_TRY(need_ptr(ctx, out, "out"));
+    if (lut) LOOKAT_TRY(need_ptr(ctx, lut, "lut"));
+    if (q) LOOKAT_TRY(need_ptr(ctx, q, "q"));
+    if (codebooks) LOOKAT_TRY(need_ptr(ctx, codebooks, "codebooks"));
+    if (seq_lens && (reinterpret_cast<uintptr_t>(seq_lens) & 3u))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "seq_lens is not 4-byte aligned");
+    if (scores_out && (reinterpret_cast<uintptr_t>(scores_out) & 3u))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "scores_out is not 4-byte aligned");
+
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return set_error(ctx, LOOKAT_ERR_CUDA, "cannot select device %d", ctx->device);
+
+    if (!lut) {
+        const size_t need = (size_t)B * c.n_q_heads * c.m * c.K * sizeof(float);
+        LOOKAT_TRY(ensure(ctx, (void **)&ctx->lut_scratch, &ctx->lut_cap, need, "table scratch"));
+        LOOKAT_TRY(launch_build_lut(ctx, static_cast<const __half *>(q), B, codebooks, ctx->lut_scratch));
+        lut = ctx->lut_scratch;
+    }
+
+    int splits = n_splits > 0 ? n_splits : attend_auto_splits(ctx, B, L_max);
+    if (splits > L_max) splits = (int)L_max;
+    long long chunk = (L_max + splits - 1) / splits;
+    chunk = (chunk + 15) / 16 * 16;
+    splits = (int)((L_max + chunk - 1) / chunk);
+    if (splits > 65535) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "more than 65535 chunks");
+    if ((long long)c.n_q_heads > 65535)
+        return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "more than 65535 query heads");
+
+    const size_t rows = (size_t)B * c.n_q_heads * splits;
+    LOOKAT_TRY(ensure(ctx, (void **)&ctx->part_o, &ctx->part_o_cap, rows * c.d_v * sizeof(float), "partials"));
+    LOOKAT_TRY(ensure(ctx, (void **)&ctx->part_ml, &ctx->part_ml_cap, rows * 2 * sizeof(float), "partials"));
+
+    AttendArgs a;
+    a.lut = lut;
+    a.codes = codes;
+    a.v = static_cast<const __half *>(v);
+    a.seq_lens = seq_lens;
+    a.uniform_len = (int)uniform_len;
+    a.part_o = ctx->part_o;
+    a.part_ml = ctx->part_ml;
+    a.scores_out = scores_out;
+    a.out = out;
+    a.B = B;
+    a.H_q = c.n_q_heads;
+    a.H_kv = c.n_kv_heads;
+    a.g = c.n_q_heads / c.n_kv_heads;
+    a.d_v = c.d_v;
+    a.m = c.m;
+    a.K = c.K;
+    a.L_max = L_max;
+    a.chunk = (int)chunk;
+    a.n_splits = splits;
+    a.scale_log2 = ctx->scale * 1.4426950408889634f;
+    LOOKAT_TRY(launch_attend(ctx, a));
+    return launch_combine(ctx, a);
+}
+
+lookat_status encode_impl(Ctx *ctx, const void *keys, int32_t B, int64_t n, const float *codebooks,
+                          uint8_t *codes, int64_t L_max, int64_t pos, unsigned long long *near_ties)
+{
+    const lookat_config &c = ctx->cfg;
+    if (B < 1 || (long long)B * c.n_kv_heads > 65535)
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "B*n_kv_heads=%lld out of range 1..65535",
+                         (long long)B * c.n_kv_heads);
+    if (n < 0 || pos < 0 || L_max < 1 || pos + n > L_max)
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "need 0 <= pos, 0 <= n, pos+n <= L_max (n=%lld pos=%lld L_max=%lld)",
+                         (long long)n, (long long)pos, (long long)L_max);
+    if (n > (1ll << 31)) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "n too large");
+    LOOKAT_TRY(need_ptr(ctx, keys, "keys"));
+    LOOKAT_TRY(need_ptr(ctx, codebooks, "codebooks"));
+    LOOKAT_TRY(need_ptr(ctx, codes, "codes"));
+    if (near_ties && (reinterpret_cast<uintptr_t>(near_ties) & 7u))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "near_ties is not 8-byte aligned");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return set_error(ctx, LOOKAT_ERR_CUDA, "cannot select device %d", ctx->device);
+    EncodeArgs a;
+    memset(&a, 0, sizeof(a));
+    a.keys = static_cast<const __half *>(keys);
+    a.codebooks = codebooks;
+    a.codes = codes;
+    a.n = n;
+    a.L_max = L_max;
+    a.pos = pos;
+    a.B = B;
+    a.near_ties = near_ties;
+    return launch_encode(ctx, a);
+}
+
+}  // namespace
+}  // namespace lookat
+
+using namespace lookat;
+
+extern "C" {
+
+lookat_status lookat_create(const lookat_config *cfg, int device, void *cuda_stream, lookat_ctx **out)
+{
+    if (!cfg || !out) return LOOKAT_ERR_INVALID_ARG;
+    const lookat_config &c = *cfg;
+    if (c.n_q_heads < 1 || c.n_kv_heads < 1 || c.n_q_heads % c.n_kv_heads != 0) return LOOKAT_ERR_INVALID_ARG;
+    if (c.d_k < 1 || c.d_k > 1024 || c.d_v < 1 || c.d_v > 1024) return LOOKAT_ERR_INVALID_ARG;
+    if (c.m < 1 || c.d_k % c.m != 0) return LOOKAT_ERR_INVALID_ARG;
+    if (c.K < 1 || c.K > 256) return LOOKAT_ERR_INVALID_ARG;
+    if (c.d_k / c.m > 128) return LOOKAT_ERR_UNSUPPORTED;          // sub-vectors of up to 128 dims
+    if (!(c.scale >= 0.f)) return LOOKAT_ERR_INVALID_ARG;          // also rejects NaN
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
+        cudaGetLastError();
+        return LOOKAT_ERR_CUDA;
+    }
+    Ctx *ctx = new (std::nothrow) Ctx;
+    if (!ctx) return LOOKAT_ERR_NOMEM;
+    memset(ctx, 0, sizeof(Ctx));
+    ctx->cfg = c;
+    ctx->device = device;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->scale = c.scale > 0.f ? c.scale : 1.0f / sqrtf((float)c.d_k);
+    DeviceGuard guard(device);
+    cudaDeviceProp prop;
+    if (!guard.ok || cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx;
+        return LOOKAT_ERR_CUDA;
+    }
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    for (int i = 0; i < kTimingSlots; ++i) {
+        if (cudaEventCreate(&ctx->ev0[i]) != cudaSuccess || cudaEventCreate(&ctx->ev1[i]) != cudaSuccess) {
+            cudaGetLastError();
+            lookat_destroy(reinterpret_cast<lookat_ctx *>(ctx));
+            return LOOKAT_ERR_CUDA;
+        }
+    }
+    *out = reinterpret_cast<lookat_ctx *>(ctx);
+    return LOOKAT_OK;
+}
+
+void lookat_destroy(lookat_ctx *handle)
+{
+    if (!handle) return;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    DeviceGuard guard(ctx->device);
+    cudaStreamSynchronize(ctx->stream);
+    void *bufs[] = {ctx->part_o, ctx->part_ml, ctx->lut_scratch, ctx->fit_sums, ctx->fit_cnt, ctx->fit_assign,
+                    ctx->step_q,  ctx->step_k,  ctx->step_out};
+    for (void *p : bufs)
+        if (p) cudaFree(p);
+    for (int i = 0; i < kTimingSlots; ++i) {
+        if (ctx->ev0[i]) cudaEventDestroy(ctx->ev0[i]);
+        if (ctx->ev1[i]) cudaEventDestroy(ctx->ev1[i]);
+    }
+    cudaGetLastError();
+    delete ctx;
+}
+
+const char *lookat_last_error(const lookat_ctx *handle)
+{
+    return handle ? reinterpret_cast<const Ctx *>(handle)->err : "context is NULL";
+}
+
+uint64_t lookat_kernel_launches(const lookat_ctx *handle)
+{
+    return handle ? reinterpret_cast<const Ctx *>(handle)->launches : 0;
+}
+
+void lookat_set_timing(lookat_ctx *handle, int32_t enabled)
+{
+    if (!handle) return;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    if (enabled) {
+        ctx->timed_ms = 0.0;
+        ctx->timed_n = 0;
+        ctx->ev_next = 0;
+        memset(ctx->ev_used, 0, sizeof(ctx->ev_used));
+    }
+    ctx->timing = enabled ? 1 : 0;
+}
+
+double lookat_attend_kernel_ms(lookat_ctx *handle)
+{
+    if (!handle) return -1.0;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    for (int s = 0; s < kTimingSlots; ++s) {
+        if (!ctx->ev_used[s]) continue;
+        float ms = 0.f;
+        cudaEventSynchronize(ctx->ev1[s]);
+        if (cudaEventElapsedTime(&ms, ctx->ev0[s], ctx->ev1[s]) == cudaSuccess) {
+            ctx->timed_ms += ms;
+            ctx->timed_n += 1;
+        }
+        ctx->ev_used[s] = 0;
+    }
+    return ctx->timed_n ? ctx->timed_ms / (double)ctx->timed_n : -1.0;
+}
+
+lookat_status lookat_build_lut(lookat_ctx *handle, const void *q, int32_t B, const float *codebooks, float *lut)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    if (B < 1 || B > 65535) return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "B=%d out of range 1..65535", B);
+    if (ctx->cfg.n_q_heads > 65535) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "more than 65535 query heads");
+    LOOKAT_TRY(need_ptr(ctx, q, "q"));
+    LOOKAT_TRY(need_ptr(ctx, codebooks, "codebooks"));
+    LOOKAT_TRY(need_ptr(ctx, lut, "lut"));
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return set_error(ctx, LOOKAT_ERR_CUDA, "cannot select device %d", ctx->device);
+    return launch_build_lut(ctx, static_cast<const __half *>(q), B, codebooks, lut);
+}
+
+lookat_status lookat_attend(lookat_ctx *handle, const float *lut, const void *q, const float *codebooks,
+                            const uint8_t *codes, const void *v, int32_t B, int64_t L_max,
+                            const int32_t *seq_lens, int32_t n_splits, float *out, float *scores_out)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    return attend_impl(reinterpret_cast<Ctx *>(handle), lut, q, codebooks, codes, v, B, L_max, seq_lens, L_max,
+                       n_splits, out, scores_out);
+}
+
+lookat_status lookat_encode_keys(lookat_ctx *handle, const void *keys, int32_t B, int64_t n,
+                                 const float *codebooks, uint8_t *codes, int64_t L_max, int64_t pos,
+                                 unsigned long long *near_ties)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    return encode_impl(reinterpret_cast<Ctx *>(handle), keys, B, n, codebooks, codes, L_max, pos, near_ties);
+}
+
+lookat_status lookat_fit_codebooks(lookat_ctx *handle, const void *keys, int32_t B, int64_t n, int32_t iters,
+                                   uint64_t seed, const float *init, float *codebooks, double *distortion)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    const lookat_config &c = ctx->cfg;
+    if (B < 1 || (long long)B * c.n_kv_heads > 65535)
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "B*n_kv_heads out of range 1..65535");
+    if (n < 1 || (long long)B * n > (1ll << 22))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "need 1 <= B*n <= 2^22 keys per head (B*n=%lld)",
+                         (long long)B * n);
+    if (iters < 0 || iters > 100000) return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "iters=%d out of range", iters);
+    LOOKAT_TRY(need_ptr(ctx, keys, "keys"));
+    LOOKAT_TRY(need_ptr(ctx, codebooks, "codebooks"));
+    if (init) LOOKAT_TRY(need_ptr(ctx, init, "init"));
+    if (distortion && (reinterpret_cast<uintptr_t>(distortion) & 7u))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "distortion is not 8-byte aligned");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return set_error(ctx, LOOKAT_ERR_CUDA, "cannot select device %d", ctx->device);
+
+    const int d_sub = c.d_k / c.m;
+    const size_t clusters = (size_t)c.n_kv_heads * c.m * c.K;
+    const bool fresh_sums = clusters * d_sub * 8 > ctx->fit_sums_cap;
+    const bool fresh_cnt = clusters * 8 > ctx->fit_cnt_cap;
+    LOOKAT_TRY(ensure(ctx, (void **)&ctx->fit_sums, &ctx->fit_sums_cap, clusters * d_sub * 8, "k-means sums"));
+    LOOKAT_TRY(ensure(ctx, (void **)&ctx->fit_cnt, &ctx->fit_cnt_cap, clusters * 8, "k-means counts"));
+    LOOKAT_TRY(ensure(ctx, (void **)&ctx->fit_assign, &ctx->fit_assign_cap,
+                      (size_t)B * c.n_kv_heads * n * c.m, "k-means assignments"));
+    // sums and counts are left at zero by every update; fresh buffers are cleared here
+    if (fresh_sums && cudaMemsetAsync(ctx->fit_sums, 0, ctx->fit_sums_cap, ctx->stream) != cudaSuccess)
+        return set_error(ctx, LOOKAT_ERR_CUDA, "memset failed");
+    if (fresh_cnt && cudaMemsetAsync(ctx->fit_cnt, 0, ctx->fit_cnt_cap, ctx->stream) != cudaSuccess)
+        return set_error(ctx, LOOKAT_ERR_CUDA, "memset failed");
+    if (distortion &&
+        cudaMemsetAsync(distortion, 0, (size_t)c.n_kv_heads * c.m * (iters + 1) * sizeof(double), ctx->stream) !=
+            cudaSuccess)
+        return set_error(ctx, LOOKAT_ERR_CUDA, "memset failed");
+
+    LOOKAT_TRY(launch_fit_init(ctx, static_cast<const __half *>(keys), B, n, seed, init, codebooks));
+    for (int it = 0; it <= iters; ++it) {
+        const bool last = it == iters;
+        if (last && !distortion) break;                   // the closing pass only measures
+        EncodeArgs a;
+        memset(&a, 0, sizeof(a));
+        a.keys = static_cast<const __half *>(keys);
+        a.codebooks = codebooks;
+        a.codes = ctx->fit_assign;
+        a.n = n;
+        a.L_max = n;
+        a.pos = 0;
+        a.B = B;
+        a.sums = ctx->fit_sums;
+        a.cnt = ctx->fit_cnt;
+        a.distortion = distortion ? distortion + it : nullptr;
+        a.distortion_stride = iters + 1;
+        LOOKAT_TRY(launch_encode(ctx, a));
+        // the closing pass also filled the sums; the update below only clears them then
+        LOOKAT_TRY(launch_fit_update(ctx, last ? nullptr : codebooks));
+    }
+    return LOOKAT_OK;
+}
+
+lookat_status lookat_decode_step_host(lookat_ctx *handle, const void *q_host, const void *k_new_host,
+                                      const void *v_new_host, int32_t B, const float *codebooks, uint8_t *codes,
+                                      void *v, int64_t L_max, int64_t pos, int32_t n_splits, float *out_host)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    const lookat_config &c = ctx->cfg;
+    if (!q_host || !k_new_host || !v_new_host || !out_host)
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "a host buffer is NULL");
+    if (B < 1 || B > 65535) return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "B=%d out of range", B);
+    if (pos < 0 || pos >= L_max)
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "need 0 <= pos < L_max (pos=%lld L_max=%lld)", (long long)pos,
+                         (long long)L_max);
+    LOOKAT_TRY(need_ptr(ctx, codebooks, "codebooks"));
+    LOOKAT_TRY(need_ptr(ctx, codes, "codes"));
+    LOOKAT_TRY(need_ptr(ctx, v, "v"));
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return set_error(ctx, LOOKAT_ERR_CUDA, "cannot select device %d", ctx->device);
+
+    const size_t q_bytes = (size_t)B * c.n_q_heads * c.d_k * 2;
+    const size_t k_bytes = (size_t)B * c.n_kv_heads * c.d_k * 2;
+    const size_t v_row = (size_t)c.d_v * 2;
+    const size_t out_bytes = (size_t)B * c.n_q_heads * c.d_v * 4;
+    LOOKAT_TRY(ensure(ctx, &ctx->step_q, &ctx->step_q_cap, q_bytes, "step staging"));
+    LOOKAT_TRY(ensure(ctx, &ctx->step_k, &ctx->step_k_cap, k_bytes, "step staging"));
+    LOOKAT_TRY(ensure(ctx, (void **)&ctx->step_out, &ctx->step_out_cap, out_bytes, "step staging"));
+
+    cudaStream_t s = ctx->stream;
+    cudaError_t e = cudaMemcpyAsync(ctx->step_q, q_host, q_bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->step_k, k_new_host, k_bytes, cudaMemcpyHostToDevice, s);
+    // value rows go straight into the cache: B*H_kv rows of d_v halves, one per (b, h), at token pos
+    if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync(static_cast<char *>(v) + (size_t)pos * v_row, (size_t)L_max * v_row, v_new_host, v_row,
+                              v_row, (size_t)B * c.n_kv_heads, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return set_error(ctx, LOOKAT_ERR_CUDA, "host-to-device copy: %s", cudaGetErrorString(e));
+
+    LOOKAT_TRY(encode_impl(ctx, ctx->step_k, B, 1, codebooks, codes, L_max, pos, nullptr));
+    // attend over tokens 0..pos of every row
+    LOOKAT_TRY(attend_impl(ctx, nullptr, ctx->step_q, codebooks, codes, v, B, L_max, nullptr, pos + 1, n_splits,
+                           ctx->step_out, nullptr));
+    e = cudaMemcpyAsync(out_host, ctx->step_out, out_bytes, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return set_error(ctx, LOOKAT_ERR_CUDA, "device-to-host copy: %s", cudaGetErrorString(e));
+    return LOOKAT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,120 @@
+// Internal declarations shared by the translation units of liblookat.so.
+// Not part of the public interface (that is include/lookat.h).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lookat.h"
+
+namespace lookat {
+
+constexpr int kTimingSlots = 64;
+
+// Context: configuration, stream, scratch owned by the library.
+struct Ctx {
+    lookat_config cfg;
+    int device;
+    cudaStream_t stream;
+    int sm_count;
+    int max_smem_optin;
+    float scale;           // resolved softmax scale
+    char err[512];
+    uint64_t launches;
+
+    // attend scratch: chunk partials  o [B][H_q][splits][d_v], (M, l) [B][H_q][splits][2]
+    float *part_o;
+    float *part_ml;
+    size_t part_o_cap, part_ml_cap;       // in floats
+    // tables built on behalf of the caller (lookat_attend with lut == NULL)
+    float *lut_scratch;
+    size_t lut_cap;                        // in floats
+    // k-means scratch
+    unsigned long long *fit_sums;          // [H_kv][m][K][d_sub] fixed-point sums
+    unsigned long long *fit_cnt;           // [H_kv][m][K]
+    uint8_t *fit_assign;                   // [B][H_kv][n][m]
+    size_t fit_sums_cap, fit_cnt_cap, fit_assign_cap;
+    // decode-step staging (device copies of the host rows)
+    void *step_q, *step_k;
+    float *step_out;
+    size_t step_q_cap, step_k_cap, step_out_cap;   // bytes
+
+    // per-launch timing of the attend kernel
+    int timing;
+    cudaEvent_t ev0[kTimingSlots], ev1[kTimingSlots];
+    int ev_used[kTimingSlots];
+    int ev_next;
+    double timed_ms;
+    long timed_n;
+};
+
+lookat_status set_error(Ctx *ctx, lookat_status st, const char *fmt, ...);
+lookat_status check_launch(Ctx *ctx, const char *what);
+lookat_status ensure(Ctx *ctx, void **ptr, size_t *cap, size_t need_bytes, const char *what);
+
+// ---- launchers (each validates nothing: the API layer has done it) ----
+struct AttendArgs {
+    const float *lut;          // [B][H_q][m][K]
+    const uint8_t *codes;      // [B][H_kv][L_max][m]
+    const __half *v;           // [B][H_kv][L_max][d_v]
+    const int32_t *seq_lens;   // [B] or null
+    int uniform_len;           // tokens per row when seq_lens is null
+    float *part_o;             // [B][H_q][n_splits][d_v]
+    float *part_ml;            // [B][H_q][n_splits][2]
+    float *scores_out;         // [B][H_q][L_max] or null
+    float *out;                // [B][H_q][d_v]
+    int B, H_q, H_kv, g, d_v, m, K;
+    long long L_max;
+    int chunk;                 // tokens per split (multiple of 16)
+    int n_splits;
+    float scale_log2;          // scale * log2(e)
+};
+
+// Chooses the number of sequence chunks for a launch (n_splits == 0 in the API).
+int attend_auto_splits(const Ctx *ctx, int B, long long L_max);
+// True when the tensor-core streaming kernel covers this shape.
+bool attend_fast_path(const Ctx *ctx, const void *codes, const void *v, long long L_max);
+lookat_status launch_attend(Ctx *ctx, const AttendArgs &a);
+lookat_status launch_combine(Ctx *ctx, const AttendArgs &a);
+
+lookat_status launch_build_lut(Ctx *ctx, const __half *q, int B, const float *codebooks, float *lut);
+
+struct EncodeArgs {
+    const __half *keys;        // [B][H_kv][n][d_k]
+    const float *codebooks;    // [H_kv][m][K][d_sub]
+    uint8_t *codes;            // [B][H_kv][L_max][m]
+    long long n, L_max, pos;
+    int B;
+    unsigned long long *near_ties;   // or null
+    // k-means mode (all null for plain encoding)
+    unsigned long long *sums;        // [H_kv][m][K][d_sub]
+    unsigned long long *cnt;         // [H_kv][m][K]
+    double *distortion;              // &D[0][0][it], stride (iters+1) per problem; or null
+    int distortion_stride;
+};
+lookat_status launch_encode(Ctx *ctx, const EncodeArgs &a);
+
+lookat_status launch_fit_init(Ctx *ctx, const __half *keys, int B, long long n, uint64_t seed,
+                              const float *init, float *codebooks);
+lookat_status launch_fit_update(Ctx *ctx, float *codebooks);
+
+// ---- small device helpers ----
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Every finite fp16 is an integer multiple of 2^-24; this returns that integer.
+__device__ __forceinline__ long long half_to_fixed24(__half hv)
+{
+    unsigned short h = __half_as_ushort(hv);
+    int e = (h >> 10) & 0x1f;
+    long long f = h & 0x3ff;
+    long long v = (e == 0) ? f : ((f | 0x400) << (e - 1));
+    return (h & 0x8000) ? -v : v;
+}
+
+}  // namespace lookat
