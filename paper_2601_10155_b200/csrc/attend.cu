@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(kThreads, 2) attend_stream_kernel(AttendArgs a
     const int part = n >> 2;                              // 0: weight, 1: its fp16 remainder
     const bool head_ok = hl < heads_here;
 
-    const int seq_len = a.seq_lens ? a.seq_lens[b] : a.uniform_len;
+    const int seq_len = (int)min((long long)(a.seq_lens ? a.seq_lens[b] : a.uniform_len), a.L_max);
     const long long chunk_lo = (long long)split * a.chunk;
     const long long chunk_hi = min((long long)seq_len, chunk_lo + a.chunk);
 
@@ -344,7 +344,7 @@ __global__ void __launch_bounds__(kGenThreads) attend_generic_kernel(AttendArgs 
     const int split = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x;
     const int kvh = hq / a.g;
-    const int seq_len = a.seq_lens ? a.seq_lens[b] : a.uniform_len;
+    const int seq_len = (int)min((long long)(a.seq_lens ? a.seq_lens[b] : a.uniform_len), a.L_max);
     const long long chunk_lo = (long long)split * a.chunk;
     const long long chunk_hi = min((long long)seq_len, chunk_lo + a.chunk);
 

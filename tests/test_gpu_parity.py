@@ -1,0 +1,312 @@
+"""GPU parity: every C-ABI call of the CUDA library against the CPU oracle on
+the same seeded inputs.  Stages are checked with a verified hand-off: attend
+is fed the ORACLE's codes and codebooks, so one stage's permitted deviations
+(near-tie codes) cannot leak into the next stage's comparison.
+
+Tolerances (stated by the benchmark spec): codes bit-exact except near ties (relative
+distance gap in (0, 1e-6)); raw scores |d| <= 1e-4 (1 + |s|); outputs <= 2e-3
+max abs.  Tables: |d| <= 1e-5 (1 + |lut|).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2601_10155_b200 import synth
+from paper_2601_10155_b200.binding import Lookat, LookatError
+
+pytestmark = pytest.mark.gpu
+
+SCORE_TOL = 1e-4
+OUT_TOL = 2e-3
+LUT_TOL = 1e-5
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def ctx_for(w, **kw):
+    return Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K, **kw)
+
+
+def random_books(w, seed):
+    rng = np.random.default_rng(seed)
+    return rng.standard_normal((w.n_kv_heads, w.m, w.K, w.d_sub)).astype(np.float32)
+
+
+def check_codes(gpu_codes, ref_codes, gap):
+    """Bit-exact outside the oracle's near-tie flags; returns (#mismatch inside, #flags)."""
+    diff = gpu_codes != ref_codes
+    near = (gap > 0) & (gap < 1e-6)
+    outside = diff & ~near
+    assert outside.sum() == 0, f"{outside.sum()} code mismatches that are not near ties"
+    return int((diff & near).sum()), int(near.sum())
+
+
+def check_attend(w, lk, q, books, codes, v, seq_lens=None, n_splits=0, scale=None):
+    lut64 = oracle.build_lut(q, books)
+    ref_out, ref_s = oracle.attend(lut64, codes, v, seq_lens=seq_lens, scale=scale, d_k=w.d_k,
+                                   want_scores=True)
+    scores = torch.full((w.B, w.n_q_heads, codes.shape[2]), float("nan"), device="cuda")
+    out = lk.lookat_attend(dev(codes), dev(v), q=dev(q), codebooks=dev(books),
+                           seq_lens=None if seq_lens is None else dev(np.asarray(seq_lens, np.int32)),
+                           n_splits=n_splits, scores_out=scores)
+    torch.cuda.synchronize()
+    out = out.cpu().numpy().astype(np.float64)
+    s = scores.cpu().numpy().astype(np.float64)
+    valid = ~np.isnan(ref_s)
+    assert np.array_equal(np.isnan(s), ~valid), "scores written outside seq_len or missing inside"
+    err_s = np.abs(s[valid] - ref_s[valid]) / (1 + np.abs(ref_s[valid]))
+    assert err_s.max(initial=0) <= SCORE_TOL, f"score error {err_s.max()}"
+    err_o = np.abs(out - ref_out).max()
+    assert err_o <= OUT_TOL, f"output error {err_o}"
+    return err_o
+
+
+# ------------------------------------------------------------------ tables
+@pytest.mark.parametrize("shape", [
+    dict(B=2, n_q_heads=4, n_kv_heads=2, d_k=32, m=4, K=16),
+    dict(B=3, n_q_heads=12, n_kv_heads=12, d_k=64, m=2, K=256),
+    dict(B=2, n_q_heads=8, n_kv_heads=2, d_k=128, m=8, K=256),
+    dict(B=1, n_q_heads=3, n_kv_heads=1, d_k=24, m=8, K=7),          # d_sub = 3
+    dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=16, m=16, K=255),       # d_sub = 1
+])
+def test_build_lut_matches_oracle(shape):
+    w = synth.small_workload(**shape)
+    q = synth.make_queries(w)
+    books = random_books(w, 1)
+    lk = ctx_for(w)
+    lut = lk.lookat_build_lut(dev(q), dev(books)).cpu().numpy()
+    ref = oracle.build_lut(q, books)
+    assert np.all(np.abs(lut - ref) <= LUT_TOL * (1 + np.abs(ref)))
+    # fp64 accumulation then one rounding: equal to the rounded oracle table
+    assert np.array_equal(lut, ref.astype(np.float32))
+
+
+# ------------------------------------------------------------------ encoding
+@pytest.mark.parametrize("shape", [
+    dict(B=2, n_kv_heads=2, n_q_heads=2, d_k=32, m=4, K=16, L=300),        # d_sub 8, tile kernel
+    dict(B=1, n_kv_heads=3, n_q_heads=3, d_k=64, m=4, K=256, L=1500),      # d_sub 16
+    dict(B=2, n_kv_heads=2, n_q_heads=2, d_k=64, m=2, K=256, L=700),       # d_sub 32
+    dict(B=1, n_kv_heads=2, n_q_heads=2, d_k=64, m=16, K=200, L=900),      # d_sub 4
+    dict(B=1, n_kv_heads=2, n_q_heads=2, d_k=24, m=8, K=31, L=5000),       # d_sub 3, generic kernel
+    dict(B=1, n_kv_heads=1, n_q_heads=1, d_k=128, m=1, K=64, L=2100),      # d_sub 128, generic kernel
+    dict(B=2, n_kv_heads=2, n_q_heads=2, d_k=16, m=16, K=256, L=800),      # d_sub 1
+    dict(B=4, n_kv_heads=2, n_q_heads=2, d_k=64, m=4, K=256, L=3),         # few keys: warp kernel
+])
+def test_encode_matches_oracle(shape):
+    w = synth.small_workload(**shape)
+    keys = synth.make_keys(w)
+    books, _ = oracle.fit_codebooks(keys[:, :, :min(w.L, 512)], w.m, w.K, iters=2, seed=3)
+    ref, gap = oracle.encode_keys(keys, books, want_gap=True)
+    lk = ctx_for(w)
+    ties = torch.zeros(1, dtype=torch.int64, device="cuda")
+    codes = lk.lookat_encode_keys(dev(keys), dev(books), near_ties=ties).cpu().numpy()
+    inside, flagged = check_codes(codes, ref, gap)
+    assert int(ties.item()) == flagged
+
+
+def test_encode_duplicate_centroids_and_exact_ties_take_lowest_index():
+    w = synth.small_workload(B=1, n_kv_heads=2, n_q_heads=2, d_k=32, m=4, K=64, L=2000)
+    keys = synth.make_keys(w)
+    books, _ = oracle.fit_codebooks(keys[:, :, :256], w.m, 32, iters=1, seed=1)
+    books = np.concatenate([books, books], axis=2)             # every centroid twice
+    ref, gap = oracle.encode_keys(keys, books, want_gap=True)
+    assert ref.max() < 32 and np.all(gap == 0)
+    lk = ctx_for(w)
+    for n in (2000, 5):                                          # tile kernel and warp kernel
+        codes = lk.lookat_encode_keys(dev(keys[:, :, :n]), dev(books)).cpu().numpy()
+        assert np.array_equal(codes, ref[:, :, :n])
+
+
+def test_encode_appends_at_odd_positions_without_touching_neighbours():
+    w = synth.small_workload(B=2, n_kv_heads=2, n_q_heads=2, d_k=32, m=4, K=16, L=64)
+    keys = synth.make_keys(w)
+    books = random_books(w, 5)
+    lk = ctx_for(w)
+    cache = torch.full((w.B, w.n_kv_heads, 101, w.m), 255, dtype=torch.uint8, device="cuda")
+    ref = np.full((w.B, w.n_kv_heads, 101, w.m), 255, dtype=np.uint8)
+    for pos, n in ((0, 1), (1, 1), (2, 5), (7, 30), (37, 1), (100, 1)):
+        lk.lookat_encode_keys(dev(keys[:, :, :n]), dev(books), codes=cache, pos=pos)
+        oracle.encode_keys(keys[:, :, :n], books, codes=ref, L_max=101, pos=pos)
+    assert np.array_equal(cache.cpu().numpy(), ref)
+    with pytest.raises(LookatError):
+        lk.lookat_encode_keys(dev(keys[:, :, :2]), dev(books), codes=cache, pos=100)
+
+
+# ------------------------------------------------------------------ k-means
+@pytest.mark.parametrize("shape,iters", [
+    (dict(B=2, n_kv_heads=2, n_q_heads=2, d_k=32, m=4, K=32, L=900), 6),
+    (dict(B=1, n_kv_heads=3, n_q_heads=3, d_k=64, m=4, K=256, L=128), 4),      # N < K: every key a centroid
+    (dict(B=8, n_kv_heads=2, n_q_heads=2, d_k=64, m=2, K=256, L=512), 5),
+    (dict(B=1, n_kv_heads=1, n_q_heads=1, d_k=24, m=8, K=9, L=700), 7),        # d_sub 3
+    (dict(B=3, n_kv_heads=2, n_q_heads=2, d_k=16, m=2, K=1, L=101), 2),        # K = 1: the mean
+])
+def test_fit_matches_oracle(shape, iters):
+    w = synth.small_workload(**shape)
+    keys = synth.make_keys(w)
+    lk = ctx_for(w)
+    books, trace = lk.lookat_fit_codebooks(dev(keys), iters, seed=17, want_distortion=True)
+    books, trace = books.cpu().numpy(), trace.cpu().numpy()
+    ref_books, ref_trace = oracle.fit_codebooks(keys, w.m, w.K, iters, seed=17)
+    # single step from the same start: assignments, hence exact means, must agree bit for bit
+    one, _ = oracle.fit_codebooks(keys, w.m, w.K, 1, seed=17)
+    one_gpu = lk.lookat_fit_codebooks(dev(keys), 1, seed=17).cpu().numpy()
+    assert np.array_equal(one_gpu, one)
+    if np.array_equal(books, ref_books):
+        np.testing.assert_allclose(trace, ref_trace, rtol=1e-11, atol=1e-300)
+    else:
+        # only a near-tie decision may split the two runs; both are valid Lloyd runs
+        np.testing.assert_allclose(trace[..., -1], ref_trace[..., -1], rtol=1e-4)
+    assert np.all(trace[..., 1:] <= trace[..., :-1] * (1 + 1e-7))
+
+
+def test_fit_with_given_start_and_fixed_point():
+    rng = np.random.default_rng(12)
+    K, d_sub, per = 6, 4, 40
+    centres = (rng.permutation(K)[:, None] * 16.0 + rng.integers(-2, 3, (K, d_sub))).astype(np.float64)
+    pts = centres[:, None, :] + rng.integers(-8, 9, (K, per, d_sub)) / 16.0
+    perm = rng.permutation(K * per)
+    x = pts.reshape(-1, d_sub)[perm]
+    keys = x.astype(np.float16).reshape(1, 1, K * per, d_sub)
+    true_means = np.stack([x[(perm // per) == c].mean(0) for c in range(K)]).astype(np.float32)
+    lk = Lookat(1, 1, d_sub, 8, 1, K)
+    init = dev(true_means.reshape(1, 1, K, d_sub))
+    books = lk.lookat_fit_codebooks(dev(keys), 3, init=init).cpu().numpy()
+    assert np.array_equal(books[0, 0], true_means)
+
+
+# ------------------------------------------------------------------ attend
+ATTEND_SHAPES = [
+    # streaming kernel: d_v in {64,128}, m in {1,2,4,8,16}
+    dict(B=2, n_q_heads=8, n_kv_heads=2, d_k=128, d_v=128, m=8, K=256, L=1000),      # g=4
+    dict(B=2, n_q_heads=12, n_kv_heads=12, d_k=64, d_v=64, m=4, K=256, L=129),       # g=1
+    dict(B=3, n_q_heads=4, n_kv_heads=2, d_k=64, d_v=64, m=2, K=256, L=1025),        # g=2
+    dict(B=1, n_q_heads=3, n_kv_heads=1, d_k=64, d_v=128, m=16, K=255, L=333),       # g=3, K=255
+    dict(B=1, n_q_heads=16, n_kv_heads=2, d_k=64, d_v=64, m=1, K=16, L=4097),        # g=8: two head groups
+    dict(B=2, n_q_heads=6, n_kv_heads=1, d_k=32, d_v=128, m=4, K=2, L=48),           # g=6: 4 + 2
+    # generic kernel: other d_v / m / odd row pitch
+    dict(B=2, n_q_heads=4, n_kv_heads=2, d_k=32, d_v=8, m=4, K=16, L=200),
+    dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=64, m=64, K=11, L=127),         # m = d_k
+    dict(B=2, n_q_heads=2, n_kv_heads=1, d_k=8, d_v=200, m=8, K=256, L=31),
+    dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=64, m=4, K=256, L=7),           # L*m not a multiple of 16
+]
+
+
+@pytest.mark.parametrize("shape", ATTEND_SHAPES)
+@pytest.mark.parametrize("q_scale", [1.0, 0.1, 0.0])
+def test_attend_matches_oracle(shape, q_scale):
+    w = synth.small_workload(**shape)
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, q_scale)
+    books, _ = oracle.fit_codebooks(keys[:, :, :min(w.L, 400)], w.m, w.K, iters=2, seed=3)
+    codes = oracle.encode_keys(keys, books)
+    lk = ctx_for(w)
+    check_attend(w, lk, q, books, codes, v)
+
+
+@pytest.mark.parametrize("shape", [ATTEND_SHAPES[0], ATTEND_SHAPES[2], ATTEND_SHAPES[6]])
+def test_attend_is_independent_of_the_split_count_and_handles_ragged_rows(shape):
+    w = synth.small_workload(**shape)
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.3)
+    books = random_books(w, 2)
+    codes = oracle.encode_keys(keys, books)
+    lk = ctx_for(w)
+    seq_lens = [0, w.L, 1][:w.B] if w.B <= 3 else None
+    outs = []
+    for n_splits in (1, 2, 3, 7, 64, 0):
+        check_attend(w, lk, q, books, codes, v, seq_lens=seq_lens, n_splits=n_splits)
+        out = lk.lookat_attend(dev(codes), dev(v), q=dev(q), codebooks=dev(books), n_splits=n_splits)
+        outs.append(out.cpu().numpy())
+    for o in outs[1:]:
+        np.testing.assert_allclose(o, outs[0], rtol=0, atol=2e-5)
+    for L_row in (1, 15, 16, 17, w.L - 1):
+        check_attend(w, lk, q, books, codes, v, seq_lens=[L_row] * w.B, n_splits=3)
+
+
+def test_attend_with_prebuilt_tables_and_explicit_scale():
+    w = synth.small_workload(B=2, n_q_heads=8, n_kv_heads=2, d_k=64, d_v=64, m=4, K=64, L=500)
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.5)
+    books = random_books(w, 9)
+    codes = oracle.encode_keys(keys, books)
+    lk = ctx_for(w, scale=0.05)
+    lut = lk.lookat_build_lut(dev(q), dev(books))
+    out = lk.lookat_attend(dev(codes), dev(v), lut=lut).cpu().numpy()
+    ref = oracle.attend(oracle.build_lut(q, books), codes, v, scale=0.05)
+    assert np.abs(out - ref).max() <= OUT_TOL
+    check_attend(w, lk, q, books, codes, v, scale=0.05)
+
+
+def test_exactness_special_case_on_the_gpu():
+    """N <= K: the fitted codebooks hold every key, ADC attention equals exact attention."""
+    w = synth.WORKLOADS["gpt2_l128_m4"]
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w)
+    lk = ctx_for(w)
+    books = lk.lookat_fit_codebooks(dev(keys), w.fit_iters, seed=w.seed)
+    codes = lk.lookat_encode_keys(dev(keys), books)
+    out = lk.lookat_attend(codes, dev(v), q=dev(q), codebooks=books).cpu().numpy()
+    exact = oracle.exact_attention(q, keys, v)
+    assert np.abs(out - exact).max() <= OUT_TOL
+    assert np.array_equal(codes.cpu().numpy(), oracle.encode_keys(keys, books.cpu().numpy()))
+
+
+def test_gpt2_shapes_end_to_end_with_handoff():
+    """The 64x configuration (m=2) at L=1024, batch 8: GPU codebooks vs oracle, codes vs oracle,
+    then attend on the oracle's codes."""
+    w = synth.WORKLOADS["gpt2_b8_l1024_m2"]
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w)
+    lk = ctx_for(w)
+    iters = 3
+    books_gpu = lk.lookat_fit_codebooks(dev(keys), iters, seed=w.seed).cpu().numpy()
+    books, _ = oracle.fit_codebooks(keys, w.m, w.K, iters, seed=w.seed)
+    ref_codes, gap = oracle.encode_keys(keys, books, want_gap=True)
+    codes = lk.lookat_encode_keys(dev(keys), dev(books)).cpu().numpy()
+    check_codes(codes, ref_codes, gap)
+    if not ((gap > 0) & (gap < 1e-6)).any():
+        assert np.array_equal(books_gpu, books)
+    for q_scale in (1.0, 0.1):
+        check_attend(w, lk, synth.make_queries(w, q_scale), books, ref_codes, v)
+
+
+def test_decode_step_from_host_buffers():
+    w = synth.small_workload(B=3, n_q_heads=8, n_kv_heads=2, d_k=64, d_v=64, m=4, K=64, L=300)
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.4)
+    books = random_books(w, 4)
+    lk = ctx_for(w)
+    L_max = 320
+    codes_ref = np.zeros((w.B, w.n_kv_heads, L_max, w.m), np.uint8)
+    oracle.encode_keys(keys, books, codes=codes_ref, L_max=L_max, pos=0)
+    v_cache = np.zeros((w.B, w.n_kv_heads, L_max, w.d_v), np.float16)
+    v_cache[:, :, :w.L - 1] = v[:, :, :w.L - 1]
+    codes_dev = dev(codes_ref)
+    codes_dev[:, :, w.L - 1] = 77                      # the step must write this row
+    v_dev = dev(v_cache)
+    out_host = torch.empty((w.B, w.n_q_heads, w.d_v), dtype=torch.float32).pin_memory()
+    lk.lookat_decode_step_host(torch.from_numpy(q).pin_memory(),
+                               torch.from_numpy(np.ascontiguousarray(keys[:, :, w.L - 1])).pin_memory(),
+                               torch.from_numpy(np.ascontiguousarray(v[:, :, w.L - 1])).pin_memory(),
+                               dev(books), codes_dev, v_dev, w.L - 1, out_host)
+    assert np.array_equal(codes_dev.cpu().numpy()[:, :, :w.L], codes_ref[:, :, :w.L])
+    assert np.array_equal(v_dev.cpu().numpy()[:, :, w.L - 1], v[:, :, w.L - 1])
+    ref = oracle.attend(oracle.build_lut(q, books), codes_ref[:, :, :w.L], v, d_k=w.d_k)
+    assert np.abs(out_host.numpy() - ref).max() <= OUT_TOL
+
+
+def test_invalid_arguments_are_rejected_without_launching():
+    w = synth.small_workload()
+    lk = ctx_for(w)
+    before = lk.lookat_kernel_launches()
+    codes = torch.zeros((w.B, w.n_kv_heads, 32, w.m), dtype=torch.uint8, device="cuda")
+    v = torch.zeros((w.B, w.n_kv_heads, 32, w.d_v), dtype=torch.float16, device="cuda")
+    with pytest.raises(LookatError):
+        lk.lookat_attend(codes, v)                                       # neither lut nor (q, codebooks)
+    with pytest.raises(LookatError):
+        lk.lookat_attend(codes, v, n_splits=-1, lut=torch.zeros((w.B, w.n_q_heads, w.m, w.K), device="cuda"))
+    with pytest.raises((TypeError, ValueError)):
+        lk.lookat_attend(codes.cpu(), v)                                  # host tensor: no CPU path
+    assert lk.lookat_kernel_launches() == before
+    for bad in (dict(m=3), dict(K=0), dict(K=257), dict(n_kv_heads=3)):
+        kw = dict(n_q_heads=4, n_kv_heads=2, d_k=32, d_v=32, m=4, K=16)
+        kw.update(bad)
+        with pytest.raises(LookatError):
+            Lookat(**kw)
