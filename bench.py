@@ -1,0 +1,355 @@
+"""Benchmark of the LOOKAT decode-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl lookat|reference] [--workload NAME]
+
+One step = one decode step of the whole batch: encode the newest key of every
+(batch row, KV head) into the code cache, build the lookup tables for the
+step's queries, and attend (ADC scores, softmax, value sum, chunk merge) over
+all cached tokens.  Codebooks are fitted and the cache is encoded once before
+the timed region (offline calibration and prefill); their device times are
+reported under "setup".  Metric: tokens*heads scored per second
+(B * H_q * L / step time), whole job.
+
+With N > 1 (torchrun, one rank per GPU) every rank runs its own replica of
+the workload; there is no exchange between ranks on this path.
+
+--impl reference times the CPU oracle (tests' reference implementation) on
+the host cores for the same step on a bounded sample of the workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2601_10155_b200 import synth  # noqa: E402
+
+METRIC = "adc_decode_attention_tokens_heads_per_s"
+UNIT = "tokens*heads/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) of one attend_stream_kernel launch on this workload as counted by ncu
+# (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture has been summarised
+# under profiles/.
+ATTEND_DRAM_TRAFFIC_BYTES = None
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and clock-event reasons of one GPU through NVML from a thread."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting"}
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def sample(self):
+        if self._h is None:
+            return
+        nv = self._nv
+        try:
+            self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+            try:
+                bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+            except Exception:
+                bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+            for bit, name in self.REASONS.items():
+                if bits & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self.sample()
+            time.sleep(0.002)
+
+    def start(self):
+        self._stop.clear()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": int(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+def oracle_step_sample(w, rows: int):
+    """Inputs of the oracle's decode step for the first `rows` batch rows, all made on the CPU
+    (generator + the oracle's own k-means and encoder on a small calibration draw)."""
+    import oracle
+    wr = synth.Workload(**{**w.__dict__, "B": rows})
+    keys, v, q = synth.make_keys(wr), synth.make_values(wr), synth.make_queries(wr)
+    calib = synth.make_calibration_keys(wr, 2048)
+    books, _ = oracle.fit_codebooks(calib, w.m, w.K, iters=1, seed=w.seed)
+    codes = oracle.encode_keys(keys, books)
+    return wr, keys, v, q, books, codes
+
+
+def oracle_step(wr, keys, v, q, books, codes):
+    """The same step the GPU times: encode the newest key, build tables, attend."""
+    import oracle
+    L = wr.L
+    oracle.encode_keys(keys[:, :, L - 1:L], books, codes=codes, L_max=L, pos=L - 1)
+    return oracle.decode_step(q, books, codes, v)
+
+
+def time_oracle(w, budget_s: float = 12.0):
+    import oracle
+    rows = 1
+    sample = oracle_step_sample(w, rows)
+    t0 = time.perf_counter()
+    oracle_step(*sample)
+    t1 = time.perf_counter() - t0
+    reps = int(max(1, min(20, budget_s / max(t1, 1e-3))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle_step(*sample)
+    dt = (time.perf_counter() - t0) / reps
+    units = rows * w.n_q_heads * w.L
+    return {"value": units / dt, "unit": UNIT, "cores": oracle.n_threads(), "kind": "oracle",
+            "sample": f"{rows} of {w.B} batch rows ({w.n_q_heads} query heads x {w.L} tokens), "
+                      f"mean of {reps} steps of {dt * 1e3:.1f} ms; fp64, OpenMP over (row, head)"}
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    rows = 1
+    sample = oracle_step_sample(w, rows)
+    for _ in range(args.warmup):
+        oracle_step(*sample)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(*sample)
+    dt = (time.perf_counter() - t0) / args.steps
+    units = rows * w.n_q_heads * w.L
+    value = units / dt
+    sample_txt = (f"each step: {rows} of {w.B} batch rows ({w.n_q_heads} query heads x {w.L} tokens); "
+                  "fp64, OpenMP over (row, head)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.n_threads(), "kind": "oracle",
+                             "sample": sample_txt},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w):
+    return {"workload": w.name, "batch": w.B, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
+            "d_k": w.d_k, "d_v": w.d_v, "seq_len": w.L, "m": w.m, "K": w.K, "v_dtype": "fp16",
+            "codebooks": f"fp32, {w.fit_iters} Lloyd iterations on "
+                         f"{w.fit_keys_per_head or w.B * w.L} keys per KV head",
+            "l2": "inputs larger than L2 (codes + V >> 126 MB), no flush needed"}
+
+
+# ----------------------------------------------------------------------------- GPU leg
+def run_lookat(args, w):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2601_10155_b200.binding import Lookat
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    # every rank runs the same replica shape on its own inputs (seed offset by rank)
+    wr = synth.Workload(**{**w.__dict__, "seed": w.seed + 7919 * rank})
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K, device=local_rank)
+
+    t_gen = time.perf_counter()
+    keys = dev(synth.make_keys(wr))
+    v = dev(synth.make_values(wr))
+    q_np = synth.make_queries(wr)
+    q = dev(q_np)
+    t_gen = time.perf_counter() - t_gen
+
+    # ---- setup: calibration (k-means) and prefill encoding, timed but outside the step ----
+    n_fit = w.fit_keys_per_head or w.B * w.L
+    per_row = max(1, n_fit // w.B)
+    fit_keys = keys[:, :, :per_row].contiguous()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    ev[0].record()
+    books = lk.lookat_fit_codebooks(fit_keys, w.fit_iters, seed=w.seed)
+    ev[1].record()
+    ties = torch.zeros(1, dtype=torch.int64, device="cuda")
+    codes = lk.lookat_encode_keys(keys, books, near_ties=ties)
+    ev[2].record()
+    torch.cuda.synchronize()
+    fit_ms, enc_ms = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
+    del fit_keys
+
+    L = w.L
+    new_k = keys[:, :, L - 1:L].contiguous()              # the newest key of every (row, KV head)
+    out = torch.empty((w.B, w.n_q_heads, w.d_v), dtype=torch.float32, device="cuda")
+    lut = torch.empty((w.B, w.n_q_heads, w.m, w.K), dtype=torch.float32, device="cuda")
+
+    def step():
+        lk.lookat_encode_keys(new_k, books, codes=codes, pos=L - 1)
+        lk.lookat_build_lut(q, books, lut=lut)
+        lk.lookat_attend(codes, v, lut=lut, out=out, n_splits=args.splits)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    launches0 = lk.lookat_kernel_launches()
+    lk.lookat_set_timing(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    sampler.sample()
+    barrier()
+    sampler.stop()
+    lk.lookat_set_timing(False)
+    elapsed_ms = e0.elapsed_time(e1)
+    attend_ms = lk.lookat_attend_kernel_ms()
+    launches = lk.lookat_kernel_launches() - launches0
+    if world > 1:
+        t = torch.tensor([elapsed_ms, attend_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms, attend_ms = float(t[0]), float(t[1])
+
+    # ---- end to end: host buffers in, host buffer out, through the C-ABI call ----
+    q_host = torch.from_numpy(q_np).pin_memory()
+    k_host = new_k.reshape(w.B, w.n_kv_heads, w.d_k).cpu().pin_memory()
+    v_host = v[:, :, L - 1].contiguous().cpu().pin_memory()
+    out_host = torch.empty((w.B, w.n_q_heads, w.d_v), dtype=torch.float32).pin_memory()
+    for _ in range(3):
+        lk.lookat_decode_step_host(q_host, k_host, v_host, books, codes, v, L - 1, out_host, n_splits=args.splits)
+    barrier()
+    e2e_steps = args.steps
+    t0 = time.perf_counter()
+    e0.record()
+    for _ in range(e2e_steps):
+        lk.lookat_decode_step_host(q_host, k_host, v_host, books, codes, v, L - 1, out_host, n_splits=args.splits)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t[0])
+    same = bool(torch.allclose(out_host.cuda(), out, rtol=0, atol=1e-5))
+
+    if rank == 0:
+        units_per_step = w.B * w.n_q_heads * L * world
+        ms_per_step = elapsed_ms / args.steps
+        value = units_per_step / (ms_per_step * 1e-3)
+        peak, peak_kind = measured_peak_gbs()
+        alg_bytes = (w.m + 2 * w.d_v) * w.B * w.n_kv_heads * L           # per attend launch
+        achieved = alg_bytes / (attend_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(w),
+            "roofline": {"bound": "hbm", "kernel": "attend_stream_kernel", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
+                         "traffic": ATTEND_DRAM_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": alg_bytes,
+                         "kernel_ms": attend_ms, "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS},
+            "e2e": {"value": units_per_step / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": int(q_host.numel() * 2 + k_host.numel() * 2 + v_host.numel() * 2),
+                    "d2h_bytes_per_step": int(out_host.numel() * 4), "ms_per_step": e2e_ms / e2e_steps,
+                    "matches_device_path": same},
+            "gpu_launches": int(launches),
+            "clocks": sampler.summary(),
+            "step_hbm_gbs": (alg_bytes + lut.numel() * 8 + books.numel() * 4) / (ms_per_step * 1e-3) / 1e9,
+            "setup": {"fit_ms": fit_ms, "bulk_encode_ms": enc_ms,
+                      "bulk_encode_keys_per_s": w.B * w.n_kv_heads * L / (enc_ms * 1e-3),
+                      "near_ties": int(ties.item()), "input_generation_s": t_gen},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = time_oracle(w)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="lookat", choices=["lookat", "reference"])
+    ap.add_argument("--workload", default="gqa_32k_m8", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--splits", type=int, default=0, help="sequence chunks per row (0: library default)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_lookat(args, w)
+
+
+if __name__ == "__main__":
+    main()
