@@ -343,8 +343,12 @@ def main():
     ap.add_argument("--workload", default="gqa_32k_m8", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--splits", type=int, default=0, help="sequence chunks per row (0: library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the workload's batch size (smaller cases for profiler captures)")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
+    if args.batch > 0:
+        w = synth.Workload(**{**w.__dict__, "B": args.batch, "name": f"{w.name}_b{args.batch}"})
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -116,27 +116,15 @@ lookat_status attend_impl(Ctx *ctx, const float *lut, const void *q, const float
         lut = ctx->lut_scratch;
     }
 
-    int splits = n_splits > 0 ? n_splits : attend_auto_splits(ctx, B, L_max);
-    if (splits > L_max) splits = (int)L_max;
-    long long chunk = (L_max + splits - 1) / splits;
-    chunk = (chunk + 15) / 16 * 16;
-    splits = (int)((L_max + chunk - 1) / chunk);
-    if (splits > 65535) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "more than 65535 chunks");
     if ((long long)c.n_q_heads > 65535)
         return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "more than 65535 query heads");
-
-    const size_t rows = (size_t)B * c.n_q_heads * splits;
-    LOOKAT_TRY(ensure(ctx, (void **)&ctx->part_o, &ctx->part_o_cap, rows * c.d_v * sizeof(float), "partials"));
-    LOOKAT_TRY(ensure(ctx, (void **)&ctx->part_ml, &ctx->part_ml_cap, rows * 2 * sizeof(float), "partials"));
-
     AttendArgs a;
+    memset(&a, 0, sizeof(a));
     a.lut = lut;
     a.codes = codes;
     a.v = static_cast<const __half *>(v);
     a.seq_lens = seq_lens;
     a.uniform_len = (int)uniform_len;
-    a.part_o = ctx->part_o;
-    a.part_ml = ctx->part_ml;
     a.scores_out = scores_out;
     a.out = out;
     a.B = B;
@@ -147,9 +135,13 @@ lookat_status attend_impl(Ctx *ctx, const float *lut, const void *q, const float
     a.m = c.m;
     a.K = c.K;
     a.L_max = L_max;
-    a.chunk = (int)chunk;
-    a.n_splits = splits;
     a.scale_log2 = ctx->scale * 1.4426950408889634f;
+    size_t po = 0, pml = 0;
+    LOOKAT_TRY(plan_attend(ctx, a, n_splits, &po, &pml));
+    LOOKAT_TRY(ensure(ctx, (void **)&ctx->part_o, &ctx->part_o_cap, po * sizeof(float), "partials"));
+    LOOKAT_TRY(ensure(ctx, (void **)&ctx->part_ml, &ctx->part_ml_cap, pml * sizeof(float), "partials"));
+    a.part_o = ctx->part_o;
+    a.part_ml = ctx->part_ml;
     LOOKAT_TRY(launch_attend(ctx, a));
     return launch_combine(ctx, a);
 }

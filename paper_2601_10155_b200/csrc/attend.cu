@@ -1,21 +1,27 @@
 // Fused ADC scoring + online softmax + value accumulation (Section 3.5 "Lookup
-// and Sum"; Algorithm 1, second loop and continuation), split over sequence
-// chunks, plus the merge of the chunk partials.
+// and Sum"; Algorithm 1, second loop and continuation), split over the
+// sequence, plus the merge of the partial results.
 //
-// Streaming kernel (attend_stream_kernel), one CTA per (chunk, KV head x head
-// group, batch row); each of its 8 warps walks 16-token tiles on its own:
-//   * codes and V go from global memory straight to registers with 16-byte
-//     loads, one tile ahead of the arithmetic (V is ~97 % of the bytes; nothing
-//     is reused, so it is never staged in shared memory),
-//   * the query group's tables sit in shared memory, one padded table set per
-//     head; a lane scores two (token, head) pairs per tile by m gathers each,
+// Streaming kernel (attend_stream_kernel).  Work is the flat sequence of
+// (unit, 16-token tile) pairs, unit = (batch row, KV head, group of <= 4 query
+// heads sharing that KV head); each persistent CTA owns one contiguous range of
+// it, so all CTAs stream the same number of bytes and the tables are reloaded
+// only where a range crosses into the next unit.  Inside a CTA the 16 warps take
+// tiles round-robin and never wait for each other in the token loop:
+//   * V rows and codes travel global -> shared memory with 16-byte cp.async
+//     into a private ring of STAGES tiles per warp (rows padded by 16 bytes so
+//     that the fragment reads are bank-conflict free); a warp moves a landed
+//     tile into registers and refills its slot at once, so close to STAGES
+//     tiles of about 4 KB stay in flight per warp,
+//   * the unit's tables sit in shared memory, one set per head, sets shifted by
+//     8 banks; a lane scores two (token, head) pairs per tile, m gathers each,
 //   * the weighted value sum  O^T[d_v x heads] += V^T[d_v x 16 tokens] . P[16 x heads]
 //     runs on the tensor cores (mma.sync m16n8k16, fp16 in, fp32 accumulate).
-//     The 8 columns hold the <= 4 heads of the group twice: the fp16 rounding of
-//     each weight and the fp16 rounding of its remainder, so weights carry
-//     ~22 bits.  The token-pair operand layout is produced from the row-major V
-//     registers by byte permutes.
-// Up to 4 query heads of a KV head share one pass over that head's codes and V.
+//     The 8 columns hold the <= 4 heads twice: the fp16 rounding of each weight
+//     and the fp16 rounding of its remainder, so weights carry ~22 bits.  The
+//     token-pair operand layout comes from the row-major V rows by byte permutes.
+// A warp writes one partial (max, sum, weighted values) per unit it touched;
+// combine_stream_kernel merges the partials of every (batch row, query head).
 //
 // Generic kernel (attend_generic_kernel): any shape, plain loads, tables read
 // from global memory; used where the streaming kernel's layout assumptions
@@ -26,19 +32,22 @@ namespace lookat {
 
 namespace {
 
-constexpr int kWarps = 8;
+constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
 constexpr int kTile = 16;           // tokens per warp step (the MMA's k extent)
 constexpr int kHeadPad = 8;         // floats between the table sets of two heads (bank shift)
 constexpr float kNegBig = -1.0e30f; // running-max start: finite, so differences never give NaN
 
-__device__ __forceinline__ uint4 ldg_stream16(const void *p)
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
 {
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::128B.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-                 : "l"(p));
-    return r;
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global.L2::128B [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
 __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
@@ -70,7 +79,7 @@ struct CodePair {                    // the codes of two consecutive tokens
 };
 
 template <int M_SUB>
-__device__ __forceinline__ CodePair<M_SUB> load_code_pair(const uint8_t *p)
+__device__ __forceinline__ CodePair<M_SUB> read_code_pair(const unsigned char *p)
 {
     CodePair<M_SUB> c;
     if constexpr (M_SUB == 16) {
@@ -99,103 +108,135 @@ __device__ __forceinline__ int code_at(const CodePair<M_SUB> &c, int token01, in
     return (c.w[byte >> 2] >> (8 * (byte & 3))) & 0xff;
 }
 
-template <int DV>
-struct VTile {                       // 4 tokens x (DV/64) 16-byte pieces per lane
-    uint4 r[DV / 64][4];
+// Position in the flat tile sequence: tile `lt` of unit `unit`, with that unit's row facts.
+struct TileCursor {
+    long long T;         // flat index
+    int unit, lt;
+    int b, kvh;          // batch row and KV head of the unit
+    int len;             // tokens in that batch row (0 beyond the last unit)
 };
 
-template <int M_SUB, int DV>
-__global__ void __launch_bounds__(kThreads, 2) attend_stream_kernel(AttendArgs a)
+__device__ __forceinline__ void cursor_enter_unit(const AttendArgs &a, TileCursor &c, int hgroups)
 {
-    extern __shared__ __align__(16) float smem[];
+    const int kv_row = c.unit / hgroups;
+    c.b = kv_row / a.H_kv;
+    c.kvh = kv_row - c.b * a.H_kv;
+    c.len = c.unit < a.n_units
+                ? (int)min((long long)(a.seq_lens ? a.seq_lens[c.b] : a.uniform_len), a.L_max)
+                : 0;
+}
 
-    const int split = blockIdx.x;
-    const int hgroups = (a.g + 3) >> 2;
-    const int kvh = blockIdx.y / hgroups;
-    const int hgrp = blockIdx.y % hgroups;
-    const int b = blockIdx.z;
+__device__ __forceinline__ TileCursor cursor_at(const AttendArgs &a, long long T, int hgroups)
+{
+    TileCursor c;
+    c.T = T;
+    c.unit = (int)(T / a.tiles_per_unit);
+    c.lt = (int)(T - (long long)c.unit * a.tiles_per_unit);
+    cursor_enter_unit(a, c, hgroups);
+    return c;
+}
+
+__device__ __forceinline__ void cursor_advance(const AttendArgs &a, TileCursor &c, int step, int hgroups)
+{
+    c.T += step;
+    c.lt += step;
+    if (c.lt >= a.tiles_per_unit) {
+        do {
+            c.lt -= a.tiles_per_unit;
+            c.unit += 1;
+        } while (c.lt >= a.tiles_per_unit);
+        cursor_enter_unit(a, c, hgroups);
+    }
+}
+
+// Tokens of the cursor's tile that exist (0..16).
+__device__ __forceinline__ int cursor_valid(const TileCursor &c)
+{
+    const int left = c.len - c.lt * kTile;
+    return left >= kTile ? kTile : (left > 0 ? left : 0);
+}
+
+template <int M_SUB, int DV, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    constexpr int ROW = DV * 2 + 16;                      // a V row plus 16 bytes of padding
+    constexpr int SLOT = kTile * ROW + kTile * M_SUB;     // V rows, then the tile's codes
+    constexpr int V_CHUNKS = kTile * DV * 2 / 512;        // 16-byte pieces per lane and tile
+
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int n = lane >> 2, q = lane & 3;
-    const int heads_here = min(4, a.g - hgrp * 4);        // query heads this CTA serves
-    const int hq0 = kvh * a.g + hgrp * 4;                 // first of them
-    const int hl = n & 3;                                 // head this lane scores
+    const int hl = n & 3;                                 // head (within the group) this lane scores
     const int part = n >> 2;                              // 0: weight, 1: its fp16 remainder
-    const bool head_ok = hl < heads_here;
-
-    const int seq_len = (int)min((long long)(a.seq_lens ? a.seq_lens[b] : a.uniform_len), a.L_max);
-    const long long chunk_lo = (long long)split * a.chunk;
-    const long long chunk_hi = min((long long)seq_len, chunk_lo + a.chunk);
-
+    const int hgroups = (a.g + 3) >> 2;
+    const int heads_max = a.g < 4 ? a.g : 4;
     const int table = M_SUB * a.K;                        // floats per head
     const int head_stride = table + kHeadPad;
+    const int lut_bytes = (heads_max * head_stride * 4 + 15) & ~15;
 
-    // ---- stage the tables of this head group ----
-    if (chunk_lo < chunk_hi) {
-        for (int h = 0; h < heads_here; ++h) {
-            const float *src = a.lut + ((size_t)b * a.H_q + hq0 + h) * table;
-            float *dst = smem + h * head_stride;
-            if ((table & 3) == 0) {
-                for (int i = tid; i < (table >> 2); i += kThreads)
-                    reinterpret_cast<float4 *>(dst)[i] = reinterpret_cast<const float4 *>(src)[i];
+    float *lut_s = reinterpret_cast<float *>(smem_raw);
+    unsigned char *ring = smem_raw + lut_bytes + (size_t)warp * STAGES * SLOT;
+    const float *my_table = lut_s + hl * head_stride;
+
+    // ---- this CTA's range of the flat tile sequence ----
+    long long T_lo, T_hi;
+    const long long c = blockIdx.x;
+    if (a.splits_per_unit > 0) {
+        const long long u = c / a.splits_per_unit, s = c - u * a.splits_per_unit;
+        T_lo = u * a.tiles_per_unit + s * a.tiles_per_cta;
+        T_hi = min((u + 1) * a.tiles_per_unit, T_lo + a.tiles_per_cta);
+    } else {
+        T_lo = c * a.tiles_per_cta;
+        T_hi = min((long long)a.n_units * a.tiles_per_unit, T_lo + a.tiles_per_cta);
+    }
+
+    // ---- producer: the cursor's tile into ring slot `slot` (always closes one copy group) ----
+    auto issue = [&](const TileCursor &pc, int slot) {
+        const int nv = pc.T < T_hi ? cursor_valid(pc) : 0;
+        if (nv > 0) {
+            const size_t row0 = ((size_t)pc.b * a.H_kv + pc.kvh) * a.L_max + (size_t)pc.lt * kTile;
+            const unsigned char *vsrc = reinterpret_cast<const unsigned char *>(a.v) + row0 * (DV * 2);
+            const unsigned char *csrc = a.codes + row0 * M_SUB;
+            unsigned char *dst = ring + slot * SLOT;
+            if (nv == kTile) {
+#pragma unroll
+                for (int it = 0; it < V_CHUNKS; ++it) {
+                    const int off = lane * 16 + it * 512;
+                    cp_async16(dst + (off / (DV * 2)) * ROW + (off % (DV * 2)), vsrc + off);
+                }
+                if (lane < M_SUB) cp_async16(dst + kTile * ROW + lane * 16, csrc + lane * 16);
             } else {
-                for (int i = tid; i < table; i += kThreads) dst[i] = src[i];
+                // ragged end of a row: rows at or beyond seq_len are never read, zeros stand in
+#pragma unroll
+                for (int it = 0; it < V_CHUNKS; ++it) {
+                    const int off = lane * 16 + it * 512;
+                    const int row = off / (DV * 2);
+                    unsigned char *d = dst + row * ROW + (off % (DV * 2));
+                    if (row < nv) cp_async16(d, vsrc + off);
+                    else *reinterpret_cast<uint4 *>(d) = make_uint4(0, 0, 0, 0);
+                }
+                if (lane < kTile) {
+#pragma unroll
+                    for (int j = 0; j < M_SUB; ++j)
+                        dst[kTile * ROW + lane * M_SUB + j] = lane < nv ? csrc[lane * M_SUB + j] : 0;
+                }
             }
         }
-    }
-    __syncthreads();
+        cp_async_commit();
+    };
 
-    const size_t kv_row = (size_t)b * a.H_kv + kvh;
-    const uint8_t *codes = a.codes + kv_row * a.L_max * M_SUB;
-    const __half *vbase = a.v + kv_row * a.L_max * DV;
-    const float *my_table = smem + hl * head_stride;
-    float *scores_row =
-        (a.scores_out && head_ok) ? a.scores_out + ((size_t)b * a.H_q + hq0 + hl) * a.L_max : nullptr;
-
+    // ---- running state of the unit being accumulated ----
     float acc[DV / 16][4];
-#pragma unroll
-    for (int i = 0; i < DV / 16; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
     float m_run = kNegBig, l_run = 0.f;
 
     // token offsets inside a tile: the two this lane scores, the four whose V it holds
     const int ts_off = 2 * q + 8 * part;
     const int tv_off[4] = {2 * q, 2 * q + 1, 2 * q + 8, 2 * q + 9};
 
-    auto load_tile = [&](long long t0, VTile<DV> &vt, CodePair<M_SUB> &cp) {
-        const bool full = t0 + kTile <= chunk_hi;
-        if (full) {
-            cp = load_code_pair<M_SUB>(codes + (t0 + ts_off) * M_SUB);
-#pragma unroll
-            for (int gI = 0; gI < DV / 64; ++gI)
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    vt.r[gI][k] = ldg_stream16(vbase + (t0 + tv_off[k]) * DV + gI * 64 + n * 8);
-        } else {
-            // ragged tail: never read a token at or beyond chunk_hi
-            if (t0 + ts_off + 1 < chunk_hi) {
-                cp = load_code_pair<M_SUB>(codes + (t0 + ts_off) * M_SUB);
-            } else {
-#pragma unroll
-                for (int i = 0; i < (2 * M_SUB + 3) / 4; ++i) cp.w[i] = 0;
-                if (t0 + ts_off < chunk_hi) {
-                    const uint8_t *p = codes + (t0 + ts_off) * M_SUB;
-#pragma unroll
-                    for (int j = 0; j < M_SUB; ++j) cp.w[j >> 2] |= (uint32_t)p[j] << (8 * (j & 3));
-                }
-            }
-#pragma unroll
-            for (int gI = 0; gI < DV / 64; ++gI)
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    if (t0 + tv_off[k] < chunk_hi)
-                        vt.r[gI][k] = ldg_stream16(vbase + (t0 + tv_off[k]) * DV + gI * 64 + n * 8);
-                    else
-                        vt.r[gI][k] = make_uint4(0, 0, 0, 0);
-                }
-        }
-    };
-
-    auto process_tile = [&](long long t0, const VTile<DV> &vt, const CodePair<M_SUB> &cp) {
+    // one tile, already in registers: vr = this lane's 16-byte V pieces, cp = its two tokens' codes
+    auto process_tile = [&](int t0, int nv, const uint4 (&vr)[DV / 64][4], const CodePair<M_SUB> &cp,
+                            bool head_ok, float *scores_row) {
         // ---- lookup-and-sum for this lane's two (token, head) pairs ----
         float s0 = 0.f, s1 = 0.f;
         if (head_ok) {
@@ -205,11 +246,10 @@ __global__ void __launch_bounds__(kThreads, 2) attend_stream_kernel(AttendArgs a
                 s1 += my_table[j * a.K + code_at<M_SUB>(cp, 1, j)];
             }
         }
-        const long long ts = t0 + ts_off;
-        const bool ok0 = head_ok && ts < chunk_hi, ok1 = head_ok && ts + 1 < chunk_hi;
+        const bool ok0 = head_ok && ts_off < nv, ok1 = head_ok && ts_off + 1 < nv;
         if (scores_row) {
-            if (ok0) scores_row[ts] = s0;
-            if (ok1) scores_row[ts + 1] = s1;
+            if (ok0) scores_row[t0 + ts_off] = s0;
+            if (ok1) scores_row[t0 + ts_off + 1] = s1;
         }
         const float x0 = ok0 ? s0 * a.scale_log2 : -INFINITY;
         const float x1 = ok1 ? s1 * a.scale_log2 : -INFINITY;
@@ -247,88 +287,147 @@ __global__ void __launch_bounds__(kThreads, 2) attend_stream_kernel(AttendArgs a
         // ---- O^T += V^T P on the tensor cores ----
 #pragma unroll
         for (int gI = 0; gI < DV / 64; ++gI) {
-            const uint32_t x[4] = {vt.r[gI][0].x, vt.r[gI][0].y, vt.r[gI][0].z, vt.r[gI][0].w};
-            const uint32_t y[4] = {vt.r[gI][1].x, vt.r[gI][1].y, vt.r[gI][1].z, vt.r[gI][1].w};
-            const uint32_t z[4] = {vt.r[gI][2].x, vt.r[gI][2].y, vt.r[gI][2].z, vt.r[gI][2].w};
-            const uint32_t w[4] = {vt.r[gI][3].x, vt.r[gI][3].y, vt.r[gI][3].z, vt.r[gI][3].w};
+            const uint32_t xs[4] = {vr[gI][0].x, vr[gI][0].y, vr[gI][0].z, vr[gI][0].w};
+            const uint32_t ys[4] = {vr[gI][1].x, vr[gI][1].y, vr[gI][1].z, vr[gI][1].w};
+            const uint32_t zs[4] = {vr[gI][2].x, vr[gI][2].y, vr[gI][2].z, vr[gI][2].w};
+            const uint32_t ws[4] = {vr[gI][3].x, vr[gI][3].y, vr[gI][3].z, vr[gI][3].w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint32_t a0 = __byte_perm(x[i], y[i], 0x5410);   // dv even, tokens 2q,2q+1
-                const uint32_t a1 = __byte_perm(x[i], y[i], 0x7632);   // dv odd
-                const uint32_t a2 = __byte_perm(z[i], w[i], 0x5410);   // tokens 2q+8,2q+9
-                const uint32_t a3 = __byte_perm(z[i], w[i], 0x7632);
+                const uint32_t a0 = __byte_perm(xs[i], ys[i], 0x5410);   // dv even, tokens 2q,2q+1
+                const uint32_t a1 = __byte_perm(xs[i], ys[i], 0x7632);   // dv odd
+                const uint32_t a2 = __byte_perm(zs[i], ws[i], 0x5410);   // tokens 2q+8,2q+9
+                const uint32_t a3 = __byte_perm(zs[i], ws[i], 0x7632);
                 mma_16816(acc[gI * 4 + i], a0, a1, a2, a3, b0, b1);
             }
         }
     };
 
-    // ---- walk this warp's tiles, loads one tile ahead ----
-    const long long stride = (long long)kWarps * kTile;
-    long long t0 = chunk_lo + (long long)warp * kTile;
-    VTile<DV> vA, vB;
-    CodePair<M_SUB> cA, cB;
-    if (t0 < chunk_hi) load_tile(t0, vA, cA);
-    while (t0 < chunk_hi) {
-        const long long t1 = t0 + stride;
-        if (t1 < chunk_hi) load_tile(t1, vB, cB);
-        process_tile(t0, vA, cA);
-        if (t1 >= chunk_hi) break;
-        const long long t2 = t1 + stride;
-        if (t2 < chunk_hi) load_tile(t2, vA, cA);
-        process_tile(t1, vB, cB);
-        t0 = t2;
+    // ---- prologue: fill the ring with this warp's first STAGES tiles ----
+    TileCursor cc = cursor_at(a, T_lo + warp, hgroups);   // tile this warp consumes next
+    TileCursor pc = cc;                                   // tile it copies next
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) {
+        issue(pc, s);
+        cursor_advance(a, pc, kWarps, hgroups);
     }
+    int slot = 0;                                          // ring slot of the consumer's tile
 
-    // ---- fold the weight and remainder columns, reduce l over the head's lanes ----
-#pragma unroll
-    for (int i = 0; i < DV / 16; ++i)
-#pragma unroll
-        for (int k = 0; k < 4; ++k) acc[i][k] += __shfl_xor_sync(0xffffffffu, acc[i][k], 2);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);
+    // ---- one pass per unit this CTA's range touches ----
+    const int unit_first = (int)(T_lo / a.tiles_per_unit);
+    const int unit_last = T_hi > T_lo ? (int)((T_hi - 1) / a.tiles_per_unit) : unit_first - 1;
+    for (int unit = unit_first; unit <= unit_last; ++unit) {
+        const int hgrp = unit % hgroups;
+        const int kv_row = unit / hgroups;
+        const int b = kv_row / a.H_kv, kvh = kv_row - b * a.H_kv;
+        const int heads_here = min(4, a.g - hgrp * 4);
+        const int hq0 = kvh * a.g + hgrp * 4;
+        const bool head_ok = hl < heads_here;
 
-    // ---- merge the 8 warps through shared memory (the tables are no longer needed) ----
-    __syncthreads();
-    float *w_o = smem;                                   // [kWarps][4][DV]
-    float *w_m = smem + kWarps * 4 * DV;                 // [kWarps][4]
-    float *w_l = w_m + kWarps * 4;                       // [kWarps][4]
-    if (q < 2) {
+        __syncthreads();                                   // every warp is done with the previous tables
+        for (int h = 0; h < heads_here; ++h) {
+            const float *src = a.lut + ((size_t)b * a.H_q + hq0 + h) * table;
+            float *dst = lut_s + h * head_stride;
+            if ((table & 3) == 0) {
+                for (int i = tid; i < (table >> 2); i += kThreads)
+                    reinterpret_cast<float4 *>(dst)[i] = __ldg(reinterpret_cast<const float4 *>(src) + i);
+            } else {
+                for (int i = tid; i < table; i += kThreads) dst[i] = __ldg(src + i);
+            }
+        }
+        __syncthreads();
+
 #pragma unroll
-        for (int i = 0; i < DV / 16; ++i) {
-            const int dv = (i >> 2) * 64 + n * 8 + 2 * (i & 3);
-            float *o = w_o + (warp * 4 + 2 * q) * DV + dv;
-            o[0] = acc[i][0];          // (dv, head 2q)
-            o[DV] = acc[i][1];         // (dv, head 2q+1)
-            o[1] = acc[i][2];          // (dv+1, head 2q)
-            o[DV + 1] = acc[i][3];     // (dv+1, head 2q+1)
+        for (int i = 0; i < DV / 16; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+        m_run = kNegBig;
+        l_run = 0.f;
+        float *scores_row =
+            (a.scores_out && head_ok) ? a.scores_out + ((size_t)b * a.H_q + hq0 + hl) * a.L_max : nullptr;
+
+        const long long seg_hi = min(T_hi, (long long)(unit + 1) * a.tiles_per_unit);
+        while (cc.T < seg_hi) {
+            cp_async_wait<STAGES - 1>();                   // this lane's copies of the tile have landed
+            __syncwarp();                                  // ... and every other lane's
+            const int nv = cursor_valid(cc);
+            const unsigned char *sl = ring + slot * SLOT;
+            uint4 vr[DV / 64][4];
+            CodePair<M_SUB> cp;
+            if (nv > 0) {                                  // tile -> registers, so the slot can be refilled
+                cp = read_code_pair<M_SUB>(sl + kTile * ROW + ts_off * M_SUB);
+#pragma unroll
+                for (int gI = 0; gI < DV / 64; ++gI)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        vr[gI][k] = *reinterpret_cast<const uint4 *>(sl + tv_off[k] * ROW + gI * 128 + n * 16);
+            }
+            __syncwarp();                                  // all lanes have read the slot
+            issue(pc, slot);
+            cursor_advance(a, pc, kWarps, hgroups);
+            if (nv > 0) process_tile(cc.lt * kTile, nv, vr, cp, head_ok, scores_row);
+            slot = slot + 1 == STAGES ? 0 : slot + 1;
+            cursor_advance(a, cc, kWarps, hgroups);
+        }
+
+        // ---- this warp's partial for the unit: fold the weight and remainder columns ----
+#pragma unroll
+        for (int i = 0; i < DV / 16; ++i)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) acc[i][k] += __shfl_xor_sync(0xffffffffu, acc[i][k], 2);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);
+
+        const size_t pslot = ((size_t)(c + unit) * kWarps + warp) * 4;     // + head
+        if (q < 2) {
+#pragma unroll
+            for (int i = 0; i < DV / 16; ++i) {
+                const int dv = (i >> 2) * 64 + n * 8 + 2 * (i & 3);
+                float *o = a.part_o + (pslot + 2 * q) * DV + dv;
+                *reinterpret_cast<float2 *>(o) = make_float2(acc[i][0], acc[i][2]);         // head 2q
+                *reinterpret_cast<float2 *>(o + DV) = make_float2(acc[i][1], acc[i][3]);    // head 2q+1
+            }
+        }
+        if (q == 0 && part == 0) {
+            a.part_ml[(pslot + hl) * 2] = m_run;
+            a.part_ml[(pslot + hl) * 2 + 1] = l_run;
         }
     }
-    if (q == 0 && part == 0) {
-        w_m[warp * 4 + hl] = m_run;
-        w_l[warp * 4 + hl] = l_run;
-    }
-    __syncthreads();
+    cp_async_wait<0>();
+}
 
-    for (int idx = tid; idx < heads_here * DV; idx += kThreads) {
-        const int h = idx / DV, dv = idx % DV;
-        float M = kNegBig;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, w_m[w * 4 + h]);
-        float o = 0.f, l = 0.f;
-#pragma unroll
+// Merge of the streaming kernel's partials for one (batch row, query head):
+// M = max_i M_i, l = sum l_i 2^(M_i-M), o = sum o_i 2^(M_i-M) / l over every (CTA, warp) that
+// touched the row's unit.  Partials without tokens carry l = 0 and add nothing.
+template <int DV>
+__global__ void __launch_bounds__(DV) combine_stream_kernel(AttendArgs a)
+{
+    const int row = blockIdx.x;                         // b * H_q + hq
+    const int b = row / a.H_q, hq = row - b * a.H_q;
+    const int kvh = hq / a.g, hin = hq - kvh * a.g;
+    const int hgroups = (a.g + 3) >> 2;
+    const int unit = (b * a.H_kv + kvh) * hgroups + (hin >> 2);
+    const int hl = hin & 3;
+    long long c_lo, c_hi;
+    if (a.splits_per_unit > 0) {
+        c_lo = (long long)unit * a.splits_per_unit;
+        c_hi = c_lo + a.splits_per_unit - 1;
+    } else {
+        c_lo = (long long)unit * a.tiles_per_unit / a.tiles_per_cta;
+        c_hi = ((long long)(unit + 1) * a.tiles_per_unit - 1) / a.tiles_per_cta;
+    }
+    const int dv = threadIdx.x;
+    float M = kNegBig;
+    for (long long c = c_lo; c <= c_hi; ++c)
+        for (int w = 0; w < kWarps; ++w)
+            M = fmaxf(M, a.part_ml[((((size_t)(c + unit) * kWarps + w) * 4) + hl) * 2]);
+    float l = 0.f, o = 0.f;
+    for (long long c = c_lo; c <= c_hi; ++c)
         for (int w = 0; w < kWarps; ++w) {
-            const float f = ex2_approx(w_m[w * 4 + h] - M);
-            o += f * w_o[(w * 4 + h) * DV + dv];
-            l += f * w_l[w * 4 + h];
+            const size_t p = ((size_t)(c + unit) * kWarps + w) * 4 + hl;
+            const float f = ex2_approx(a.part_ml[p * 2] - M);
+            l += f * a.part_ml[p * 2 + 1];
+            o += f * a.part_o[p * DV + dv];
         }
-        const size_t row = ((size_t)b * a.H_q + hq0 + h) * a.n_splits + split;
-        a.part_o[row * DV + dv] = o;
-        if (dv == 0) {
-            a.part_ml[row * 2] = M;
-            a.part_ml[row * 2 + 1] = l;
-        }
-    }
+    a.out[(size_t)row * DV + dv] = l > 0.f ? o / l : 0.f;
 }
 
 // Any shape.  One CTA per (chunk, query head, batch row); 128 threads.
@@ -363,9 +462,9 @@ __global__ void __launch_bounds__(kGenThreads) attend_generic_kernel(AttendArgs 
         const int cnt = (int)min((long long)kGenBlockTokens, chunk_hi - blk);
         float mloc = -INFINITY;
         for (int t = tid; t < cnt; t += kGenThreads) {
-            const uint8_t *c = codes + (blk + t) * a.m;
+            const uint8_t *cd = codes + (blk + t) * a.m;
             float s = 0.f;
-            for (int j = 0; j < a.m; ++j) s += __ldg(lut + j * a.K + c[j]);
+            for (int j = 0; j < a.m; ++j) s += __ldg(lut + j * a.K + cd[j]);
             if (scores_row) scores_row[blk + t] = s;
             const float x = s * a.scale_log2;
             xs[t] = x;
@@ -418,9 +517,8 @@ __global__ void __launch_bounds__(kGenThreads) attend_generic_kernel(AttendArgs 
     }
 }
 
-// Merge of the chunk partials: M = max_i M_i, l = sum l_i 2^(M_i-M),
-// o = sum o_i 2^(M_i-M) / l.  A chunk without tokens carries l = 0 and adds nothing.
-__global__ void combine_kernel(AttendArgs a)
+// Merge of the generic kernel's chunk partials.
+__global__ void combine_generic_kernel(AttendArgs a)
 {
     const size_t row = blockIdx.x;                      // b * H_q + hq
     const float *ml = a.part_ml + row * a.n_splits * 2;
@@ -437,66 +535,132 @@ __global__ void combine_kernel(AttendArgs a)
     }
 }
 
-template <int M_SUB, int DV>
-lookat_status launch_stream(Ctx *ctx, const AttendArgs &a)
-{
-    const int hgroups = (a.g + 3) / 4;
-    const int heads = a.g < 4 ? a.g : 4;
-    size_t lut_bytes = (size_t)heads * (M_SUB * a.K + kHeadPad) * sizeof(float);
-    size_t merge_bytes = (size_t)(kWarps * 4 * DV + 2 * kWarps * 4) * sizeof(float);
-    size_t smem = lut_bytes > merge_bytes ? lut_bytes : merge_bytes;
-    auto kern = attend_stream_kernel<M_SUB, DV>;
-    if (smem > 48 * 1024) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return check_launch(ctx, "attend: shared-memory opt-in");
-    }
-    dim3 grid(a.n_splits, a.H_kv * hgroups, a.B);
-    kern<<<grid, kThreads, smem, ctx->stream>>>(a);
-    return check_launch(ctx, "attend_stream_kernel");
-}
-
-template <int M_SUB>
-lookat_status launch_stream_dv(Ctx *ctx, const AttendArgs &a)
-{
-    if (a.d_v == 64) return launch_stream<M_SUB, 64>(ctx, a);
-    return launch_stream<M_SUB, 128>(ctx, a);
-}
-
-}  // namespace
-
-bool attend_fast_path(const Ctx *ctx, const void *codes, const void *v, long long L_max)
+// ---- host side: kernel choice, decomposition, launches ----
+bool stream_shape_ok(const Ctx *ctx, const AttendArgs &a)
 {
     const lookat_config &c = ctx->cfg;
     const bool m_ok = c.m == 1 || c.m == 2 || c.m == 4 || c.m == 8 || c.m == 16;
     const bool dv_ok = c.d_v == 64 || c.d_v == 128;
-    const int heads = c.n_q_heads / c.n_kv_heads < 4 ? c.n_q_heads / c.n_kv_heads : 4;
-    const size_t lut_bytes = (size_t)heads * (c.m * c.K + kHeadPad) * sizeof(float);
-    // rows of the code cache must start on a 16-byte boundary for the vector loads
-    const bool rows_ok = (L_max * c.m) % 16 == 0 && ((uintptr_t)codes % 16) == 0 && ((uintptr_t)v % 16) == 0;
-    return m_ok && dv_ok && rows_ok && lut_bytes <= (size_t)ctx->max_smem_optin;
+    // rows of the code cache and of V must start on 16-byte boundaries for the 16-byte copies
+    const bool rows_ok = (a.L_max * c.m) % 16 == 0 && ((uintptr_t)a.codes % 16) == 0 &&
+                         ((uintptr_t)a.v % 16) == 0 && ((uintptr_t)a.lut % 16) == 0;
+    return m_ok && dv_ok && rows_ok;
 }
 
-int attend_auto_splits(const Ctx *ctx, int B, long long L_max)
+size_t stream_smem_bytes(const AttendArgs &a, int stages)
 {
-    const lookat_config &c = ctx->cfg;
-    const int g = c.n_q_heads / c.n_kv_heads;
-    const long long units = (long long)B * c.n_kv_heads * ((g + 3) / 4);
-    const long long resident = 2LL * ctx->sm_count;            // CTAs resident at once
-    long long max_splits = L_max / 256;                         // keep chunks >= 256 tokens
-    if (max_splits < 1) max_splits = 1;
-    long long want = (8 * resident + units - 1) / units;        // about 8 waves of CTAs
-    if (want < 1) want = 1;
-    long long n = want < max_splits ? want : max_splits;
-    // prefer a CTA count that is a whole number of waves
-    for (long long cand = n; cand <= max_splits && cand <= n + 8; ++cand)
-        if ((units * cand) % resident == 0) { n = cand; break; }
-    if (n > 4096) n = 4096;
-    return (int)n;
+    const int heads = a.g < 4 ? a.g : 4;
+    const size_t lut_bytes = ((size_t)heads * (a.m * a.K + kHeadPad) * 4 + 15) & ~(size_t)15;
+    const size_t slot = (size_t)kTile * (a.d_v * 2 + 16) + (size_t)kTile * a.m;
+    return lut_bytes + (size_t)kWarps * stages * slot;
+}
+
+int stream_stages(const Ctx *ctx, const AttendArgs &a)
+{
+    const int options[2] = {4, 2};
+    for (int s : options)
+        if (stream_smem_bytes(a, s) <= (size_t)ctx->max_smem_optin) return s;
+    return 0;
+}
+
+template <int M_SUB, int DV, int STAGES>
+lookat_status stream_kernel_ready(Ctx *ctx, const AttendArgs &a, int *ctas_per_sm)
+{
+    auto kern = attend_stream_kernel<M_SUB, DV, STAGES>;
+    const size_t smem = stream_smem_bytes(a, STAGES);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return check_launch(ctx, "attend: shared-memory opt-in");
+    int nb = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, kThreads, smem) != cudaSuccess || nb < 1)
+        return set_error(ctx, LOOKAT_ERR_CUDA, "attend: the streaming kernel does not fit on an SM");
+    *ctas_per_sm = nb;
+    return LOOKAT_OK;
+}
+
+template <int M_SUB, int DV, int STAGES>
+lookat_status stream_launch(Ctx *ctx, const AttendArgs &a)
+{
+    attend_stream_kernel<M_SUB, DV, STAGES>
+        <<<a.n_ctas, kThreads, stream_smem_bytes(a, STAGES), ctx->stream>>>(a);
+    return check_launch(ctx, "attend_stream_kernel");
+}
+
+// Calls f.template operator()<M_SUB, DV, STAGES>() for the runtime (m, d_v, stages).
+template <typename F>
+lookat_status dispatch_stream(int m, int d_v, int stages, F &&f)
+{
+#define LOOKAT_CASE(M, D, S) \
+    if (m == M && d_v == D && stages == S) return f.template operator()<M, D, S>();
+#define LOOKAT_CASES(M) \
+    LOOKAT_CASE(M, 64, 4) LOOKAT_CASE(M, 64, 2) LOOKAT_CASE(M, 128, 4) LOOKAT_CASE(M, 128, 2)
+    LOOKAT_CASES(1) LOOKAT_CASES(2) LOOKAT_CASES(4) LOOKAT_CASES(8) LOOKAT_CASES(16)
+#undef LOOKAT_CASES
+#undef LOOKAT_CASE
+    return LOOKAT_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_floats, size_t *part_ml_floats)
+{
+    const int stages = stream_shape_ok(ctx, a) ? stream_stages(ctx, a) : 0;
+    if (stages) {
+        const int hgroups = (a.g + 3) / 4;
+        const long long units = (long long)a.B * a.H_kv * hgroups;
+        const long long tpu = (a.L_max + kTile - 1) / kTile;
+        if (units > (1ll << 30) || units * tpu > (1ll << 40))
+            return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "attend: problem too large");
+        int per_sm = 0;
+        lookat_status st = dispatch_stream(a.m, a.d_v, stages, [&]<int M, int D, int S>() {
+            return stream_kernel_ready<M, D, S>(ctx, a, &per_sm);
+        });
+        if (st != LOOKAT_OK) return st;
+        a.stream = 1;
+        a.n_units = (int)units;
+        a.tiles_per_unit = (int)tpu;
+        if (n_splits > 0) {
+            long long splits = n_splits < tpu ? n_splits : tpu;
+            a.tiles_per_cta = (tpu + splits - 1) / splits;
+            splits = (tpu + a.tiles_per_cta - 1) / a.tiles_per_cta;
+            if (units * splits > (1ll << 30)) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "attend: too many chunks");
+            a.splits_per_unit = (int)splits;
+            a.n_ctas = (int)(units * splits);
+        } else {
+            const long long total = units * tpu;
+            long long ctas = (long long)per_sm * ctx->sm_count;
+            if (ctas > total) ctas = total;
+            a.tiles_per_cta = (total + ctas - 1) / ctas;
+            a.splits_per_unit = 0;
+            a.n_ctas = (int)((total + a.tiles_per_cta - 1) / a.tiles_per_cta);
+        }
+        const size_t slots = (size_t)a.n_ctas + (size_t)a.n_units;
+        *part_o_floats = slots * kWarps * 4 * a.d_v;
+        *part_ml_floats = slots * kWarps * 4 * 2;
+        return LOOKAT_OK;
+    }
+    // generic kernel: chunks of whole 16-token groups, at least 256 tokens unless asked otherwise
+    a.stream = 0;
+    long long splits = n_splits;
+    if (splits <= 0) {
+        const long long rows = (long long)a.B * a.H_q;
+        splits = (4ll * ctx->sm_count + rows - 1) / rows;
+        const long long max_splits = a.L_max / 256 > 0 ? a.L_max / 256 : 1;
+        if (splits > max_splits) splits = max_splits;
+    }
+    if (splits > a.L_max) splits = a.L_max;
+    long long chunk = (a.L_max + splits - 1) / splits;
+    chunk = (chunk + 15) / 16 * 16;
+    splits = (a.L_max + chunk - 1) / chunk;
+    if (splits > 65535) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "attend: more than 65535 chunks");
+    a.chunk = (int)chunk;
+    a.n_splits = (int)splits;
+    *part_o_floats = (size_t)a.B * a.H_q * splits * a.d_v;
+    *part_ml_floats = (size_t)a.B * a.H_q * splits * 2;
+    return LOOKAT_OK;
 }
 
 lookat_status launch_attend(Ctx *ctx, const AttendArgs &a)
 {
-    const bool fast = attend_fast_path(ctx, a.codes, a.v, a.L_max);
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (ctx->timing) {
         const int s = ctx->ev_next;
@@ -514,14 +678,10 @@ lookat_status launch_attend(Ctx *ctx, const AttendArgs &a)
         cudaEventRecord(e0, ctx->stream);
     }
     lookat_status st;
-    if (fast) {
-        switch (a.m) {
-            case 1: st = launch_stream_dv<1>(ctx, a); break;
-            case 2: st = launch_stream_dv<2>(ctx, a); break;
-            case 4: st = launch_stream_dv<4>(ctx, a); break;
-            case 8: st = launch_stream_dv<8>(ctx, a); break;
-            default: st = launch_stream_dv<16>(ctx, a); break;
-        }
+    if (a.stream) {
+        st = dispatch_stream(a.m, a.d_v, stream_stages(ctx, a), [&]<int M, int D, int S>() {
+            return stream_launch<M, D, S>(ctx, a);
+        });
     } else {
         dim3 grid(a.n_splits, a.H_q, a.B);
         attend_generic_kernel<<<grid, kGenThreads, 0, ctx->stream>>>(a);
@@ -537,9 +697,14 @@ lookat_status launch_attend(Ctx *ctx, const AttendArgs &a)
 
 lookat_status launch_combine(Ctx *ctx, const AttendArgs &a)
 {
+    if (a.stream) {
+        if (a.d_v == 64) combine_stream_kernel<64><<<a.B * a.H_q, 64, 0, ctx->stream>>>(a);
+        else combine_stream_kernel<128><<<a.B * a.H_q, 128, 0, ctx->stream>>>(a);
+        return check_launch(ctx, "combine_stream_kernel");
+    }
     int threads = a.d_v < 32 ? 32 : (a.d_v > 256 ? 256 : ((a.d_v + 31) / 32) * 32);
-    combine_kernel<<<a.B * a.H_q, threads, 0, ctx->stream>>>(a);
-    return check_launch(ctx, "combine_kernel");
+    combine_generic_kernel<<<a.B * a.H_q, threads, 0, ctx->stream>>>(a);
+    return check_launch(ctx, "combine_generic_kernel");
 }
 
 }  // namespace lookat

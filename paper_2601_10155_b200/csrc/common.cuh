@@ -26,10 +26,10 @@ struct Ctx {
     // attend scratch: chunk partials  o [B][H_q][splits][d_v], (M, l) [B][H_q][splits][2]
     float *part_o;
     float *part_ml;
-    size_t part_o_cap, part_ml_cap;       // in floats
+    size_t part_o_cap, part_ml_cap;       // bytes
     // tables built on behalf of the caller (lookat_attend with lut == NULL)
     float *lut_scratch;
-    size_t lut_cap;                        // in floats
+    size_t lut_cap;                        // bytes
     // k-means scratch
     unsigned long long *fit_sums;          // [H_kv][m][K][d_sub] fixed-point sums
     unsigned long long *fit_cnt;           // [H_kv][m][K]
@@ -66,15 +66,23 @@ struct AttendArgs {
     float *out;                // [B][H_q][d_v]
     int B, H_q, H_kv, g, d_v, m, K;
     long long L_max;
-    int chunk;                 // tokens per split (multiple of 16)
-    int n_splits;
+    // generic kernel: one CTA per (chunk, query head, batch row)
+    int chunk;                 // tokens per chunk (multiple of 16)
+    int n_splits;              // chunks per row
+    // streaming kernel: the (unit, 16-token tile) pairs form one flat sequence, unit =
+    // (batch row, KV head, group of <= 4 query heads); CTA c owns a contiguous range of it
+    int stream;                // 1: streaming kernel and its partial layout
+    int n_units;
+    int tiles_per_unit;        // ceil(L_max / 16)
+    long long tiles_per_cta;
+    int n_ctas;
+    int splits_per_unit;       // > 0: CTA c = chunk c % splits of unit c / splits; 0: flat ranges
     float scale_log2;          // scale * log2(e)
 };
 
-// Chooses the number of sequence chunks for a launch (n_splits == 0 in the API).
-int attend_auto_splits(const Ctx *ctx, int B, long long L_max);
-// True when the tensor-core streaming kernel covers this shape.
-bool attend_fast_path(const Ctx *ctx, const void *codes, const void *v, long long L_max);
+// Fills the decomposition fields of `a` (kernel choice, chunking) for n_splits as given to the
+// API (0 = library's choice) and returns the partial-buffer sizes in floats.
+lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_floats, size_t *part_ml_floats);
 lookat_status launch_attend(Ctx *ctx, const AttendArgs &a);
 lookat_status launch_combine(Ctx *ctx, const AttendArgs &a);
 
