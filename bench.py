@@ -240,12 +240,11 @@ def run_lookat(args, w):
     L = w.L
     new_k = keys[:, :, L - 1:L].contiguous()              # the newest key of every (row, KV head)
     out = torch.empty((w.B, w.n_q_heads, w.d_v), dtype=torch.float32, device="cuda")
-    lut = torch.empty((w.B, w.n_q_heads, w.m, w.K), dtype=torch.float32, device="cuda")
 
     def step():
+        # append: encode the newest key; then Algorithm 1 (tables, lookup-sum, softmax, value sum)
         lk.lookat_encode_keys(new_k, books, codes=codes, pos=L - 1)
-        lk.lookat_build_lut(q, books, lut=lut)
-        lk.lookat_attend(codes, v, lut=lut, out=out, n_splits=args.splits)
+        lk.lookat_attend(codes, v, q=q, codebooks=books, out=out, n_splits=args.splits)
 
     def barrier():
         torch.cuda.synchronize()
@@ -321,7 +320,7 @@ def run_lookat(args, w):
                     "matches_device_path": same},
             "gpu_launches": int(launches),
             "clocks": sampler.summary(),
-            "step_hbm_gbs": (alg_bytes + lut.numel() * 8 + books.numel() * 4) / (ms_per_step * 1e-3) / 1e9,
+            "step_hbm_gbs": (alg_bytes + books.numel() * 4) / (ms_per_step * 1e-3) / 1e9,
             "setup": {"fit_ms": fit_ms, "bulk_encode_ms": enc_ms,
                       "bulk_encode_keys_per_s": w.B * w.n_kv_heads * L / (enc_ms * 1e-3),
                       "near_ties": int(ties.item()), "input_generation_s": t_gen},

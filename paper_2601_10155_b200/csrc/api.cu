@@ -109,18 +109,14 @@ lookat_status attend_impl(Ctx *ctx, const float *lut, const void *q, const float
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return set_error(ctx, LOOKAT_ERR_CUDA, "cannot select device %d", ctx->device);
 
-    if (!lut) {
-        const size_t need = (size_t)B * c.n_q_heads * c.m * c.K * sizeof(float);
-        LOOKAT_TRY(ensure(ctx, (void **)&ctx->lut_scratch, &ctx->lut_cap, need, "table scratch"));
-        LOOKAT_TRY(launch_build_lut(ctx, static_cast<const __half *>(q), B, codebooks, ctx->lut_scratch));
-        lut = ctx->lut_scratch;
-    }
-
     if ((long long)c.n_q_heads > 65535)
         return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "more than 65535 query heads");
     AttendArgs a;
     memset(&a, 0, sizeof(a));
     a.lut = lut;
+    a.q = static_cast<const __half *>(q);
+    a.codebooks = codebooks;
+    a.d_k = c.d_k;
     a.codes = codes;
     a.v = static_cast<const __half *>(v);
     a.seq_lens = seq_lens;
@@ -138,10 +134,28 @@ lookat_status attend_impl(Ctx *ctx, const float *lut, const void *q, const float
     a.scale_log2 = ctx->scale * 1.4426950408889634f;
     size_t po = 0, pml = 0;
     LOOKAT_TRY(plan_attend(ctx, a, n_splits, &po, &pml));
+    if (!a.lut && !a.fused_lut) {
+        // this shape builds its tables with the stand-alone kernel first
+        const size_t need = (size_t)B * c.n_q_heads * c.m * c.K * sizeof(float);
+        LOOKAT_TRY(ensure(ctx, (void **)&ctx->lut_scratch, &ctx->lut_cap, need, "table scratch"));
+        LOOKAT_TRY(launch_build_lut(ctx, a.q, B, codebooks, ctx->lut_scratch));
+        a.lut = ctx->lut_scratch;
+    }
     LOOKAT_TRY(ensure(ctx, (void **)&ctx->part_o, &ctx->part_o_cap, po * sizeof(float), "partials"));
     LOOKAT_TRY(ensure(ctx, (void **)&ctx->part_ml, &ctx->part_ml_cap, pml * sizeof(float), "partials"));
     a.part_o = ctx->part_o;
     a.part_ml = ctx->part_ml;
+    if (a.stream) {
+        // arrival counters of the units, all zero between launches (the kernel resets them)
+        const size_t need = (size_t)a.n_units * sizeof(unsigned);
+        if (need > ctx->tickets_cap) {
+            LOOKAT_TRY(ensure(ctx, (void **)&ctx->tickets, &ctx->tickets_cap, need, "unit counters"));
+            if (cudaMemsetAsync(ctx->tickets, 0, ctx->tickets_cap, ctx->stream) != cudaSuccess)
+                return set_error(ctx, LOOKAT_ERR_CUDA, "memset failed");
+        }
+        a.tickets = ctx->tickets;
+        return launch_attend(ctx, a);
+    }
     LOOKAT_TRY(launch_attend(ctx, a));
     return launch_combine(ctx, a);
 }
@@ -233,7 +247,7 @@ void lookat_destroy(lookat_ctx *handle)
     Ctx *ctx = reinterpret_cast<Ctx *>(handle);
     DeviceGuard guard(ctx->device);
     cudaStreamSynchronize(ctx->stream);
-    void *bufs[] = {ctx->part_o, ctx->part_ml, ctx->lut_scratch, ctx->fit_sums, ctx->fit_cnt, ctx->fit_assign,
+    void *bufs[] = {ctx->part_o, ctx->part_ml, ctx->tickets, ctx->lut_scratch, ctx->fit_sums, ctx->fit_cnt, ctx->fit_assign,
                     ctx->step_q,  ctx->step_k,  ctx->step_out};
     for (void *p : bufs)
         if (p) cudaFree(p);

@@ -19,9 +19,13 @@
 //     runs on the tensor cores (mma.sync m16n8k16, fp16 in, fp32 accumulate).
 //     The 8 columns hold the <= 4 heads twice: the fp16 rounding of each weight
 //     and the fp16 rounding of its remainder, so weights carry ~22 bits.  The
-//     token-pair operand layout comes from the row-major V rows by byte permutes.
-// A warp writes one partial (max, sum, weighted values) per unit it touched;
-// combine_stream_kernel merges the partials of every (batch row, query head).
+//     V^T operand comes from the row-major V rows by ldmatrix with transpose.
+// With q and codebooks instead of ready tables, a CTA builds the tables of a
+// unit itself when it enters the unit (fp64 accumulation as in lut.cu).
+// At the end of a unit the warps of a CTA merge through shared memory into one
+// partial (max, sum, weighted values) per (CTA, unit); the CTA that arrives last
+// at a unit (a counter per unit, no waiting) merges the unit's partials and
+// writes the output rows.
 //
 // Generic kernel (attend_generic_kernel): any shape, plain loads, tables read
 // from global memory; used where the streaming kernel's layout assumptions
@@ -38,10 +42,16 @@ constexpr int kTile = 16;           // tokens per warp step (the MMA's k extent)
 constexpr int kHeadPad = 8;         // floats between the table sets of two heads (bank shift)
 constexpr float kNegBig = -1.0e30f; // running-max start: finite, so differences never give NaN
 
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
+__device__ __forceinline__ void cp_async16(unsigned smem_dst, const void *gmem_src)
 {
-    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global.L2::128B [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+    asm volatile("cp.async.cg.shared.global.L2::128B [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+// Four 8x8 fp16 matrices, transposed on the way: lane l gives the address of one 16-byte matrix row.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], unsigned smem_src)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(smem_src));
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -60,17 +70,14 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// fp16 rounding of p (part 0) or of what that rounding left over (part 1).
-__device__ __forceinline__ __half weight_part(float p, int part)
+// Two weights as packed fp16: their roundings (part 0) or what the roundings left over (part 1).
+__device__ __forceinline__ uint32_t weight_pair(float w0, float w1, int part)
 {
-    __half h = __float2half_rn(p);
-    if (part) h = __float2half_rn(p - __half2float(h));
-    return h;
-}
-
-__device__ __forceinline__ uint32_t pack_half2(__half lo, __half hi)
-{
-    return (uint32_t)__half_as_ushort(lo) | ((uint32_t)__half_as_ushort(hi) << 16);
+    const __half2 h = __floats2half2_rn(w0, w1);
+    const float2 f = __half22float2(h);
+    const __half2 r = __floats2half2_rn(w0 - f.x, w1 - f.y);
+    const __half2 out = part ? r : h;
+    return *reinterpret_cast<const uint32_t *>(&out);
 }
 
 template <int M_SUB>
@@ -104,8 +111,8 @@ __device__ __forceinline__ CodePair<M_SUB> read_code_pair(const unsigned char *p
 template <int M_SUB>
 __device__ __forceinline__ int code_at(const CodePair<M_SUB> &c, int token01, int j)
 {
-    int byte = token01 * M_SUB + j;
-    return (c.w[byte >> 2] >> (8 * (byte & 3))) & 0xff;
+    const int byte = token01 * M_SUB + j;
+    return (int)__byte_perm(c.w[byte >> 2], 0u, 0x4440u | (unsigned)(byte & 3));
 }
 
 // Position in the flat tile sequence: tile `lt` of unit `unit`, with that unit's row facts.
@@ -175,9 +182,22 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
     const int head_stride = table + kHeadPad;
     const int lut_bytes = (heads_max * head_stride * 4 + 15) & ~15;
 
+    // shared memory: [tables | merge buffer (same bytes, used in turn)] [queries, fp64] [rings]
+    const int merge_bytes = kWarps * 4 * (DV + 2) * 4;
+    const int region0 = lut_bytes > merge_bytes ? lut_bytes : merge_bytes;
+    const int q_bytes = a.fused_lut ? (heads_max * a.d_k * 8 + 15) & ~15 : 0;
     float *lut_s = reinterpret_cast<float *>(smem_raw);
-    unsigned char *ring = smem_raw + lut_bytes + (size_t)warp * STAGES * SLOT;
+    double *q_s = reinterpret_cast<double *>(smem_raw + region0);
+    unsigned char *ring = smem_raw + region0 + q_bytes + (size_t)warp * STAGES * SLOT;
+    const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ring);
     const float *my_table = lut_s + hl * head_stride;
+
+    // a lane copies the 16-byte piece (lane*16 + it*512) of a tile's V bytes, it = 0..V_CHUNKS-1
+    constexpr int ROWS_PER_IT = 512 / (DV * 2);
+    const int copy_row = (lane * 16) / (DV * 2);
+    const unsigned copy_dst = (unsigned)(copy_row * ROW + (lane * 16) % (DV * 2));
+    // ... and reads, per MMA, one row of four 8x8 blocks: tokens (lane&7) + 8*bit4, dv 8*bit3
+    const unsigned frag_src = (unsigned)(((lane & 7) + ((lane >> 4) & 1) * 8) * ROW + ((lane >> 3) & 1) * 16);
 
     // ---- this CTA's range of the flat tile sequence ----
     long long T_lo, T_hi;
@@ -199,22 +219,19 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             const unsigned char *vsrc = reinterpret_cast<const unsigned char *>(a.v) + row0 * (DV * 2);
             const unsigned char *csrc = a.codes + row0 * M_SUB;
             unsigned char *dst = ring + slot * SLOT;
+            const unsigned dst_s = ring_s + slot * SLOT;
             if (nv == kTile) {
 #pragma unroll
-                for (int it = 0; it < V_CHUNKS; ++it) {
-                    const int off = lane * 16 + it * 512;
-                    cp_async16(dst + (off / (DV * 2)) * ROW + (off % (DV * 2)), vsrc + off);
-                }
-                if (lane < M_SUB) cp_async16(dst + kTile * ROW + lane * 16, csrc + lane * 16);
+                for (int it = 0; it < V_CHUNKS; ++it)
+                    cp_async16(dst_s + copy_dst + it * (ROWS_PER_IT * ROW), vsrc + lane * 16 + it * 512);
+                if (lane < M_SUB) cp_async16(dst_s + kTile * ROW + lane * 16, csrc + lane * 16);
             } else {
                 // ragged end of a row: rows at or beyond seq_len are never read, zeros stand in
 #pragma unroll
                 for (int it = 0; it < V_CHUNKS; ++it) {
-                    const int off = lane * 16 + it * 512;
-                    const int row = off / (DV * 2);
-                    unsigned char *d = dst + row * ROW + (off % (DV * 2));
-                    if (row < nv) cp_async16(d, vsrc + off);
-                    else *reinterpret_cast<uint4 *>(d) = make_uint4(0, 0, 0, 0);
+                    const unsigned d = copy_dst + it * (ROWS_PER_IT * ROW);
+                    if (copy_row + it * ROWS_PER_IT < nv) cp_async16(dst_s + d, vsrc + lane * 16 + it * 512);
+                    else *reinterpret_cast<uint4 *>(dst + d) = make_uint4(0, 0, 0, 0);
                 }
                 if (lane < kTile) {
 #pragma unroll
@@ -230,12 +247,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
     float acc[DV / 16][4];
     float m_run = kNegBig, l_run = 0.f;
 
-    // token offsets inside a tile: the two this lane scores, the four whose V it holds
+    // token offset inside a tile of the two tokens this lane scores
     const int ts_off = 2 * q + 8 * part;
-    const int tv_off[4] = {2 * q, 2 * q + 1, 2 * q + 8, 2 * q + 9};
 
-    // one tile, already in registers: vr = this lane's 16-byte V pieces, cp = its two tokens' codes
-    auto process_tile = [&](int t0, int nv, const uint4 (&vr)[DV / 64][4], const CodePair<M_SUB> &cp,
+    // one tile, already in registers: vf = V^T operand fragments (MMA i covers dv 16i..16i+15),
+    // cp = the codes of this lane's two tokens
+    auto process_tile = [&](int t0, int nv, const uint32_t (&vf)[DV / 16][4], const CodePair<M_SUB> &cp,
                             bool head_ok, float *scores_row) {
         // ---- lookup-and-sum for this lane's two (token, head) pairs ----
         float s0 = 0.f, s1 = 0.f;
@@ -281,25 +298,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         const float o1 = __shfl_xor_sync(0xffffffffu, p1, 16);
         const float w0 = part ? o0 : p0, w1 = part ? o1 : p1;   // tokens 2q, 2q+1
         const float w2 = part ? p0 : o0, w3 = part ? p1 : o1;   // tokens 2q+8, 2q+9
-        const uint32_t b0 = pack_half2(weight_part(w0, part), weight_part(w1, part));
-        const uint32_t b1 = pack_half2(weight_part(w2, part), weight_part(w3, part));
+        const uint32_t b0 = weight_pair(w0, w1, part);
+        const uint32_t b1 = weight_pair(w2, w3, part);
 
         // ---- O^T += V^T P on the tensor cores ----
 #pragma unroll
-        for (int gI = 0; gI < DV / 64; ++gI) {
-            const uint32_t xs[4] = {vr[gI][0].x, vr[gI][0].y, vr[gI][0].z, vr[gI][0].w};
-            const uint32_t ys[4] = {vr[gI][1].x, vr[gI][1].y, vr[gI][1].z, vr[gI][1].w};
-            const uint32_t zs[4] = {vr[gI][2].x, vr[gI][2].y, vr[gI][2].z, vr[gI][2].w};
-            const uint32_t ws[4] = {vr[gI][3].x, vr[gI][3].y, vr[gI][3].z, vr[gI][3].w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t a0 = __byte_perm(xs[i], ys[i], 0x5410);   // dv even, tokens 2q,2q+1
-                const uint32_t a1 = __byte_perm(xs[i], ys[i], 0x7632);   // dv odd
-                const uint32_t a2 = __byte_perm(zs[i], ws[i], 0x5410);   // tokens 2q+8,2q+9
-                const uint32_t a3 = __byte_perm(zs[i], ws[i], 0x7632);
-                mma_16816(acc[gI * 4 + i], a0, a1, a2, a3, b0, b1);
-            }
-        }
+        for (int i = 0; i < DV / 16; ++i) mma_16816(acc[i], vf[i][0], vf[i][1], vf[i][2], vf[i][3], b0, b1);
     };
 
     // ---- prologue: fill the ring with this warp's first STAGES tiles ----
@@ -313,6 +317,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
     int slot = 0;                                          // ring slot of the consumer's tile
 
     // ---- one pass per unit this CTA's range touches ----
+    __shared__ int s_last;
+    float *mg = reinterpret_cast<float *>(smem_raw);      // merge buffer [kWarps][4][DV+2], aliases the tables
+    constexpr int MG = DV + 2;
     const int unit_first = (int)(T_lo / a.tiles_per_unit);
     const int unit_last = T_hi > T_lo ? (int)((T_hi - 1) / a.tiles_per_unit) : unit_first - 1;
     for (int unit = unit_first; unit <= unit_last; ++unit) {
@@ -323,15 +330,50 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         const int hq0 = kvh * a.g + hgrp * 4;
         const bool head_ok = hl < heads_here;
 
-        __syncthreads();                                   // every warp is done with the previous tables
-        for (int h = 0; h < heads_here; ++h) {
-            const float *src = a.lut + ((size_t)b * a.H_q + hq0 + h) * table;
-            float *dst = lut_s + h * head_stride;
-            if ((table & 3) == 0) {
-                for (int i = tid; i < (table >> 2); i += kThreads)
-                    reinterpret_cast<float4 *>(dst)[i] = __ldg(reinterpret_cast<const float4 *>(src) + i);
-            } else {
-                for (int i = tid; i < table; i += kThreads) dst[i] = __ldg(src + i);
+        __syncthreads();                                   // the previous unit's merge is over
+        if (a.lut) {
+            for (int h = 0; h < heads_here; ++h) {
+                const float *src = a.lut + ((size_t)b * a.H_q + hq0 + h) * table;
+                float *dst = lut_s + h * head_stride;
+                if ((table & 3) == 0) {
+                    for (int i = tid; i < (table >> 2); i += kThreads)
+                        reinterpret_cast<float4 *>(dst)[i] = __ldg(reinterpret_cast<const float4 *>(src) + i);
+                } else {
+                    for (int i = tid; i < table; i += kThreads) dst[i] = __ldg(src + i);
+                }
+            }
+        } else {
+            // Section 3.5 "Precomputation Lookup Tables" for the heads of this unit:
+            // lut[h][j][c] = q_h^(j) . C_j[c], fp64 accumulation, one rounding.
+            for (int i = tid; i < heads_here * a.d_k; i += kThreads)
+                q_s[i] = (double)__half2float(a.q[((size_t)b * a.H_q + hq0) * a.d_k + i]);
+            __syncthreads();
+            const int d_sub = a.d_k / M_SUB;
+            const float *book = a.codebooks + (size_t)kvh * table * d_sub;
+            for (int e = tid; e < table; e += kThreads) {
+                const float *cen = book + (size_t)e * d_sub;
+                const double *qj = q_s + (e / a.K) * d_sub;
+                double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
+                auto step = [&](int i, float cf) {
+                    const double cv = (double)cf;
+                    t0 = fma(qj[i], cv, t0);
+                    if (heads_here > 1) t1 = fma(qj[a.d_k + i], cv, t1);
+                    if (heads_here > 2) t2 = fma(qj[2 * a.d_k + i], cv, t2);
+                    if (heads_here > 3) t3 = fma(qj[3 * a.d_k + i], cv, t3);
+                };
+                if ((d_sub & 3) == 0) {
+#pragma unroll 4
+                    for (int i = 0; i < d_sub; i += 4) {
+                        const float4 c4 = __ldg(reinterpret_cast<const float4 *>(cen + i));
+                        step(i, c4.x); step(i + 1, c4.y); step(i + 2, c4.z); step(i + 3, c4.w);
+                    }
+                } else {
+                    for (int i = 0; i < d_sub; ++i) step(i, __ldg(cen + i));
+                }
+                lut_s[e] = (float)t0;
+                if (heads_here > 1) lut_s[head_stride + e] = (float)t1;
+                if (heads_here > 2) lut_s[2 * head_stride + e] = (float)t2;
+                if (heads_here > 3) lut_s[3 * head_stride + e] = (float)t3;
             }
         }
         __syncthreads();
@@ -349,25 +391,23 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             __syncwarp();                                  // ... and every other lane's
             const int nv = cursor_valid(cc);
             const unsigned char *sl = ring + slot * SLOT;
-            uint4 vr[DV / 64][4];
+            uint32_t vf[DV / 16][4];
             CodePair<M_SUB> cp;
             if (nv > 0) {                                  // tile -> registers, so the slot can be refilled
                 cp = read_code_pair<M_SUB>(sl + kTile * ROW + ts_off * M_SUB);
 #pragma unroll
-                for (int gI = 0; gI < DV / 64; ++gI)
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        vr[gI][k] = *reinterpret_cast<const uint4 *>(sl + tv_off[k] * ROW + gI * 128 + n * 16);
+                for (int i = 0; i < DV / 16; ++i)
+                    ldmatrix_x4_trans(vf[i], ring_s + slot * SLOT + frag_src + i * 32);
             }
             __syncwarp();                                  // all lanes have read the slot
             issue(pc, slot);
             cursor_advance(a, pc, kWarps, hgroups);
-            if (nv > 0) process_tile(cc.lt * kTile, nv, vr, cp, head_ok, scores_row);
+            if (nv > 0) process_tile(cc.lt * kTile, nv, vf, cp, head_ok, scores_row);
             slot = slot + 1 == STAGES ? 0 : slot + 1;
             cursor_advance(a, cc, kWarps, hgroups);
         }
 
-        // ---- this warp's partial for the unit: fold the weight and remainder columns ----
+        // ---- this warp's result for the unit: fold the weight and remainder columns ----
 #pragma unroll
         for (int i = 0; i < DV / 16; ++i)
 #pragma unroll
@@ -376,58 +416,80 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);
 
-        const size_t pslot = ((size_t)(c + unit) * kWarps + warp) * 4;     // + head
+        __syncthreads();                                   // every warp is done with the tables
         if (q < 2) {
 #pragma unroll
             for (int i = 0; i < DV / 16; ++i) {
-                const int dv = (i >> 2) * 64 + n * 8 + 2 * (i & 3);
-                float *o = a.part_o + (pslot + 2 * q) * DV + dv;
-                *reinterpret_cast<float2 *>(o) = make_float2(acc[i][0], acc[i][2]);         // head 2q
-                *reinterpret_cast<float2 *>(o + DV) = make_float2(acc[i][1], acc[i][3]);    // head 2q+1
+                float *o = mg + (warp * 4 + 2 * q) * MG + 16 * i + n;
+                o[0] = acc[i][0];              // (dv, head 2q)
+                o[MG] = acc[i][1];             // (dv, head 2q+1)
+                o[8] = acc[i][2];              // (dv + 8, head 2q)
+                o[MG + 8] = acc[i][3];         // (dv + 8, head 2q+1)
             }
         }
         if (q == 0 && part == 0) {
-            a.part_ml[(pslot + hl) * 2] = m_run;
-            a.part_ml[(pslot + hl) * 2 + 1] = l_run;
+            mg[(warp * 4 + hl) * MG + DV] = m_run;
+            mg[(warp * 4 + hl) * MG + DV + 1] = l_run;
+        }
+        __syncthreads();
+
+        // ---- merge the warps: one partial per (CTA, unit) ----
+        const size_t pslot = (size_t)(c + unit) * 4;       // + head
+        for (int idx = tid; idx < heads_here * DV; idx += kThreads) {
+            const int h = idx / DV, dv = idx - h * DV;
+            float M = kNegBig;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) M = fmaxf(M, mg[(w * 4 + h) * MG + DV]);
+            float o = 0.f, l = 0.f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                const float f = ex2_approx(mg[(w * 4 + h) * MG + DV] - M);
+                o += f * mg[(w * 4 + h) * MG + dv];
+                l += f * mg[(w * 4 + h) * MG + DV + 1];
+            }
+            a.part_o[(pslot + h) * DV + dv] = o;
+            if (dv == 0) {
+                a.part_ml[(pslot + h) * 2] = M;
+                a.part_ml[(pslot + h) * 2 + 1] = l;
+            }
+        }
+
+        // ---- the CTA that completes a unit merges the unit's partials into the output ----
+        long long c_lo, c_hi;
+        if (a.splits_per_unit > 0) {
+            c_lo = (long long)unit * a.splits_per_unit;
+            c_hi = c_lo + a.splits_per_unit - 1;
+        } else {
+            c_lo = (long long)unit * a.tiles_per_unit / a.tiles_per_cta;
+            c_hi = ((long long)(unit + 1) * a.tiles_per_unit - 1) / a.tiles_per_cta;
+        }
+        __threadfence();                                   // this thread's partial writes are visible
+        __syncthreads();
+        if (tid == 0) {
+            const unsigned arrived = atomicAdd(a.tickets + unit, 1u);
+            s_last = arrived == (unsigned)(c_hi - c_lo);
+            if (s_last) a.tickets[unit] = 0u;              // ready for the next launch
+        }
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            for (int idx = tid; idx < heads_here * DV; idx += kThreads) {
+                const int h = idx / DV, dv = idx - h * DV;
+                float M = kNegBig;
+                for (long long cp2 = c_lo; cp2 <= c_hi; ++cp2)
+                    M = fmaxf(M, __ldcg(a.part_ml + ((size_t)(cp2 + unit) * 4 + h) * 2));
+                float o = 0.f, l = 0.f;
+                for (long long cp2 = c_lo; cp2 <= c_hi; ++cp2) {
+                    const size_t pp = (size_t)(cp2 + unit) * 4 + h;
+                    const float f = ex2_approx(__ldcg(a.part_ml + pp * 2) - M);
+                    l += f * __ldcg(a.part_ml + pp * 2 + 1);
+                    o += f * __ldcg(a.part_o + pp * DV + dv);
+                }
+                a.out[((size_t)b * a.H_q + hq0 + h) * DV + dv] = l > 0.f ? o / l : 0.f;
+            }
         }
     }
     cp_async_wait<0>();
-}
-
-// Merge of the streaming kernel's partials for one (batch row, query head):
-// M = max_i M_i, l = sum l_i 2^(M_i-M), o = sum o_i 2^(M_i-M) / l over every (CTA, warp) that
-// touched the row's unit.  Partials without tokens carry l = 0 and add nothing.
-template <int DV>
-__global__ void __launch_bounds__(DV) combine_stream_kernel(AttendArgs a)
-{
-    const int row = blockIdx.x;                         // b * H_q + hq
-    const int b = row / a.H_q, hq = row - b * a.H_q;
-    const int kvh = hq / a.g, hin = hq - kvh * a.g;
-    const int hgroups = (a.g + 3) >> 2;
-    const int unit = (b * a.H_kv + kvh) * hgroups + (hin >> 2);
-    const int hl = hin & 3;
-    long long c_lo, c_hi;
-    if (a.splits_per_unit > 0) {
-        c_lo = (long long)unit * a.splits_per_unit;
-        c_hi = c_lo + a.splits_per_unit - 1;
-    } else {
-        c_lo = (long long)unit * a.tiles_per_unit / a.tiles_per_cta;
-        c_hi = ((long long)(unit + 1) * a.tiles_per_unit - 1) / a.tiles_per_cta;
-    }
-    const int dv = threadIdx.x;
-    float M = kNegBig;
-    for (long long c = c_lo; c <= c_hi; ++c)
-        for (int w = 0; w < kWarps; ++w)
-            M = fmaxf(M, a.part_ml[((((size_t)(c + unit) * kWarps + w) * 4) + hl) * 2]);
-    float l = 0.f, o = 0.f;
-    for (long long c = c_lo; c <= c_hi; ++c)
-        for (int w = 0; w < kWarps; ++w) {
-            const size_t p = ((size_t)(c + unit) * kWarps + w) * 4 + hl;
-            const float f = ex2_approx(a.part_ml[p * 2] - M);
-            l += f * a.part_ml[p * 2 + 1];
-            o += f * a.part_o[p * DV + dv];
-        }
-    a.out[(size_t)row * DV + dv] = l > 0.f ? o / l : 0.f;
 }
 
 // Any shape.  One CTA per (chunk, query head, batch row); 128 threads.
@@ -551,8 +613,11 @@ size_t stream_smem_bytes(const AttendArgs &a, int stages)
 {
     const int heads = a.g < 4 ? a.g : 4;
     const size_t lut_bytes = ((size_t)heads * (a.m * a.K + kHeadPad) * 4 + 15) & ~(size_t)15;
+    const size_t merge_bytes = (size_t)kWarps * 4 * (a.d_v + 2) * 4;
+    const size_t region0 = lut_bytes > merge_bytes ? lut_bytes : merge_bytes;
+    const size_t q_bytes = a.fused_lut ? ((size_t)heads * a.d_k * 8 + 15) & ~(size_t)15 : 0;
     const size_t slot = (size_t)kTile * (a.d_v * 2 + 16) + (size_t)kTile * a.m;
-    return lut_bytes + (size_t)kWarps * stages * slot;
+    return region0 + q_bytes + (size_t)kWarps * stages * slot;
 }
 
 int stream_stages(const Ctx *ctx, const AttendArgs &a)
@@ -603,7 +668,9 @@ lookat_status dispatch_stream(int m, int d_v, int stages, F &&f)
 
 lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_floats, size_t *part_ml_floats)
 {
+    a.fused_lut = (!a.lut && a.d_k <= 256) ? 1 : 0;    // tables built inside the streaming kernel
     const int stages = stream_shape_ok(ctx, a) ? stream_stages(ctx, a) : 0;
+    if (!stages) a.fused_lut = 0;
     if (stages) {
         const int hgroups = (a.g + 3) / 4;
         const long long units = (long long)a.B * a.H_kv * hgroups;
@@ -633,9 +700,9 @@ lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_
             a.splits_per_unit = 0;
             a.n_ctas = (int)((total + a.tiles_per_cta - 1) / a.tiles_per_cta);
         }
-        const size_t slots = (size_t)a.n_ctas + (size_t)a.n_units;
-        *part_o_floats = slots * kWarps * 4 * a.d_v;
-        *part_ml_floats = slots * kWarps * 4 * 2;
+        const size_t slots = (size_t)a.n_ctas + (size_t)a.n_units;     // slot of (CTA c, unit u) = c + u
+        *part_o_floats = slots * 4 * a.d_v;
+        *part_ml_floats = slots * 4 * 2;
         return LOOKAT_OK;
     }
     // generic kernel: chunks of whole 16-token groups, at least 256 tokens unless asked otherwise
@@ -697,11 +764,7 @@ lookat_status launch_attend(Ctx *ctx, const AttendArgs &a)
 
 lookat_status launch_combine(Ctx *ctx, const AttendArgs &a)
 {
-    if (a.stream) {
-        if (a.d_v == 64) combine_stream_kernel<64><<<a.B * a.H_q, 64, 0, ctx->stream>>>(a);
-        else combine_stream_kernel<128><<<a.B * a.H_q, 128, 0, ctx->stream>>>(a);
-        return check_launch(ctx, "combine_stream_kernel");
-    }
+    // the streaming kernel merges its partials itself; only the generic kernel needs this pass
     int threads = a.d_v < 32 ? 32 : (a.d_v > 256 ? 256 : ((a.d_v + 31) / 32) * 32);
     combine_generic_kernel<<<a.B * a.H_q, threads, 0, ctx->stream>>>(a);
     return check_launch(ctx, "combine_generic_kernel");

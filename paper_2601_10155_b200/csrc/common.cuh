@@ -27,6 +27,8 @@ struct Ctx {
     float *part_o;
     float *part_ml;
     size_t part_o_cap, part_ml_cap;       // bytes
+    unsigned *tickets;                     // attend: per-unit arrival counters, zero between launches
+    size_t tickets_cap;
     // tables built on behalf of the caller (lookat_attend with lut == NULL)
     float *lut_scratch;
     size_t lut_cap;                        // bytes
@@ -55,7 +57,12 @@ lookat_status ensure(Ctx *ctx, void **ptr, size_t *cap, size_t need_bytes, const
 
 // ---- launchers (each validates nothing: the API layer has done it) ----
 struct AttendArgs {
-    const float *lut;          // [B][H_q][m][K]
+    const float *lut;          // [B][H_q][m][K], or null: built from q and codebooks
+    const __half *q;           // [B][H_q][d_k]            (used when lut is null)
+    const float *codebooks;    // [H_kv][m][K][d_sub]      (used when lut is null)
+    int d_k;
+    int fused_lut;             // 1: the streaming kernel builds its tables itself
+    unsigned *tickets;         // [n_units] arrival counters (streaming kernel)
     const uint8_t *codes;      // [B][H_kv][L_max][m]
     const __half *v;           // [B][H_kv][L_max][d_v]
     const int32_t *seq_lens;   // [B] or null

@@ -236,16 +236,45 @@ encode_warp_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K, long long n_ta
     const float *book = a.codebooks + (size_t)problem * K * d_sub;
     const __half *x = a.keys + (size_t)key * d_k + j * d_sub;
 
+    // lane l owns centroids l, l+32, ... (at most 8, K <= 256); dimensions in the outer loop so
+    // that the lane's centroid loads of one step are independent of each other
+    float d[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) d[k] = 0.f;
+    if ((d_sub & 3) == 0) {
+        for (int i = 0; i < d_sub; i += 4) {
+            const float x0 = __half2float(x[i]), x1 = __half2float(x[i + 1]);
+            const float x2 = __half2float(x[i + 2]), x3 = __half2float(x[i + 3]);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int c = lane + 32 * k;
+                if (c < K) {
+                    const float4 cv = __ldg(reinterpret_cast<const float4 *>(book + (size_t)c * d_sub + i));
+                    float t = x0 - cv.x; d[k] = fmaf(t, t, d[k]);
+                    t = x1 - cv.y; d[k] = fmaf(t, t, d[k]);
+                    t = x2 - cv.z; d[k] = fmaf(t, t, d[k]);
+                    t = x3 - cv.w; d[k] = fmaf(t, t, d[k]);
+                }
+            }
+        }
+    } else {
+        for (int i = 0; i < d_sub; ++i) {
+            const float xi = __half2float(x[i]);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int c = lane + 32 * k;
+                if (c < K) {
+                    const float t = xi - __ldg(book + (size_t)c * d_sub + i);
+                    d[k] = fmaf(t, t, d[k]);
+                }
+            }
+        }
+    }
     Best r;
     r.best = INFINITY; r.second = INFINITY; r.idx = 0x7fffffff;
-    for (int c = lane; c < K; c += 32) {
-        float d = 0.f;
-        for (int i = 0; i < d_sub; ++i) {
-            const float tt = __half2float(x[i]) - book[(size_t)c * d_sub + i];
-            d = fmaf(tt, tt, d);
-        }
-        consider(r, d, c);
-    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+        if (lane + 32 * k < K) consider(r, d[k], lane + 32 * k);
     // merge lanes: smaller distance wins, then smaller index; the loser's best is a runner-up
     for (int s = 16; s; s >>= 1) {
         const float ob = __shfl_xor_sync(0xffffffffu, r.best, s);
