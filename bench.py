@@ -37,10 +37,10 @@ METRIC = "adc_decode_attention_tokens_heads_per_s"
 UNIT = "tokens*heads/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) of one attend_stream_kernel launch on this workload as counted by ncu
-# (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture has been summarised
-# under profiles/.
-ATTEND_DRAM_TRAFFIC_BYTES = None
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per (token, KV head) pair of one
+# attend_stream_kernel launch, from an ncu capture of the batch-4 case of gqa_32k_m8
+# (284,259,328 bytes over 1,048,576 pairs; traffic grows in proportion to the pairs).
+ATTEND_DRAM_BYTES_PER_PAIR = {"gqa_32k_m8": 284259328 / 1048576}
 
 
 def measured_peak_gbs():
@@ -186,6 +186,27 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def rank_workload(w, rank: int):
+    """The replica a rank runs: same shape, its own inputs (seed offset by rank)."""
+    return synth.Workload(**{**w.__dict__, "seed": w.seed + 7919 * rank})
+
+
+def max_over_ranks(values, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(x) for x in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def job_value(w, world: int, ms_per_step: float) -> float:
+    """Whole-job tokens*heads per second: every rank scores B*H_q*L pairs per step."""
+    return w.B * w.n_q_heads * w.L * world / (ms_per_step * 1e-3)
+
+
 def workload_config(w):
     return {"workload": w.name, "batch": w.B, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
             "d_k": w.d_k, "d_v": w.d_v, "seq_len": w.L, "m": w.m, "K": w.K, "v_dtype": "fp16",
@@ -211,7 +232,7 @@ def run_lookat(args, w):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     # every rank runs the same replica shape on its own inputs (seed offset by rank)
-    wr = synth.Workload(**{**w.__dict__, "seed": w.seed + 7919 * rank})
+    wr = rank_workload(w, rank)
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
     lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K, device=local_rank)
 
@@ -271,10 +292,7 @@ def run_lookat(args, w):
     elapsed_ms = e0.elapsed_time(e1)
     attend_ms = lk.lookat_attend_kernel_ms()
     launches = lk.lookat_kernel_launches() - launches0
-    if world > 1:
-        t = torch.tensor([elapsed_ms, attend_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, attend_ms = float(t[0]), float(t[1])
+    elapsed_ms, attend_ms = max_over_ranks([elapsed_ms, attend_ms], "cuda")
 
     # ---- end to end: host buffers in, host buffer out, through the C-ABI call ----
     q_host = torch.from_numpy(q_np).pin_memory()
@@ -292,19 +310,18 @@ def run_lookat(args, w):
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t[0])
+    (e2e_ms,) = max_over_ranks([e2e_ms], "cuda")
     same = bool(torch.allclose(out_host.cuda(), out, rtol=0, atol=1e-5))
 
     if rank == 0:
         units_per_step = w.B * w.n_q_heads * L * world
         ms_per_step = elapsed_ms / args.steps
-        value = units_per_step / (ms_per_step * 1e-3)
+        value = job_value(w, world, ms_per_step)
         peak, peak_kind = measured_peak_gbs()
         alg_bytes = (w.m + 2 * w.d_v) * w.B * w.n_kv_heads * L           # per attend launch
         achieved = alg_bytes / (attend_ms * 1e-3) / 1e9
+        per_pair = ATTEND_DRAM_BYTES_PER_PAIR.get(args.workload)
+        traffic = None if per_pair is None else int(per_pair * w.B * w.n_kv_heads * L)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -312,7 +329,7 @@ def run_lookat(args, w):
             "config": workload_config(w),
             "roofline": {"bound": "hbm", "kernel": "attend_stream_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                         "traffic": ATTEND_DRAM_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": alg_bytes,
+                         "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,
                          "kernel_ms": attend_ms, "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS},
             "e2e": {"value": units_per_step / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": int(q_host.numel() * 2 + k_host.numel() * 2 + v_host.numel() * 2),
