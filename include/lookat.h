@@ -136,6 +136,35 @@ lookat_status lookat_attend(lookat_ctx *ctx, const float *lut, const void *q, co
                             const int32_t *seq_lens, int32_t n_splits, float *out, float *scores_out);
 
 /*
+ * lookat_attend without any allocation.  (The paper has no counterpart: it is
+ * an interface variant of lookat_attend, same arguments, same results.)
+ *
+ * For callers that cannot let a library call cudaMalloc / cudaFree: a serving
+ * process whose own pool owns all device memory, or a decode loop that cannot
+ * afford the device-wide synchronisation those calls imply.  The partial
+ * results and the per-unit counters of the attend kernel live in a fixed
+ * device array inside the library (2 MiB + 64 KiB + 16 KiB, held by every GPU
+ * that loads the library until the process exits) instead of context scratch.
+ *
+ * Limits: (CTAs launched + B*H_kv*ceil(g/4)) * 4 * d_v floats of partials must
+ * fit in 2 MiB (524,288 floats) and B*H_kv*ceil(g/4) <= 4096; with the
+ * library's own chunking (n_splits = 0) the CTA count is at most a few per SM.
+ * A problem beyond that returns LOOKAT_ERR_UNSUPPORTED and launches nothing,
+ * as does a shape whose tables cannot be built inside the kernel when lut is
+ * NULL (pass ready tables then).
+ *
+ * The first call on a device looks up the device address of the array (no
+ * allocation either); make that first call before starting a stream capture.
+ * All calls share the array: two calls whose kernels overlap on the GPU
+ * (different streams or contexts, same device) race on it and give wrong
+ * results; calls on one stream are safe.  The counters are cleared at every
+ * call, so a call cut short by an error leaves nothing behind.
+ */
+lookat_status lookat_attend_static(lookat_ctx *ctx, const float *lut, const void *q, const float *codebooks,
+                                   const uint8_t *codes, const void *v, int32_t B, int64_t L_max,
+                                   const int32_t *seq_lens, int32_t n_splits, float *out, float *scores_out);
+
+/*
  * One decode step driven from HOST buffers (what a serving loop that keeps
  * its activations on the host calls): copies the step's query, new key and
  * new value rows to the device, encodes the new key at token `pos`
