@@ -39,6 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [_nvcc(), "-O3", "-std=c++20", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-shared", "-Xcompiler", "-fPIC", "-cudart", "static", "-I", INCLUDE, "-I", CSRC]
+    cmd += os.environ.get("LOOKAT_NVCC_FLAGS", "").split()      # e.g. -DNAME for tuning experiments
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]

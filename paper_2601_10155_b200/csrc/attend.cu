@@ -30,6 +30,8 @@
 // Generic kernel (attend_generic_kernel): any shape, plain loads, tables read
 // from global memory; used where the streaming kernel's layout assumptions
 // (d_v in {64,128}, m in {1,2,4,8,16}, 16-byte aligned rows) do not hold.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace lookat {
@@ -40,11 +42,16 @@ constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
 constexpr int kTile = 16;           // tokens per warp step (the MMA's k extent)
 constexpr int kHeadPad = 8;         // floats between the table sets of two heads (bank shift)
+constexpr int kTableStride = 256;   // shared-memory entries per subspace table (codes are bytes)
 constexpr float kNegBig = -1.0e30f; // running-max start: finite, so differences never give NaN
 
 __device__ __forceinline__ void cp_async16(unsigned smem_dst, const void *gmem_src)
 {
+#ifdef LOOKAT_CP_ASYNC_PLAIN
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+#else
     asm volatile("cp.async.cg.shared.global.L2::128B [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+#endif
 }
 // Four 8x8 fp16 matrices, transposed on the way: lane l gives the address of one 16-byte matrix row.
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], unsigned smem_src)
@@ -115,44 +122,55 @@ __device__ __forceinline__ int code_at(const CodePair<M_SUB> &c, int token01, in
     return (int)__byte_perm(c.w[byte >> 2], 0u, 0x4440u | (unsigned)(byte & 3));
 }
 
-// Position in the flat tile sequence: tile `lt` of unit `unit`, with that unit's row facts.
+// Position in the flat tile sequence: tile `lt` of unit `unit`, with that unit's row facts and
+// the addresses of the tile's V rows and codes.
 struct TileCursor {
     long long T;         // flat index
     int unit, lt;
-    int b, kvh;          // batch row and KV head of the unit
-    int len;             // tokens in that batch row (0 beyond the last unit)
+    int len;             // tokens in the unit's batch row (0 beyond the last unit)
+    const unsigned char *vptr, *cptr;
 };
 
+template <int M_SUB, int DV>
 __device__ __forceinline__ void cursor_enter_unit(const AttendArgs &a, TileCursor &c, int hgroups)
 {
-    const int kv_row = c.unit / hgroups;
-    c.b = kv_row / a.H_kv;
-    c.kvh = kv_row - c.b * a.H_kv;
-    c.len = c.unit < a.n_units
-                ? (int)min((long long)(a.seq_lens ? a.seq_lens[c.b] : a.uniform_len), a.L_max)
-                : 0;
+    if (c.unit < a.n_units) {
+        const int kv_row = c.unit / hgroups;             // (batch row, KV head) of the unit
+        const int b = kv_row / a.H_kv;
+        c.len = (int)min((long long)(a.seq_lens ? a.seq_lens[b] : a.uniform_len), a.L_max);
+        const size_t row0 = (size_t)kv_row * a.L_max + (size_t)c.lt * kTile;
+        c.vptr = reinterpret_cast<const unsigned char *>(a.v) + row0 * (DV * 2);
+        c.cptr = a.codes + row0 * M_SUB;
+    } else {
+        c.len = 0;
+    }
 }
 
+template <int M_SUB, int DV>
 __device__ __forceinline__ TileCursor cursor_at(const AttendArgs &a, long long T, int hgroups)
 {
     TileCursor c;
     c.T = T;
     c.unit = (int)(T / a.tiles_per_unit);
     c.lt = (int)(T - (long long)c.unit * a.tiles_per_unit);
-    cursor_enter_unit(a, c, hgroups);
+    c.vptr = c.cptr = nullptr;
+    cursor_enter_unit<M_SUB, DV>(a, c, hgroups);
     return c;
 }
 
-__device__ __forceinline__ void cursor_advance(const AttendArgs &a, TileCursor &c, int step, int hgroups)
+template <int M_SUB, int DV>
+__device__ __forceinline__ void cursor_advance(const AttendArgs &a, TileCursor &c, int hgroups)
 {
-    c.T += step;
-    c.lt += step;
+    c.T += kWarps;
+    c.lt += kWarps;
+    c.vptr += kWarps * kTile * DV * 2;
+    c.cptr += kWarps * kTile * M_SUB;
     if (c.lt >= a.tiles_per_unit) {
         do {
             c.lt -= a.tiles_per_unit;
             c.unit += 1;
         } while (c.lt >= a.tiles_per_unit);
-        cursor_enter_unit(a, c, hgroups);
+        cursor_enter_unit<M_SUB, DV>(a, c, hgroups);
     }
 }
 
@@ -163,10 +181,27 @@ __device__ __forceinline__ int cursor_valid(const TileCursor &c)
     return left >= kTile ? kTile : (left > 0 ? left : 0);
 }
 
+#ifdef LOOKAT_PHASE_STAMPS
+// Tuning aid, compiled only on request: per CTA, the global timer at a few points of the kernel.
+__device__ unsigned long long g_phase_stamps[1024][8];
+__device__ __forceinline__ void phase_stamp(int k)
+{
+    if (threadIdx.x == 0 && blockIdx.x < 1024) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        g_phase_stamps[blockIdx.x][k] = t;
+    }
+}
+#define LOOKAT_STAMP(k) phase_stamp(k)
+#else
+#define LOOKAT_STAMP(k)
+#endif
+
 template <int M_SUB, int DV, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    LOOKAT_STAMP(0);
     constexpr int ROW = DV * 2 + 16;                      // a V row plus 16 bytes of padding
     constexpr int SLOT = kTile * ROW + kTile * M_SUB;     // V rows, then the tile's codes
     constexpr int V_CHUNKS = kTile * DV * 2 / 512;        // 16-byte pieces per lane and tile
@@ -178,8 +213,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
     const int part = n >> 2;                              // 0: weight, 1: its fp16 remainder
     const int hgroups = (a.g + 3) >> 2;
     const int heads_max = a.g < 4 ? a.g : 4;
-    const int table = M_SUB * a.K;                        // floats per head
-    const int head_stride = table + kHeadPad;
+    const int table = M_SUB * a.K;                        // floats per head in global memory
+    // in shared memory every subspace gets kTableStride entries whatever K is: offsets are constants
+    constexpr int head_stride = M_SUB * kTableStride + kHeadPad;
     const int lut_bytes = (heads_max * head_stride * 4 + 15) & ~15;
 
     // shared memory: [tables | merge buffer (same bytes, used in turn)] [queries, fp64] [rings]
@@ -215,9 +251,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
     auto issue = [&](const TileCursor &pc, int slot) {
         const int nv = pc.T < T_hi ? cursor_valid(pc) : 0;
         if (nv > 0) {
-            const size_t row0 = ((size_t)pc.b * a.H_kv + pc.kvh) * a.L_max + (size_t)pc.lt * kTile;
-            const unsigned char *vsrc = reinterpret_cast<const unsigned char *>(a.v) + row0 * (DV * 2);
-            const unsigned char *csrc = a.codes + row0 * M_SUB;
+            const unsigned char *vsrc = pc.vptr;
+            const unsigned char *csrc = pc.cptr;
             unsigned char *dst = ring + slot * SLOT;
             const unsigned dst_s = ring_s + slot * SLOT;
             if (nv == kTile) {
@@ -252,24 +287,30 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
 
     // one tile, already in registers: vf = V^T operand fragments (MMA i covers dv 16i..16i+15),
     // cp = the codes of this lane's two tokens
-    auto process_tile = [&](int t0, int nv, const uint32_t (&vf)[DV / 16][4], const CodePair<M_SUB> &cp,
-                            bool head_ok, float *scores_row) {
+    // `full` (a compile-time flag): all 16 tokens exist, all 4 heads of the group are in use and no
+    // raw scores are wanted, so none of the per-lane conditions below is needed.
+    auto process_tile = [&](auto full, int t0, int nv, const uint32_t (&vf)[DV / 16][4],
+                            const CodePair<M_SUB> &cp, bool head_ok, float *scores_row) {
+        constexpr bool FULL = decltype(full)::value;
         // ---- lookup-and-sum for this lane's two (token, head) pairs ----
         float s0 = 0.f, s1 = 0.f;
-        if (head_ok) {
+        if (FULL || head_ok) {
 #pragma unroll
             for (int j = 0; j < M_SUB; ++j) {
-                s0 += my_table[j * a.K + code_at<M_SUB>(cp, 0, j)];
-                s1 += my_table[j * a.K + code_at<M_SUB>(cp, 1, j)];
+                s0 += my_table[j * kTableStride + code_at<M_SUB>(cp, 0, j)];
+                s1 += my_table[j * kTableStride + code_at<M_SUB>(cp, 1, j)];
             }
         }
-        const bool ok0 = head_ok && ts_off < nv, ok1 = head_ok && ts_off + 1 < nv;
-        if (scores_row) {
-            if (ok0) scores_row[t0 + ts_off] = s0;
-            if (ok1) scores_row[t0 + ts_off + 1] = s1;
+        float x0 = s0 * a.scale_log2, x1 = s1 * a.scale_log2;
+        if constexpr (!FULL) {
+            const bool ok0 = head_ok && ts_off < nv, ok1 = head_ok && ts_off + 1 < nv;
+            if (scores_row) {
+                if (ok0) scores_row[t0 + ts_off] = s0;
+                if (ok1) scores_row[t0 + ts_off + 1] = s1;
+            }
+            x0 = ok0 ? x0 : -INFINITY;
+            x1 = ok1 ? x1 : -INFINITY;
         }
-        const float x0 = ok0 ? s0 * a.scale_log2 : -INFINITY;
-        const float x1 = ok1 ? s1 * a.scale_log2 : -INFINITY;
 
         // ---- running maximum per head (8 lanes share a head) ----
         float mt = fmaxf(x0, x1);
@@ -307,12 +348,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
     };
 
     // ---- prologue: fill the ring with this warp's first STAGES tiles ----
-    TileCursor cc = cursor_at(a, T_lo + warp, hgroups);   // tile this warp consumes next
-    TileCursor pc = cc;                                   // tile it copies next
+    TileCursor cc = cursor_at<M_SUB, DV>(a, T_lo + warp, hgroups);   // tile this warp consumes next
+    TileCursor pc = cc;                                              // tile it copies next
 #pragma unroll
     for (int s = 0; s < STAGES; ++s) {
         issue(pc, s);
-        cursor_advance(a, pc, kWarps, hgroups);
+        cursor_advance<M_SUB, DV>(a, pc, hgroups);
     }
     int slot = 0;                                          // ring slot of the consumer's tile
 
@@ -331,15 +372,19 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         const bool head_ok = hl < heads_here;
 
         __syncthreads();                                   // the previous unit's merge is over
+        if (unit == unit_first) LOOKAT_STAMP(1);
         if (a.lut) {
             for (int h = 0; h < heads_here; ++h) {
                 const float *src = a.lut + ((size_t)b * a.H_q + hq0 + h) * table;
                 float *dst = lut_s + h * head_stride;
-                if ((table & 3) == 0) {
+                if (a.K == kTableStride) {
                     for (int i = tid; i < (table >> 2); i += kThreads)
                         reinterpret_cast<float4 *>(dst)[i] = __ldg(reinterpret_cast<const float4 *>(src) + i);
                 } else {
-                    for (int i = tid; i < table; i += kThreads) dst[i] = __ldg(src + i);
+                    for (int i = tid; i < table; i += kThreads) {
+                        const int j = i / a.K;
+                        dst[j * kTableStride + (i - j * a.K)] = __ldg(src + i);
+                    }
                 }
             }
         } else {
@@ -348,11 +393,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             for (int i = tid; i < heads_here * a.d_k; i += kThreads)
                 q_s[i] = (double)__half2float(a.q[((size_t)b * a.H_q + hq0) * a.d_k + i]);
             __syncthreads();
+
             const int d_sub = a.d_k / M_SUB;
             const float *book = a.codebooks + (size_t)kvh * table * d_sub;
             for (int e = tid; e < table; e += kThreads) {
                 const float *cen = book + (size_t)e * d_sub;
-                const double *qj = q_s + (e / a.K) * d_sub;
+                const int j = e / a.K;
+                const int es = j * kTableStride + (e - j * a.K);      // position in the shared-memory table
+                const double *qj = q_s + j * d_sub;
                 double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
                 auto step = [&](int i, float cf) {
                     const double cv = (double)cf;
@@ -370,10 +418,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
                 } else {
                     for (int i = 0; i < d_sub; ++i) step(i, __ldg(cen + i));
                 }
-                lut_s[e] = (float)t0;
-                if (heads_here > 1) lut_s[head_stride + e] = (float)t1;
-                if (heads_here > 2) lut_s[2 * head_stride + e] = (float)t2;
-                if (heads_here > 3) lut_s[3 * head_stride + e] = (float)t3;
+                lut_s[es] = (float)t0;
+                if (heads_here > 1) lut_s[head_stride + es] = (float)t1;
+                if (heads_here > 2) lut_s[2 * head_stride + es] = (float)t2;
+                if (heads_here > 3) lut_s[3 * head_stride + es] = (float)t3;
             }
         }
         __syncthreads();
@@ -385,7 +433,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         float *scores_row =
             (a.scores_out && head_ok) ? a.scores_out + ((size_t)b * a.H_q + hq0 + hl) * a.L_max : nullptr;
 
+        if (unit == unit_first) LOOKAT_STAMP(2);
         const long long seg_hi = min(T_hi, (long long)(unit + 1) * a.tiles_per_unit);
+        const bool full_unit = heads_here == 4 && !a.scores_out;
         while (cc.T < seg_hi) {
             cp_async_wait<STAGES - 1>();                   // this lane's copies of the tile have landed
             __syncwarp();                                  // ... and every other lane's
@@ -401,12 +451,17 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             }
             __syncwarp();                                  // all lanes have read the slot
             issue(pc, slot);
-            cursor_advance(a, pc, kWarps, hgroups);
-            if (nv > 0) process_tile(cc.lt * kTile, nv, vf, cp, head_ok, scores_row);
+            cursor_advance<M_SUB, DV>(a, pc, hgroups);
+            if (nv == kTile && full_unit)
+                process_tile(std::true_type{}, 0, kTile, vf, cp, true, nullptr);
+            else if (nv > 0)
+                process_tile(std::false_type{}, cc.lt * kTile, nv, vf, cp, head_ok, scores_row);
             slot = slot + 1 == STAGES ? 0 : slot + 1;
-            cursor_advance(a, cc, kWarps, hgroups);
+            cursor_advance<M_SUB, DV>(a, cc, hgroups);
         }
 
+        if (unit == unit_first) LOOKAT_STAMP(3);
+        if (unit == unit_last) LOOKAT_STAMP(4);
         // ---- this warp's result for the unit: fold the weight and remainder columns ----
 #pragma unroll
         for (int i = 0; i < DV / 16; ++i)
@@ -454,6 +509,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             }
         }
 
+        if (unit == unit_last) LOOKAT_STAMP(5);
         // ---- the CTA that completes a unit merges the unit's partials into the output ----
         long long c_lo, c_hi;
         if (a.splits_per_unit > 0) {
@@ -490,6 +546,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         }
     }
     cp_async_wait<0>();
+    LOOKAT_STAMP(6);
+#ifdef LOOKAT_PHASE_STAMPS
+    if (threadIdx.x == 0 && blockIdx.x < 1024) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+        g_phase_stamps[blockIdx.x][7] = smid;
+    }
+#endif
 }
 
 // Any shape.  One CTA per (chunk, query head, batch row); 128 threads.
@@ -612,7 +676,7 @@ bool stream_shape_ok(const Ctx *ctx, const AttendArgs &a)
 size_t stream_smem_bytes(const AttendArgs &a, int stages)
 {
     const int heads = a.g < 4 ? a.g : 4;
-    const size_t lut_bytes = ((size_t)heads * (a.m * a.K + kHeadPad) * 4 + 15) & ~(size_t)15;
+    const size_t lut_bytes = ((size_t)heads * (a.m * kTableStride + kHeadPad) * 4 + 15) & ~(size_t)15;
     const size_t merge_bytes = (size_t)kWarps * 4 * (a.d_v + 2) * 4;
     const size_t region0 = lut_bytes > merge_bytes ? lut_bytes : merge_bytes;
     const size_t q_bytes = a.fused_lut ? ((size_t)heads * a.d_k * 8 + 15) & ~(size_t)15 : 0;
@@ -761,6 +825,13 @@ lookat_status launch_attend(Ctx *ctx, const AttendArgs &a)
     }
     return st;
 }
+
+#ifdef LOOKAT_PHASE_STAMPS
+extern "C" int lookat_debug_phase_stamps(unsigned long long *host_out)     // [1024][8]
+{
+    return (int)cudaMemcpyFromSymbol(host_out, g_phase_stamps, sizeof(unsigned long long) * 1024 * 8);
+}
+#endif
 
 lookat_status launch_combine(Ctx *ctx, const AttendArgs &a)
 {
