@@ -262,10 +262,11 @@ def run_lookat(args, w):
     new_k = keys[:, :, L - 1:L].contiguous()              # the newest key of every (row, KV head)
     out = torch.empty((w.B, w.n_q_heads, w.d_v), dtype=torch.float32, device="cuda")
 
+    new_k3 = new_k.reshape(w.B, w.n_kv_heads, w.d_k)
+
     def step():
-        # append: encode the newest key; then Algorithm 1 (tables, lookup-sum, softmax, value sum)
-        lk.lookat_encode_keys(new_k, books, codes=codes, pos=L - 1)
-        lk.lookat_attend(codes, v, q=q, codebooks=books, out=out, n_splits=args.splits)
+        # append (encode the newest key) and Algorithm 1 (tables, lookup-sum, softmax, value sum)
+        lk.lookat_decode_step(q, new_k3, books, codes, v, L - 1, out=out, n_splits=args.splits)
 
     def barrier():
         torch.cuda.synchronize()

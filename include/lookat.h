@@ -165,6 +165,27 @@ lookat_status lookat_attend_static(lookat_ctx *ctx, const float *lut, const void
                                    const int32_t *seq_lens, int32_t n_splits, float *out, float *scores_out);
 
 /*
+ * One decode step on device buffers: append and attend.  The new key of every
+ * (batch row, KV head) is encoded at token `pos` of the code cache (Section
+ * 3.4, Encoding), then Algorithm 1 runs over tokens 0..pos with tables built
+ * from q and the codebooks.  Same results as lookat_encode_keys(n = 1, pos)
+ * followed by lookat_attend with every row at pos+1 tokens; where the
+ * streaming attend kernel covers the shape, both happen in one launch (the
+ * warp that is about to read the tile holding token `pos` encodes the key
+ * first).  The value row of token `pos` must already be in the V cache.
+ *
+ *   q          fp16 [B][H_q][d_k]
+ *   k_new      fp16 [B][H_kv][d_k]
+ *   codes      in/out, uint8 [B][H_kv][L_max][m]; row pos is written
+ *   v          fp16 [B][H_kv][L_max][d_v]
+ *   out        fp32 [B][H_q][d_v]
+ * Requires 0 <= pos < L_max.
+ */
+lookat_status lookat_decode_step(lookat_ctx *ctx, const void *q, const void *k_new, const float *codebooks,
+                                 uint8_t *codes, const void *v, int32_t B, int64_t L_max, int64_t pos,
+                                 int32_t n_splits, float *out);
+
+/*
  * One decode step driven from HOST buffers (what a serving loop that keeps
  * its activations on the host calls): copies the step's query, new key and
  * new value rows to the device, encodes the new key at token `pos`

@@ -81,10 +81,14 @@ lookat_status need_ptr(Ctx *ctx, const void *p, const char *name)
         if (st__ != LOOKAT_OK) return st__;      \
     } while (0)
 
+lookat_status encode_impl(Ctx *ctx, const void *keys, int32_t B, int64_t n, const float *codebooks,
+                          uint8_t *codes, int64_t L_max, int64_t pos, unsigned long long *near_ties);
+
 lookat_status attend_impl(Ctx *ctx, const float *lut, const void *q, const float *codebooks,
                           const uint8_t *codes, const void *v, int32_t B, int64_t L_max,
                           const int32_t *seq_lens, int64_t uniform_len, int32_t n_splits, float *out,
-                          float *scores_out)
+                          float *scores_out, const void *new_keys = nullptr, uint8_t *codes_w = nullptr,
+                          int64_t new_pos = 0)
 {
     const lookat_config &c = ctx->cfg;
     if (B < 1 || B > 65535) return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "B=%d out of range 1..65535", B);
@@ -134,6 +138,16 @@ lookat_status attend_impl(Ctx *ctx, const float *lut, const void *q, const float
     a.scale_log2 = ctx->scale * 1.4426950408889634f;
     size_t po = 0, pml = 0;
     LOOKAT_TRY(plan_attend(ctx, a, n_splits, &po, &pml));
+    if (new_keys) {
+        if (a.stream) {
+            // the streaming kernel encodes the new key itself, just before it reads the key's tile
+            a.new_keys = static_cast<const __half *>(new_keys);
+            a.codes_w = codes_w;
+            a.new_pos = (int)new_pos;
+        } else {
+            LOOKAT_TRY(encode_impl(ctx, new_keys, B, 1, codebooks, codes_w, L_max, new_pos, nullptr));
+        }
+    }
     if (!a.lut && !a.fused_lut) {
         // this shape builds its tables with the stand-alone kernel first
         const size_t need = (size_t)B * c.n_q_heads * c.m * c.K * sizeof(float);
@@ -392,6 +406,22 @@ lookat_status lookat_fit_codebooks(lookat_ctx *handle, const void *keys, int32_t
     return LOOKAT_OK;
 }
 
+lookat_status lookat_decode_step(lookat_ctx *handle, const void *q, const void *k_new, const float *codebooks,
+                                 uint8_t *codes, const void *v, int32_t B, int64_t L_max, int64_t pos,
+                                 int32_t n_splits, float *out)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    if (pos < 0 || pos >= L_max)
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "need 0 <= pos < L_max (pos=%lld L_max=%lld)", (long long)pos,
+                         (long long)L_max);
+    LOOKAT_TRY(need_ptr(ctx, k_new, "k_new"));
+    LOOKAT_TRY(need_ptr(ctx, q, "q"));
+    LOOKAT_TRY(need_ptr(ctx, codebooks, "codebooks"));
+    return attend_impl(ctx, nullptr, q, codebooks, codes, v, B, L_max, nullptr, pos + 1, n_splits, out, nullptr,
+                       k_new, codes, pos);
+}
+
 lookat_status lookat_decode_step_host(lookat_ctx *handle, const void *q_host, const void *k_new_host,
                                       const void *v_new_host, int32_t B, const float *codebooks, uint8_t *codes,
                                       void *v, int64_t L_max, int64_t pos, int32_t n_splits, float *out_host)
@@ -428,10 +458,9 @@ lookat_status lookat_decode_step_host(lookat_ctx *handle, const void *q_host, co
                               v_row, (size_t)B * c.n_kv_heads, cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return set_error(ctx, LOOKAT_ERR_CUDA, "host-to-device copy: %s", cudaGetErrorString(e));
 
-    LOOKAT_TRY(encode_impl(ctx, ctx->step_k, B, 1, codebooks, codes, L_max, pos, nullptr));
-    // attend over tokens 0..pos of every row
+    // append + attend over tokens 0..pos of every row, one launch where the shape allows
     LOOKAT_TRY(attend_impl(ctx, nullptr, ctx->step_q, codebooks, codes, v, B, L_max, nullptr, pos + 1, n_splits,
-                           ctx->step_out, nullptr));
+                           ctx->step_out, nullptr, ctx->step_k, codes, pos));
     e = cudaMemcpyAsync(out_host, ctx->step_out, out_bytes, cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return set_error(ctx, LOOKAT_ERR_CUDA, "device-to-host copy: %s", cudaGetErrorString(e));

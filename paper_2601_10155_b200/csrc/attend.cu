@@ -33,6 +33,7 @@
 #include <type_traits>
 
 #include "common.cuh"
+#include "encode_warp.cuh"
 
 namespace lookat {
 
@@ -179,6 +180,18 @@ __device__ __forceinline__ int cursor_valid(const TileCursor &c)
 {
     const int left = c.len - c.lt * kTile;
     return left >= kTile ? kTile : (left > 0 ? left : 0);
+}
+
+// Append fused into attention (Section 3.4 "Encoding" for one new key): the warp encodes the key of
+// one (batch row, KV head), stores its m codes at token new_pos and fences the stores; the caller
+// synchronises the CTA before any warp copies that tile.  Kept out of line: it runs once per unit.
+__device__ __noinline__ void append_encode_warp(const __half *x_sub, const float *book, uint8_t *code_out, int K,
+                                                int d_sub, int lane)
+{
+    const int code = nearest_centroid_warp(x_sub, book, K, d_sub, lane, nullptr);
+    if (lane == 0) *code_out = (uint8_t)code;
+    __threadfence();
+    __syncwarp();
 }
 
 #ifdef LOOKAT_PHASE_STAMPS
@@ -347,6 +360,41 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         for (int i = 0; i < DV / 16; ++i) mma_16816(acc[i], vf[i][0], vf[i][1], vf[i][2], vf[i][3], b0, b1);
     };
 
+    // ---- append: the new key of every unit whose token new_pos lies in this CTA's range is encoded
+    //      before any copy of that token's tile is issued, one warp per (unit, subspace).  Normally
+    //      that tile is far down the range and the encoding runs while the first tiles are in flight
+    //      (the barriers at the start of the first unit order it before every later copy); if the
+    //      tile is among the first STAGES tiles of a warp, the encoding comes first. ----
+    auto append_new_keys = [&]() {
+        const int u_first = (int)(T_lo / a.tiles_per_unit);
+        const int u_last = T_hi > T_lo ? (int)((T_hi - 1) / a.tiles_per_unit) : u_first - 1;
+        for (int task = warp; task < (u_last - u_first + 1) * M_SUB; task += kWarps) {
+            const int u = u_first + task / M_SUB, j = task % M_SUB;
+            const long long T_new = (long long)u * a.tiles_per_unit + (a.new_pos >> 4);
+            if (T_new >= T_lo && T_new < T_hi) {
+                const int kv_row = u / hgroups, d_sub = a.d_k / M_SUB;
+                append_encode_warp(a.new_keys + (size_t)kv_row * a.d_k + j * d_sub,
+                                   a.codebooks + ((size_t)(kv_row % a.H_kv) * M_SUB + j) * a.K * d_sub,
+                                   a.codes_w + ((size_t)kv_row * a.L_max + a.new_pos) * M_SUB + j, a.K, d_sub, lane);
+            }
+        }
+    };
+    bool append_first = false;
+    if (a.new_keys) {
+        // does a new token's tile fall into the part of the range the ring prologue covers?
+        const long long head_hi = min(T_hi, T_lo + (long long)kWarps * STAGES);
+        const long long lt_new = a.new_pos >> 4;
+        const long long u0 = T_lo / a.tiles_per_unit;
+        for (long long u = u0; u * a.tiles_per_unit < head_hi; ++u) {
+            const long long T_new = u * a.tiles_per_unit + lt_new;
+            append_first = append_first || (T_new >= T_lo && T_new < head_hi);
+        }
+        if (append_first) {
+            append_new_keys();
+            __syncthreads();
+        }
+    }
+
     // ---- prologue: fill the ring with this warp's first STAGES tiles ----
     TileCursor cc = cursor_at<M_SUB, DV>(a, T_lo + warp, hgroups);   // tile this warp consumes next
     TileCursor pc = cc;                                              // tile it copies next
@@ -355,6 +403,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         issue(pc, s);
         cursor_advance<M_SUB, DV>(a, pc, hgroups);
     }
+    if (a.new_keys && !append_first) append_new_keys();
     int slot = 0;                                          // ring slot of the consumer's tile
 
     // ---- one pass per unit this CTA's range touches ----

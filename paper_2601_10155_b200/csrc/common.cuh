@@ -63,6 +63,11 @@ struct AttendArgs {
     int d_k;
     int fused_lut;             // 1: the streaming kernel builds its tables itself
     unsigned *tickets;         // [n_units] arrival counters (streaming kernel)
+    // append fused into the streaming kernel: the key of token new_pos of every (row, KV head) is
+    // encoded by the warp that is about to copy the tile holding that token
+    const __half *new_keys;    // [B][H_kv][d_k], or null
+    uint8_t *codes_w;          // the code cache, writable
+    int new_pos;
     const uint8_t *codes;      // [B][H_kv][L_max][m]
     const __half *v;           // [B][H_kv][L_max][d_v]
     const int32_t *seq_lens;   // [B] or null

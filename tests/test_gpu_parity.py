@@ -268,6 +268,36 @@ def test_gpt2_shapes_end_to_end_with_handoff():
         check_attend(w, lk, synth.make_queries(w, q_scale), books, ref_codes, v)
 
 
+@pytest.mark.parametrize("shape", [
+    dict(B=3, n_q_heads=8, n_kv_heads=2, d_k=64, d_v=64, m=4, K=64, L=300),        # streaming kernel, fused append
+    dict(B=2, n_q_heads=16, n_kv_heads=2, d_k=128, d_v=128, m=8, K=256, L=2000),   # g = 8: two head groups per KV head
+    dict(B=2, n_q_heads=4, n_kv_heads=2, d_k=32, d_v=8, m=4, K=16, L=100),         # generic kernel: separate encode
+])
+@pytest.mark.parametrize("pos_from_end", [1, 2, 17])
+def test_decode_step_on_device_appends_then_attends(shape, pos_from_end):
+    w = synth.small_workload(**shape)
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.4)
+    books, _ = oracle.fit_codebooks(keys[:, :, :256], w.m, w.K, iters=2, seed=5)
+    pos = w.L - pos_from_end
+    ref_codes, gap = oracle.encode_keys(keys[:, :, :pos + 1], books, want_gap=True)
+    assert not ((gap[:, :, pos] > 0) & (gap[:, :, pos] < 1e-6)).any()
+    cache = np.zeros((w.B, w.n_kv_heads, w.L, w.m), np.uint8)
+    cache[:, :, :pos] = ref_codes[:, :, :pos]
+    cache[:, :, pos:] = 201 % w.K                      # stale codes where the new key goes and beyond
+    lk = ctx_for(w)
+    codes_dev = dev(cache)
+    out = lk.lookat_decode_step(dev(q), dev(np.ascontiguousarray(keys[:, :, pos])), dev(books), codes_dev, dev(v), pos)
+    torch.cuda.synchronize()
+    got = codes_dev.cpu().numpy()
+    assert np.array_equal(got[:, :, :pos + 1], ref_codes)          # row pos written, bit-exact
+    assert np.all(got[:, :, pos + 1:] == 201 % w.K)                 # nothing beyond it touched
+    ref = oracle.attend(oracle.build_lut(q, books), ref_codes, v[:, :, :pos + 1], d_k=w.d_k)
+    assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
+    # and once more: the cache now holds the new code already
+    out2 = lk.lookat_decode_step(dev(q), dev(np.ascontiguousarray(keys[:, :, pos])), dev(books), codes_dev, dev(v), pos)
+    assert np.abs(out2.cpu().numpy() - ref).max() <= OUT_TOL
+
+
 def test_decode_step_from_host_buffers():
     w = synth.small_workload(B=3, n_q_heads=8, n_kv_heads=2, d_k=64, d_v=64, m=4, K=64, L=300)
     keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.4)
