@@ -298,6 +298,33 @@ def test_decode_step_on_device_appends_then_attends(shape, pos_from_end):
     assert np.abs(out2.cpu().numpy() - ref).max() <= OUT_TOL
 
 
+def test_decode_steps_grow_the_cache_like_a_generation_loop():
+    """GPT-2 shapes, several decode steps in a row: each step appends one key and value row and attends
+    over everything so far; after every step codes and output equal the oracle's."""
+    w = synth.small_workload(B=4, n_q_heads=12, n_kv_heads=12, d_k=64, d_v=64, m=4, K=256, L=70, rank=16)
+    keys, v = synth.make_keys(w), synth.make_values(w)
+    books, _ = oracle.fit_codebooks(keys[:, :, :60], w.m, w.K, iters=3, seed=2)
+    L_max = 80                                            # 80 * 4 code bytes: rows stay 16-byte aligned
+    lk = ctx_for(w)
+    start = 61
+    ref_cache = np.zeros((w.B, w.n_kv_heads, L_max, w.m), np.uint8)
+    oracle.encode_keys(keys[:, :, :start], books, codes=ref_cache, L_max=L_max, pos=0)
+    codes_dev = dev(ref_cache)
+    v_cache = np.zeros((w.B, w.n_kv_heads, L_max, w.d_v), np.float16)
+    v_cache[:, :, :start] = v[:, :, :start]
+    v_dev = dev(v_cache)
+    for step, pos in enumerate(range(start, w.L)):
+        wq = synth.small_workload(seed=100 + step, B=w.B, n_q_heads=12, n_kv_heads=12, d_k=64, rank=16)
+        q = synth.make_queries(wq, 0.5)
+        v_dev[:, :, pos] = dev(v[:, :, pos])              # the caller stores the value row
+        out = lk.lookat_decode_step(dev(q), dev(np.ascontiguousarray(keys[:, :, pos])), dev(books), codes_dev,
+                                    v_dev, pos)
+        oracle.encode_keys(keys[:, :, pos:pos + 1], books, codes=ref_cache, L_max=L_max, pos=pos)
+        ref = oracle.attend(oracle.build_lut(q, books), ref_cache[:, :, :pos + 1], v[:, :, :pos + 1], d_k=w.d_k)
+        assert np.array_equal(codes_dev.cpu().numpy(), ref_cache)
+        assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
+
+
 def test_decode_step_from_host_buffers():
     w = synth.small_workload(B=3, n_q_heads=8, n_kv_heads=2, d_k=64, d_v=64, m=4, K=64, L=300)
     keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.4)
