@@ -173,6 +173,29 @@ def reconstruct_keys(codes, codebooks):
     return k_hat
 
 
+def attend_prefill(q, codebooks, codes, v, q_pos0=0, scale=None, want_scores=False):
+    """Causal multi-query attention over the compressed keys: q fp16 [B][H_q][L_q][d_k]; query i stands
+    at position q_pos0 + i and attends tokens 0..q_pos0+i.  Returns out fp64 [B][H_q][L_q][d_v]."""
+    q = _f16(q)
+    codebooks = np.ascontiguousarray(codebooks, dtype=np.float32)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    v = _f16(v)
+    B, H_q, L_q, d_k = q.shape
+    H_kv, m, K, d_sub = codebooks.shape
+    _, _, L_max, _ = codes.shape
+    d_v = v.shape[3]
+    assert m * d_sub == d_k and H_q % H_kv == 0 and q_pos0 >= 0 and q_pos0 + L_q <= L_max
+    assert int(codes.max(initial=0)) < K
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d_k))
+    out = np.empty((B, H_q, L_q, d_v), dtype=np.float64)
+    scores = np.full((B, H_q, L_q, L_max), np.nan) if want_scores else None
+    _load().oracle_attend_prefill(_p(q), _p(codebooks), _p(codes), _p(v), B, H_q, H_kv, ctypes.c_int64(L_q),
+                                  ctypes.c_int64(L_max), ctypes.c_int64(q_pos0), d_k, d_v, m, K,
+                                  ctypes.c_double(scale), _p(out), _p(scores))
+    return (out, scores) if want_scores else out
+
+
 def decode_step(q, codebooks, codes, v, seq_lens=None, scale=None):
     """Algorithm 1 as a whole: build the tables, then attend."""
     return attend(build_lut(q, codebooks), codes, v, seq_lens=seq_lens, scale=scale,

@@ -349,3 +349,59 @@ void oracle_reconstruct_keys(const uint8_t *codes, int B, int H_kv, int64_t L_ma
             }
     }
 }
+
+/*
+ * Multi-query causal attention over the compressed keys (prefill): Algorithm 1 applied to each of
+ * L_q queries per head, query i standing at position q_pos0 + i and attending tokens 0..q_pos0+i.
+ * q fp16 [B][H_q][L_q][d_k]; out fp64 [B][H_q][L_q][d_v]; scores (optional) fp64
+ * [B][H_q][L_q][L_max], entries beyond a query's position untouched.
+ */
+void oracle_attend_prefill(const uint16_t *q, const float *codebooks, const uint8_t *codes, const uint16_t *v,
+                           int B, int H_q, int H_kv, int64_t L_q, int64_t L_max, int64_t q_pos0, int d_k,
+                           int d_v, int m, int K, double scale, double *out, double *scores)
+{
+    int g = H_q / H_kv, d_sub = d_k / m;
+    int64_t units = (int64_t)B * H_q * L_q;
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int64_t u = 0; u < units; ++u) {
+        int64_t i = u % L_q;
+        int hq = (int)((u / L_q) % H_q), b = (int)(u / (L_q * H_q));
+        int h = hq / g;
+        int64_t L = q_pos0 + i + 1;
+        const uint16_t *qi = q + (size_t)u * d_k;
+        const uint8_t *cd = codes + ((size_t)b * H_kv + h) * L_max * m;
+        const uint16_t *vv = v + ((size_t)b * H_kv + h) * L_max * d_v;
+        double *o = out + (size_t)u * d_v;
+        double *T = (double *)malloc(sizeof(double) * m * K);
+        double *s = (double *)malloc(sizeof(double) * L);
+        /* first loop of Algorithm 1: the tables of this query */
+        for (int j = 0; j < m; ++j)
+            for (int c = 0; c < K; ++c) {
+                const float *cen = codebooks + (((size_t)h * m + j) * K + c) * d_sub;
+                double acc = 0.0;
+                for (int t = 0; t < d_sub; ++t) acc += half_to_double(qi[j * d_sub + t]) * (double)cen[t];
+                T[j * K + c] = acc;
+            }
+        /* second loop and continuation */
+        double M = -INFINITY;
+        for (int64_t l = 0; l < L; ++l) {
+            double acc = 0.0;
+            for (int j = 0; j < m; ++j) acc += T[(size_t)j * K + cd[l * m + j]];
+            s[l] = acc;
+            if (scores) scores[(size_t)u * L_max + l] = acc;
+            if (acc * scale > M) M = acc * scale;
+        }
+        double Z = 0.0;
+        for (int64_t l = 0; l < L; ++l) {
+            s[l] = exp(s[l] * scale - M);
+            Z += s[l];
+        }
+        for (int t = 0; t < d_v; ++t) o[t] = 0.0;
+        for (int64_t l = 0; l < L; ++l) {
+            double a = s[l] / Z;
+            for (int t = 0; t < d_v; ++t) o[t] += a * half_to_double(vv[l * d_v + t]);
+        }
+        free(T);
+        free(s);
+    }
+}

@@ -311,3 +311,30 @@ def test_kmeans_init_rule_and_empty_clusters():
     assert np.all(trace == 0)
     codes = oracle.encode_keys(keys, books)
     assert codes.max() < 5
+
+
+# ---------------------------------------------------------------- causal multi-query (prefill)
+def test_prefill_is_algorithm_1_per_query_and_exact_attention_in_the_exact_case():
+    rng = np.random.default_rng(21)
+    B, H_q, H_kv, d_k, d_v, L, K = 2, 4, 2, 8, 8, 23, 9
+    levels = (rng.permutation(64)[:K] - 32) / 8.0
+    keys = rng.choice(levels, size=(B, H_kv, L, d_k)).astype(np.float16)
+    v = rng.standard_normal((B, H_kv, L, d_v)).astype(np.float16)
+    qs = (0.5 * rng.standard_normal((B, H_q, 7, d_k))).astype(np.float16)
+    books = np.broadcast_to(levels.astype(np.float32)[None, None, :, None], (H_kv, d_k, K, 1)).copy()
+    codes = oracle.encode_keys(keys, books)
+    q_pos0 = L - 7
+    out, scores = oracle.attend_prefill(qs, books, codes, v, q_pos0=q_pos0, want_scores=True)
+    g = H_q // H_kv
+    for i in range(7):
+        n = q_pos0 + i + 1
+        # the decode routine on the prefix (itself pinned above) ...
+        ref = oracle.attend(oracle.build_lut(qs[:, :, i], books), codes[:, :, :n], v[:, :, :n], d_k=d_k)
+        np.testing.assert_allclose(out[:, :, i], ref, rtol=1e-12, atol=1e-14)
+        # ... and plain causal softmax attention written with numpy (codebooks reproduce the keys exactly)
+        s_ref = np.einsum("bhd,bhld->bhl", qs[:, :, i].astype(np.float64),
+                          np.repeat(keys[:, :, :n].astype(np.float64), g, axis=1))
+        np.testing.assert_allclose(scores[:, :, i, :n], s_ref, rtol=1e-12, atol=1e-13)
+        assert np.isnan(scores[:, :, i, n:]).all()
+        np.testing.assert_allclose(out[:, :, i], _softmax_attention_numpy(s_ref, v[:, :, :n], d_k ** -0.5, g),
+                                   rtol=1e-12, atol=1e-14)
