@@ -165,6 +165,27 @@ lookat_status lookat_attend_static(lookat_ctx *ctx, const float *lut, const void
                                    const int32_t *seq_lens, int32_t n_splits, float *out, float *scores_out);
 
 /*
+ * Multi-query causal attention over the compressed keys (prefill): Algorithm
+ * 1 for each of L_q consecutive queries per head.  Query i stands at position
+ * q_pos0 + i and attends tokens 0 .. q_pos0 + i of the cache (its own
+ * quantised key included, so the keys up to q_pos0 + L_q - 1 must have been
+ * encoded).  The tables of a tile of queries are built on chip.
+ *
+ *   q           fp16 [B][H_q][L_q][d_k]
+ *   codes       uint8 [B][H_kv][L_max][m]
+ *   v           fp16 [B][H_kv][L_max][d_v]
+ *   out         fp32 [B][H_q][L_q][d_v]
+ *   scores_out  NULL, or fp32 [B][H_q][L_q][L_max]: raw unscaled s for the
+ *               visible (query, token) pairs (validation only)
+ * Requires 0 <= q_pos0, q_pos0 + L_q <= L_max.  d_v must be a multiple of 32
+ * (of 16 where tables of 16 queries fit in shared memory) and at most 256;
+ * otherwise LOOKAT_ERR_UNSUPPORTED.
+ */
+lookat_status lookat_attend_prefill(lookat_ctx *ctx, const void *q, const float *codebooks, const uint8_t *codes,
+                                    const void *v, int32_t B, int64_t L_q, int64_t L_max, int64_t q_pos0,
+                                    float *out, float *scores_out);
+
+/*
  * One decode step on device buffers: append and attend.  The new key of every
  * (batch row, KV head) is encoded at token `pos` of the code cache (Section
  * 3.4, Encoding), then Algorithm 1 runs over tokens 0..pos with tables built

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_PKG, "liblookat.so")
 EXPORTS = [
     "lookat_create", "lookat_destroy", "lookat_last_error", "lookat_fit_codebooks",
     "lookat_encode_keys", "lookat_build_lut", "lookat_attend", "lookat_attend_static",
-    "lookat_decode_step", "lookat_decode_step_host",
+    "lookat_attend_prefill", "lookat_decode_step", "lookat_decode_step_host",
     "lookat_kernel_launches", "lookat_set_timing", "lookat_attend_kernel_ms",
 ]
 
@@ -69,6 +69,8 @@ def load_library() -> ctypes.CDLL:
     lib.lookat_attend.restype = ctypes.c_int
     lib.lookat_attend_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, vp, i32, vp, vp]
     lib.lookat_attend_static.restype = ctypes.c_int
+    lib.lookat_attend_prefill.argtypes = [vp, vp, vp, vp, vp, i32, i64, i64, i64, vp, vp]
+    lib.lookat_attend_prefill.restype = ctypes.c_int
     lib.lookat_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, i64, i32, vp]
     lib.lookat_decode_step.restype = ctypes.c_int
     lib.lookat_decode_step_host.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i64, i64, i32, vp]
@@ -229,6 +231,21 @@ class Lookat:
             _dev(seq_lens, torch.int32, "seq_lens", (B,)), n_splits,
             _dev(out, torch.float32, "out", (B, c.n_q_heads, c.d_v)),
             _dev(scores_out, torch.float32, "scores_out", (B, c.n_q_heads, L_max))))
+        return out
+
+    def lookat_attend_prefill(self, q, codebooks, codes, v, q_pos0=0, out=None, scores_out=None):
+        c = self.cfg
+        B, H, L_max, m = codes.shape
+        L_q = q.shape[2]
+        if out is None:
+            out = torch.empty((B, c.n_q_heads, L_q, c.d_v), dtype=torch.float32, device=self.device)
+        self._check(self._lib.lookat_attend_prefill(
+            self._h, _dev(q, torch.float16, "q", (B, c.n_q_heads, L_q, c.d_k)),
+            _dev(codebooks, torch.float32, "codebooks", (c.n_kv_heads, c.m, c.K, self.d_sub)),
+            _dev(codes, torch.uint8, "codes", (B, c.n_kv_heads, L_max, c.m)),
+            _dev(v, torch.float16, "v", (B, c.n_kv_heads, L_max, c.d_v)), B, L_q, L_max, q_pos0,
+            _dev(out, torch.float32, "out", (B, c.n_q_heads, L_q, c.d_v)),
+            _dev(scores_out, torch.float32, "scores_out", (B, c.n_q_heads, L_q, L_max))))
         return out
 
     def lookat_decode_step(self, q, k_new, codebooks, codes, v, pos, out=None, n_splits=0):

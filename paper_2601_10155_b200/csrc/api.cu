@@ -406,6 +406,51 @@ lookat_status lookat_fit_codebooks(lookat_ctx *handle, const void *keys, int32_t
     return LOOKAT_OK;
 }
 
+lookat_status lookat_attend_prefill(lookat_ctx *handle, const void *q, const float *codebooks, const uint8_t *codes,
+                                    const void *v, int32_t B, int64_t L_q, int64_t L_max, int64_t q_pos0, float *out,
+                                    float *scores_out)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    const lookat_config &c = ctx->cfg;
+    if (B < 1 || B > 65535) return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "B=%d out of range 1..65535", B);
+    if (c.n_q_heads > 65535) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "more than 65535 query heads");
+    if (L_q < 1 || L_max < 1 || q_pos0 < 0 || q_pos0 + L_q > L_max || L_max > (1ll << 30))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG,
+                         "need 1 <= L_q, 0 <= q_pos0, q_pos0 + L_q <= L_max (L_q=%lld q_pos0=%lld L_max=%lld)",
+                         (long long)L_q, (long long)q_pos0, (long long)L_max);
+    LOOKAT_TRY(need_ptr(ctx, q, "q"));
+    LOOKAT_TRY(need_ptr(ctx, codebooks, "codebooks"));
+    LOOKAT_TRY(need_ptr(ctx, codes, "codes"));
+    LOOKAT_TRY(need_ptr(ctx, v, "v"));
+    LOOKAT_TRY(need_ptr(ctx, out, "out"));
+    if (scores_out && (reinterpret_cast<uintptr_t>(scores_out) & 3u))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "scores_out is not 4-byte aligned");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return set_error(ctx, LOOKAT_ERR_CUDA, "cannot select device %d", ctx->device);
+    PrefillArgs a;
+    memset(&a, 0, sizeof(a));
+    a.q = static_cast<const __half *>(q);
+    a.codebooks = codebooks;
+    a.codes = codes;
+    a.v = static_cast<const __half *>(v);
+    a.out = out;
+    a.scores_out = scores_out;
+    a.B = B;
+    a.H_q = c.n_q_heads;
+    a.H_kv = c.n_kv_heads;
+    a.g = c.n_q_heads / c.n_kv_heads;
+    a.d_k = c.d_k;
+    a.d_v = c.d_v;
+    a.m = c.m;
+    a.K = c.K;
+    a.L_q = L_q;
+    a.L_max = L_max;
+    a.q_pos0 = q_pos0;
+    a.scale_log2 = ctx->scale * 1.4426950408889634f;
+    return launch_prefill(ctx, a);
+}
+
 lookat_status lookat_decode_step(lookat_ctx *handle, const void *q, const void *k_new, const float *codebooks,
                                  uint8_t *codes, const void *v, int32_t B, int64_t L_max, int64_t pos,
                                  int32_t n_splits, float *out)

@@ -98,6 +98,19 @@ lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_
 lookat_status launch_attend(Ctx *ctx, const AttendArgs &a);
 lookat_status launch_combine(Ctx *ctx, const AttendArgs &a);
 
+struct PrefillArgs {
+    const __half *q;           // [B][H_q][L_q][d_k]
+    const float *codebooks;    // [H_kv][m][K][d_sub]
+    const uint8_t *codes;      // [B][H_kv][L_max][m]
+    const __half *v;           // [B][H_kv][L_max][d_v]
+    float *out;                // [B][H_q][L_q][d_v]
+    float *scores_out;         // [B][H_q][L_q][L_max] or null
+    int B, H_q, H_kv, g, d_k, d_v, m, K;
+    long long L_q, L_max, q_pos0;
+    float scale_log2;
+};
+lookat_status launch_prefill(Ctx *ctx, const PrefillArgs &a);
+
 lookat_status launch_build_lut(Ctx *ctx, const __half *q, int B, const float *codebooks, float *lut);
 
 struct EncodeArgs {

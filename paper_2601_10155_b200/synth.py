@@ -66,6 +66,8 @@ WORKLOADS = {
     "gpt2_b32_l1024_m4": Workload("gpt2_b32_l1024_m4", 1002, 32, 12, 12, 64, 64, 1024, 4),
     "gqa_32k_m8": Workload("gqa_32k_m8", 1003, 16, 32, 8, 128, 128, 32768, 8, rank=32,
                            scales="student_t3", fit_iters=10, fit_keys_per_head=65536),
+    "prefill_4k_m16": Workload("prefill_4k_m16", 1004, 4, 32, 32, 128, 128, 4096, 16, rank=32,
+                               fit_iters=10),
     "encode_1m_m16": Workload("encode_1m_m16", 1004, 1, 1, 1, 128, 128, 1048576, 16, rank=32,
                               fit_iters=10, fit_keys_per_head=262144),
 }
@@ -144,6 +146,18 @@ def make_queries(w: Workload, q_scale: float = 1.0) -> np.ndarray:
         rng = np.random.default_rng([w.seed, w.layer, hq, 3])
         rows = draw_rows(rng, A, w.B).astype(np.float64) * q_scale
         q[:, hq] = rows.astype(np.float16)
+    return q
+
+
+def make_prefill_queries(w: Workload, L_q: int, q_scale: float = 1.0) -> np.ndarray:
+    """fp16 queries [B][n_q_heads][L_q][d_k] for multi-query (prefill) attention, drawn like the
+    decode queries: query head hq shares the subspace of KV head hq // g."""
+    q = np.empty((w.B, w.n_q_heads, L_q, w.d_k), dtype=np.float16)
+    for hq in range(w.n_q_heads):
+        A = head_mixing_matrix(w.seed, w.layer, hq // w.g, w.d_k, w.rank, w.scales)
+        rng = np.random.default_rng([w.seed, w.layer, hq, 5])
+        rows = draw_rows(rng, A, w.B * L_q).astype(np.float64) * q_scale
+        q[:, hq] = rows.astype(np.float16).reshape(w.B, L_q, w.d_k)
     return q
 
 

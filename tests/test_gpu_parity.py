@@ -367,3 +367,34 @@ def test_invalid_arguments_are_rejected_without_launching():
         kw.update(bad)
         with pytest.raises(LookatError):
             Lookat(**kw)
+
+
+# ------------------------------------------------------------------ causal multi-query (prefill)
+@pytest.mark.parametrize("shape,L_q,q_pos0", [
+    (dict(B=2, n_q_heads=4, n_kv_heads=2, d_k=64, d_v=64, m=4, K=256, L=150), 150, 0),      # whole prompt
+    (dict(B=1, n_q_heads=8, n_kv_heads=2, d_k=128, d_v=128, m=8, K=256, L=200), 37, 163),   # a late slice
+    (dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=128, d_v=128, m=16, K=256, L=130), 130, 0),   # tables of 8 queries
+    (dict(B=2, n_q_heads=2, n_kv_heads=1, d_k=32, d_v=32, m=2, K=16, L=70), 1, 69),         # one query = a decode step
+    (dict(B=1, n_q_heads=3, n_kv_heads=3, d_k=24, d_v=16, m=8, K=7, L=65), 65, 0),          # d_sub 3, small K
+])
+@pytest.mark.parametrize("q_scale", [1.0, 0.1])
+def test_attend_prefill_matches_oracle(shape, L_q, q_pos0, q_scale):
+    w = synth.small_workload(**shape)
+    keys, v = synth.make_keys(w), synth.make_values(w)
+    q = synth.make_prefill_queries(w, L_q, q_scale)
+    books, _ = oracle.fit_codebooks(keys[:, :, :min(w.L, 300)], w.m, w.K, iters=2, seed=3)
+    codes = oracle.encode_keys(keys, books)
+    ref, ref_s = oracle.attend_prefill(q, books, codes, v, q_pos0=q_pos0, want_scores=True)
+    lk = ctx_for(w)
+    scores = torch.full((w.B, w.n_q_heads, L_q, w.L), float("nan"), device="cuda")
+    out = lk.lookat_attend_prefill(dev(q), dev(books), dev(codes), dev(v), q_pos0=q_pos0, scores_out=scores)
+    torch.cuda.synchronize()
+    s = scores.cpu().numpy().astype(np.float64)
+    visible = ~np.isnan(ref_s)
+    assert np.array_equal(np.isnan(s), ~visible), "scores written for hidden pairs or missing for visible ones"
+    assert np.all(np.abs(s[visible] - ref_s[visible]) <= SCORE_TOL * (1 + np.abs(ref_s[visible])))
+    assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
+    # the last query of a whole prompt is a decode step over the same cache
+    if q_pos0 + L_q == w.L:
+        dec = lk.lookat_attend(dev(codes), dev(v), q=dev(np.ascontiguousarray(q[:, :, -1])), codebooks=dev(books))
+        assert float((dec - out[:, :, -1]).abs().max()) <= 2e-5
