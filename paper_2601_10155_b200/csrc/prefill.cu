@@ -4,18 +4,22 @@
 //
 // One CTA per (query tile, query head, batch row), 512 threads:
 //   * the tile's lookup tables (Section 3.5 "Precomputation Lookup Tables") are
-//     built once into shared memory, query-minor: lut[j][c][ql], so the TQ
-//     lanes that score one token for the TQ queries read one contiguous row
-//     (fp64 accumulation, one rounding, as everywhere in this library),
-//   * tokens are walked in chunks of 64; the codes and V rows of the next chunk
-//     are copied (cp.async) while the current one is worked on,
-//   * every (query, token) pair is scored by m gathers (Section 3.5 "Lookup and
-//     Sum") and masked causally; one warp per query row keeps the online
-//     softmax (running maximum and sum, base 2) and writes the weights as two
-//     fp16 planes: the rounding and what the rounding left over (~22 bits),
-//   * the weighted value sum O[TQ x d_v] += P[TQ x 64] . V[64 x d_v] runs on the
-//     tensor cores (mma.sync m16n8k16, fp32 accumulate), once per plane; a warp
-//     owns 8 output columns, the V operand comes from the row-major rows by
+//     built once into shared memory, query-minor: lut[j][c][ql], so one 16-byte
+//     read serves one token for 4 queries (fp64 accumulation, one rounding, as
+//     everywhere in this library),
+//   * the CTA's two halves (8 warps each, each with its own hardware barrier)
+//     share the tables and walk alternate chunks of CHUNK tokens on their own,
+//     so one half's copies, gathers, softmax and value sum overlap the other's;
+//     each half keeps its own running maximum, sum and accumulators, merged at
+//     the end,
+//   * per chunk: codes and V rows are copied to shared memory (cp.async), every
+//     (query, token) pair is scored by m gathers (Section 3.5 "Lookup and Sum")
+//     and masked causally, one warp per query row updates the online softmax
+//     (base 2) and writes the weights as two fp16 planes (the rounding and what
+//     it left over, ~22 bits), and the weighted value sum
+//     O[TQ x d_v] += P[TQ x CHUNK] . V[CHUNK x d_v] runs on the tensor cores
+//     (mma.sync m16n8k16, fp32 accumulate), once per plane; a warp owns 8-column
+//     slices of the output, the V operand comes from the row-major rows by
 //     ldmatrix with transpose.
 // The cost is bound by the shared-memory gathers (m per pair); the tables cost
 // K*d_k multiply-adds per query.
@@ -27,33 +31,43 @@ namespace {
 
 constexpr int kPfWarps = 16;
 constexpr int kPfThreads = kPfWarps * 32;
-constexpr int kPfChunk = 64;
-constexpr int kPfSPitch = kPfChunk + 1;       // fp32 score rows, padded by one float
-constexpr int kPfPPitch = kPfChunk + 8;       // fp16 weight rows, padded by 16 bytes
+constexpr int kPfGroupWarps = 8;                  // warps per half
+constexpr int kPfGroupThreads = kPfGroupWarps * 32;
+constexpr int kPfMaxSlices = 4;                   // 8-column output slices per warp (d_v <= 256)
 constexpr float kPfNegBig = -1.0e30f;
 
+// tokens per chunk (64 or 128): fp32 score rows are padded by one float, fp16 weight rows by 16 bytes
+__host__ __device__ constexpr int pf_s_pitch(int chunk) { return chunk + 1; }
+__host__ __device__ constexpr int pf_p_pitch(int chunk) { return chunk + 8; }
 __host__ __device__ inline size_t pf_align16(size_t x) { return (x + 15) & ~(size_t)15; }
 
+// Shared-memory map; the per-half regions are `*_bytes` apart.
 struct PfLayout {
     unsigned lut, qd, codes, v, s, p_hi, p_lo, state, total;
+    unsigned codes_bytes, v_bytes, s_bytes, p_bytes, state_bytes;
     unsigned v_pitch;      // bytes per staged V row (row + 16 bytes)
     unsigned code_pitch;   // bytes per staged code row (m rounded up to 4)
 };
 
-PfLayout pf_layout(int tq, int d_k, int d_v, int m, int K)
+PfLayout pf_layout(int tq, int chunk, int d_k, int d_v, int m, int K)
 {
     PfLayout l;
     size_t off = 0;
     l.v_pitch = (unsigned)(d_v * 2 + 16);
     l.code_pitch = (unsigned)((m + 3) & ~3);
+    l.codes_bytes = (unsigned)pf_align16((size_t)chunk * l.code_pitch);
+    l.v_bytes = (unsigned)pf_align16((size_t)chunk * l.v_pitch);
+    l.s_bytes = (unsigned)pf_align16((size_t)tq * pf_s_pitch(chunk) * 4);
+    l.p_bytes = (unsigned)pf_align16((size_t)16 * pf_p_pitch(chunk) * 2);
+    l.state_bytes = (unsigned)pf_align16((size_t)3 * 16 * 4);
     l.lut = (unsigned)off;   off += pf_align16((size_t)m * K * tq * 4);
     l.qd = (unsigned)off;    off += pf_align16((size_t)tq * d_k * 8);
-    l.codes = (unsigned)off; off += 2 * pf_align16((size_t)kPfChunk * l.code_pitch);
-    l.v = (unsigned)off;     off += 2 * pf_align16((size_t)kPfChunk * l.v_pitch);
-    l.s = (unsigned)off;     off += pf_align16((size_t)tq * kPfSPitch * 4);
-    l.p_hi = (unsigned)off;  off += pf_align16((size_t)16 * kPfPPitch * 2);
-    l.p_lo = (unsigned)off;  off += pf_align16((size_t)16 * kPfPPitch * 2);
-    l.state = (unsigned)off; off += pf_align16((size_t)3 * 16 * 4);
+    l.codes = (unsigned)off; off += 2 * (size_t)l.codes_bytes;
+    l.v = (unsigned)off;     off += 2 * (size_t)l.v_bytes;
+    l.s = (unsigned)off;     off += 2 * (size_t)l.s_bytes;
+    l.p_hi = (unsigned)off;  off += 2 * (size_t)l.p_bytes;
+    l.p_lo = (unsigned)off;  off += 2 * (size_t)l.p_bytes;
+    l.state = (unsigned)off; off += 2 * (size_t)l.state_bytes;
     l.total = (unsigned)off;
     return l;
 }
@@ -68,6 +82,11 @@ __device__ __forceinline__ void pf_cp_async4(unsigned dst, const void *src)
 }
 __device__ __forceinline__ void pf_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void pf_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+// hardware barrier of one half of the CTA (ids 1 and 2; id 0 is __syncthreads)
+__device__ __forceinline__ void pf_group_barrier(int group)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(group + 1), "n"(kPfGroupThreads) : "memory");
+}
 
 __device__ __forceinline__ void pf_ldmatrix_x4(uint32_t (&r)[4], unsigned src)
 {
@@ -90,23 +109,16 @@ __device__ __forceinline__ void pf_mma(float (&c)[4], const uint32_t (&a)[4], ui
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <int TQ>
+template <int TQ, int CHUNK>
 __global__ void __launch_bounds__(kPfThreads, 1) attend_prefill_kernel(PrefillArgs a, PfLayout lay)
 {
+    constexpr int S_PITCH = pf_s_pitch(CHUNK), P_PITCH = pf_p_pitch(CHUNK);
     extern __shared__ __align__(16) unsigned char smem[];
-    float *lut = reinterpret_cast<float *>(smem + lay.lut);           // [m][K][TQ]
-    double *qd = reinterpret_cast<double *>(smem + lay.qd);           // [TQ][d_k]
-    float *s_s = reinterpret_cast<float *>(smem + lay.s);             // [TQ][65]
-    __half *p_hi = reinterpret_cast<__half *>(smem + lay.p_hi);       // [16][72]
-    __half *p_lo = reinterpret_cast<__half *>(smem + lay.p_lo);       // [16][72]
-    float *m_run = reinterpret_cast<float *>(smem + lay.state);       // [16]
-    float *l_run = m_run + 16;
-    float *alpha_s = l_run + 16;
     const unsigned smem_s = (unsigned)__cvta_generic_to_shared(smem);
-    const unsigned codes_bytes = (unsigned)pf_align16((size_t)kPfChunk * lay.code_pitch);
-    const unsigned v_bytes = (unsigned)pf_align16((size_t)kPfChunk * lay.v_pitch);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int grp = warp / kPfGroupWarps;                             // which half of the CTA
+    const int gw = warp % kPfGroupWarps, gtid = tid % kPfGroupThreads;
     const int qtile = gridDim.x - 1 - blockIdx.x;                     // long tiles first
     const int hq = blockIdx.y, b = blockIdx.z;
     const int kvh = hq / a.g;
@@ -114,55 +126,31 @@ __global__ void __launch_bounds__(kPfThreads, 1) attend_prefill_kernel(PrefillAr
     const int nq = (int)min((long long)TQ, a.L_q - q0);
     const int d_sub = a.d_k / a.m;
 
+    float *lut = reinterpret_cast<float *>(smem + lay.lut);                          // [m][K][TQ]
+    double *qd = reinterpret_cast<double *>(smem + lay.qd);                          // [TQ][d_k]
+    // this half's regions
+    unsigned char *codes_s = smem + lay.codes + grp * lay.codes_bytes;               // [CHUNK][code_pitch]
+    unsigned char *v_sm = smem + lay.v + grp * lay.v_bytes;                          // [CHUNK][v_pitch]
+    float *s_s = reinterpret_cast<float *>(smem + lay.s + grp * lay.s_bytes);        // [TQ][S_PITCH]
+    __half *p_hi = reinterpret_cast<__half *>(smem + lay.p_hi + grp * lay.p_bytes);  // [16][P_PITCH]
+    __half *p_lo = reinterpret_cast<__half *>(smem + lay.p_lo + grp * lay.p_bytes);
+    float *m_run = reinterpret_cast<float *>(smem + lay.state + grp * lay.state_bytes);   // [16] each
+    float *l_run = m_run + 16;
+    float *alpha_s = l_run + 16;
+
     // ---- queries of the tile, widened; weight planes start as zeros (rows TQ..15 stay zero) ----
     const __half *qrow = a.q + (((size_t)b * a.H_q + hq) * a.L_q + q0) * a.d_k;
     for (int i = tid; i < TQ * a.d_k; i += kPfThreads)
         qd[i] = (i / a.d_k) < nq ? (double)__half2float(qrow[i]) : 0.0;
-    for (int i = tid; i < 16 * kPfPPitch; i += kPfThreads) {
+    for (int i = gtid; i < 16 * P_PITCH; i += kPfGroupThreads) {
         p_hi[i] = __float2half(0.f);
         p_lo[i] = __float2half(0.f);
     }
-    if (tid < 16) {
-        m_run[tid] = kPfNegBig;
-        l_run[tid] = 0.f;
-        alpha_s[tid] = 1.f;
+    if (gtid < 16) {
+        m_run[gtid] = kPfNegBig;
+        l_run[gtid] = 0.f;
+        alpha_s[gtid] = 1.f;
     }
-
-    const size_t kv_row = (size_t)b * a.H_kv + kvh;
-    const uint8_t *codes = a.codes + kv_row * a.L_max * a.m;
-    const unsigned char *vrow = reinterpret_cast<const unsigned char *>(a.v + kv_row * a.L_max * a.d_v);
-    const long long pos0 = a.q_pos0 + q0;                             // position of the tile's first query
-    const long long n_tok = pos0 + nq;                                // tokens the tile's last query sees
-    const int v_vec = a.d_v / 8;                                      // 16-byte pieces per V row
-    const bool codes_by_word = (a.m & 3) == 0 && ((uintptr_t)codes & 3) == 0;
-
-    // copies of chunk `c0` into buffer `buf`; rows beyond the chunk's tokens are zeros
-    auto stage = [&](long long c0, int buf) {
-        const int n = (int)min((long long)kPfChunk, n_tok - c0);
-        unsigned char *cdst = smem + lay.codes + buf * codes_bytes;
-        const unsigned cdst_s = smem_s + lay.codes + buf * codes_bytes;
-        if (codes_by_word) {
-            const int words = a.m >> 2;
-            for (int i = tid; i < kPfChunk * words; i += kPfThreads) {
-                if (i / words < n) pf_cp_async4(cdst_s + i * 4, codes + c0 * a.m + (size_t)i * 4);
-                else reinterpret_cast<uint32_t *>(cdst)[i] = 0u;
-            }
-        } else {
-            for (int i = tid; i < kPfChunk * a.m; i += kPfThreads) {
-                const int tl = i / a.m, j = i - tl * a.m;
-                cdst[tl * lay.code_pitch + j] = tl < n ? codes[(c0 + tl) * a.m + j] : 0;
-            }
-        }
-        unsigned char *vdst = smem + lay.v + buf * v_bytes;
-        const unsigned vdst_s = smem_s + lay.v + buf * v_bytes;
-        for (int i = tid; i < kPfChunk * v_vec; i += kPfThreads) {
-            const int tl = i / v_vec, piece = i - tl * v_vec;
-            if (tl < n) pf_cp_async16(vdst_s + tl * lay.v_pitch + piece * 16, vrow + ((size_t)(c0 + tl) * v_vec + piece) * 16);
-            else *reinterpret_cast<uint4 *>(vdst + tl * lay.v_pitch + piece * 16) = make_uint4(0, 0, 0, 0);
-        }
-        pf_commit();
-    };
-    stage(0, 0);                                                       // overlaps the table build
     __syncthreads();
 
     // ---- tables of the tile: lut[j][c][ql] = q_ql^(j) . C_j[c], fp64 accumulation ----
@@ -171,77 +159,133 @@ __global__ void __launch_bounds__(kPfThreads, 1) attend_prefill_kernel(PrefillAr
         const int j = e / a.K;
         const float *cen = book + (size_t)e * d_sub;
         const double *qj = qd + j * d_sub;
-        double acc[TQ];
+        double t[TQ];
 #pragma unroll
-        for (int ql = 0; ql < TQ; ++ql) acc[ql] = 0.0;
+        for (int ql = 0; ql < TQ; ++ql) t[ql] = 0.0;
         for (int i = 0; i < d_sub; ++i) {
             const double cv = (double)__ldg(cen + i);
 #pragma unroll
-            for (int ql = 0; ql < TQ; ++ql) acc[ql] = fma(qj[ql * a.d_k + i], cv, acc[ql]);
+            for (int ql = 0; ql < TQ; ++ql) t[ql] = fma(qj[ql * a.d_k + i], cv, t[ql]);
         }
 #pragma unroll
         for (int ql = 0; ql < TQ; ql += 4)
             *reinterpret_cast<float4 *>(lut + (size_t)e * TQ + ql) =
-                make_float4((float)acc[ql], (float)acc[ql + 1], (float)acc[ql + 2], (float)acc[ql + 3]);
+                make_float4((float)t[ql], (float)t[ql + 1], (float)t[ql + 2], (float)t[ql + 3]);
     }
+    __syncthreads();
 
-    // value-sum ownership: warp w accumulates output columns 8*nt .. 8*nt+7 for nt = w, w+16
-    float acc[2][4];
-#pragma unroll
-    for (int t = 0; t < 2; ++t) acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
-    const int n_tiles = a.d_v / 8;
+    const size_t kv_row = (size_t)b * a.H_kv + kvh;
+    const uint8_t *codes = a.codes + kv_row * a.L_max * a.m;
+    const unsigned char *vrow = reinterpret_cast<const unsigned char *>(a.v + kv_row * a.L_max * a.d_v);
+    const long long pos0 = a.q_pos0 + q0;                             // position of the tile's first query
+    const long long n_tok = pos0 + nq;                                // tokens the tile's last query sees
+    const int v_vec = a.d_v / 8;                                      // 16-byte pieces per V row
+    const bool codes_by_word = (a.m & 3) == 0;
+    const int n_slices = a.d_v / 8;                                   // 8-column output slices
     float *scores_base =
         a.scores_out ? a.scores_out + (((size_t)b * a.H_q + hq) * a.L_q + q0) * a.L_max : nullptr;
+
+    // value-sum ownership: warp gw of a half accumulates output slices gw, gw+8, gw+16, gw+24
+    float acc[kPfMaxSlices][4];
+#pragma unroll
+    for (int t = 0; t < kPfMaxSlices; ++t) acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
     // ldmatrix lane addresses: weights (rows lane&15, tokens 8*(lane>>4)); V (tokens lane&15 of a
-    // 16-token step, this warp's 8 columns; lanes 16..31 repeat valid addresses that are not used)
-    const unsigned p_lane = (unsigned)(((lane & 15) * kPfPPitch + (lane >> 4) * 8) * 2);
+    // 16-token step; lanes 16..31 repeat valid addresses that are not used)
+    const unsigned p_lane = (unsigned)(((lane & 15) * P_PITCH + (lane >> 4) * 8) * 2);
     const unsigned v_lane = (unsigned)((lane & 15) * lay.v_pitch);
+    const unsigned p_hi_s = smem_s + lay.p_hi + grp * lay.p_bytes, p_lo_s = smem_s + lay.p_lo + grp * lay.p_bytes;
+    const unsigned v_s = smem_s + lay.v + grp * lay.v_bytes;
+    const unsigned codes_ss = smem_s + lay.codes + grp * lay.codes_bytes;
 
-    int buf = 0;
-    for (long long c0 = 0; c0 < n_tok; c0 += kPfChunk, buf ^= 1) {
-        const int n = (int)min((long long)kPfChunk, n_tok - c0);
+    // ---- this half's chunks: grp, grp+2, grp+4, ... ----
+    for (long long c0 = (long long)grp * CHUNK; c0 < n_tok; c0 += 2 * CHUNK) {
+        const int n = (int)min((long long)CHUNK, n_tok - c0);
+        // ---- copy the chunk's codes and V rows; rows beyond its tokens are zeros ----
+        if (codes_by_word) {
+            const int words = a.m >> 2;
+            for (int i = gtid; i < CHUNK * words; i += kPfGroupThreads) {
+                if (i / words < n) pf_cp_async4(codes_ss + i * 4, codes + c0 * a.m + (size_t)i * 4);
+                else reinterpret_cast<uint32_t *>(codes_s)[i] = 0u;
+            }
+        } else {
+            for (int i = gtid; i < CHUNK * a.m; i += kPfGroupThreads) {
+                const int tl = i / a.m, j = i - tl * a.m;
+                codes_s[tl * lay.code_pitch + j] = tl < n ? codes[(c0 + tl) * a.m + j] : 0;
+            }
+        }
+        {
+            const int tl0 = gtid / v_vec, piece = gtid - tl0 * v_vec;     // threads walk rows in steps
+            const int rows_per_pass = kPfGroupThreads / v_vec;
+            const unsigned char *src = vrow + ((size_t)(c0 + tl0) * v_vec + piece) * 16;
+            if (tl0 < rows_per_pass)
+                for (int tl = tl0; tl < CHUNK; tl += rows_per_pass, src += (size_t)rows_per_pass * v_vec * 16) {
+                    if (tl < n) pf_cp_async16(v_s + tl * lay.v_pitch + piece * 16, src);
+                    else *reinterpret_cast<uint4 *>(v_sm + tl * lay.v_pitch + piece * 16) = make_uint4(0, 0, 0, 0);
+                }
+        }
+        pf_commit();
         pf_wait_all();
-        __syncthreads();                      // chunk c0 has landed; the previous chunk's readers are done
-        if (c0 + kPfChunk < n_tok) stage(c0 + kPfChunk, buf ^ 1);
+        pf_group_barrier(grp);                // the chunk has landed for the whole half
 
-        // ---- lookup-and-sum for every (query, token) pair of the chunk, causal mask ----
-        const unsigned char *codes_s = smem + lay.codes + buf * codes_bytes;
-        for (int idx = tid; idx < TQ * kPfChunk; idx += kPfThreads) {
-            const int ql = idx % TQ, tl = idx / TQ;
+        // ---- lookup-and-sum for every (query, token) pair of the chunk, causal mask;
+        //      a thread scores one token for 4 consecutive queries: every gather is one 16-byte read ----
+        for (int idx = gtid; idx < (TQ / 4) * CHUNK; idx += kPfGroupThreads) {
+            const int qg = idx % (TQ / 4), tl = idx / (TQ / 4);
             const unsigned char *cd = codes_s + tl * lay.code_pitch;
-            float s = 0.f;
-            if ((a.m & 3) == 0) {
+            const float4 *row = reinterpret_cast<const float4 *>(lut) + qg;     // + entry * (TQ/4)
+            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+            auto add = [&](int entry) {
+                const float4 t = row[entry * (TQ / 4)];
+                s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+            };
+            if (codes_by_word) {
                 for (int j4 = 0; j4 < a.m; j4 += 4) {
                     const uint32_t wd = *reinterpret_cast<const uint32_t *>(cd + j4);
-                    s += lut[((size_t)(j4 + 0) * a.K + (wd & 0xff)) * TQ + ql];
-                    s += lut[((size_t)(j4 + 1) * a.K + ((wd >> 8) & 0xff)) * TQ + ql];
-                    s += lut[((size_t)(j4 + 2) * a.K + ((wd >> 16) & 0xff)) * TQ + ql];
-                    s += lut[((size_t)(j4 + 3) * a.K + (wd >> 24)) * TQ + ql];
+                    add((j4 + 0) * a.K + (int)(wd & 0xff));
+                    add((j4 + 1) * a.K + (int)((wd >> 8) & 0xff));
+                    add((j4 + 2) * a.K + (int)((wd >> 16) & 0xff));
+                    add((j4 + 3) * a.K + (int)(wd >> 24));
                 }
             } else {
-                for (int j = 0; j < a.m; ++j) s += lut[((size_t)j * a.K + cd[j]) * TQ + ql];
+                for (int j = 0; j < a.m; ++j) add(j * a.K + cd[j]);
             }
-            const bool valid = ql < nq && tl < n && c0 + tl <= pos0 + ql;
-            if (scores_base && valid) scores_base[(size_t)ql * a.L_max + c0 + tl] = s;
-            s_s[ql * kPfSPitch + tl] = valid ? s * a.scale_log2 : -INFINITY;
+            const float sv[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int ql = qg * 4 + k;
+                const bool valid = ql < nq && tl < n && c0 + tl <= pos0 + ql;
+                if (scores_base && valid) scores_base[(size_t)ql * a.L_max + c0 + tl] = sv[k];
+                s_s[ql * S_PITCH + tl] = valid ? sv[k] * a.scale_log2 : -INFINITY;
+            }
         }
-        __syncthreads();
+        pf_group_barrier(grp);
 
         // ---- online softmax, one warp per query row; weights as fp16 rounding + remainder ----
-        for (int r = warp; r < TQ; r += kPfWarps) {
-            const float x0 = s_s[r * kPfSPitch + lane], x1 = s_s[r * kPfSPitch + lane + 32];
-            float mx = fmaxf(x0, x1);
+        for (int r = gw; r < TQ; r += kPfGroupWarps) {
+            constexpr int PER = CHUNK / 32;                           // values per lane
+            float x[PER], p[PER];
+            float mx = -INFINITY;
+#pragma unroll
+            for (int k = 0; k < PER; ++k) {
+                x[k] = s_s[r * S_PITCH + lane + 32 * k];
+                mx = fmaxf(mx, x[k]);
+            }
             for (int d = 16; d; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
             const float m_old = m_run[r];
             const float m_new = fmaxf(m_old, mx);
-            const float p0 = ex2_approx(x0 - m_new), p1 = ex2_approx(x1 - m_new);
-            float sum = p0 + p1;
+            float sum = 0.f;
+#pragma unroll
+            for (int k = 0; k < PER; ++k) {
+                p[k] = ex2_approx(x[k] - m_new);
+                sum += p[k];
+            }
             for (int d = 16; d; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
-            const __half h0 = __float2half_rn(p0), h1 = __float2half_rn(p1);
-            p_hi[r * kPfPPitch + lane] = h0;
-            p_hi[r * kPfPPitch + lane + 32] = h1;
-            p_lo[r * kPfPPitch + lane] = __float2half_rn(p0 - __half2float(h0));
-            p_lo[r * kPfPPitch + lane + 32] = __float2half_rn(p1 - __half2float(h1));
+#pragma unroll
+            for (int k = 0; k < PER; ++k) {
+                const __half h = __float2half_rn(p[k]);
+                p_hi[r * P_PITCH + lane + 32 * k] = h;
+                p_lo[r * P_PITCH + lane + 32 * k] = __float2half_rn(p[k] - __half2float(h));
+            }
             if (lane == 0) {
                 const float al = ex2_approx(m_old - m_new);
                 alpha_s[r] = al;
@@ -249,61 +293,73 @@ __global__ void __launch_bounds__(kPfThreads, 1) attend_prefill_kernel(PrefillAr
                 m_run[r] = m_new;
             }
         }
-        __syncthreads();
+        pf_group_barrier(grp);
 
-        // ---- O += P V on the tensor cores: this warp's output columns ----
-        const unsigned v_s = smem_s + lay.v + buf * v_bytes;
+        // ---- O += P V on the tensor cores: this warp's output slices ----
         const float al0 = alpha_s[lane >> 2], al1 = alpha_s[(lane >> 2) + 8];
 #pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            const int nt = warp + t * kPfWarps;
-            if (nt < n_tiles) {
+        for (int t = 0; t < kPfMaxSlices; ++t) {
+            const int nt = gw + t * kPfGroupWarps;
+            if (nt < n_slices) {
                 acc[t][0] *= al0; acc[t][1] *= al0; acc[t][2] *= al1; acc[t][3] *= al1;
 #pragma unroll
-                for (int ks = 0; ks < kPfChunk / 16; ks += 2) {
-                    // V operands of two 16-token steps: tokens 16ks..+7 and +8..15, 8 columns
-                    uint32_t vb0[2], vb1[2];
-                    pf_ldmatrix_x2_trans(vb0, v_s + (ks * 16) * lay.v_pitch + v_lane + nt * 16);
-                    pf_ldmatrix_x2_trans(vb1, v_s + ((ks + 1) * 16) * lay.v_pitch + v_lane + nt * 16);
-                    uint32_t ph[4], pl[4];
-                    pf_ldmatrix_x4(ph, smem_s + lay.p_hi + p_lane + ks * 32);
-                    pf_ldmatrix_x4(pl, smem_s + lay.p_lo + p_lane + ks * 32);
-                    pf_mma(acc[t], ph, vb0[0], vb0[1]);
-                    pf_mma(acc[t], pl, vb0[0], vb0[1]);
-                    pf_ldmatrix_x4(ph, smem_s + lay.p_hi + p_lane + (ks + 1) * 32);
-                    pf_ldmatrix_x4(pl, smem_s + lay.p_lo + p_lane + (ks + 1) * 32);
-                    pf_mma(acc[t], ph, vb1[0], vb1[1]);
-                    pf_mma(acc[t], pl, vb1[0], vb1[1]);
+                for (int ks = 0; ks < CHUNK / 16; ++ks) {
+                    uint32_t vb[2], ph[4], pl[4];                     // V: tokens 16ks..+7 and +8..15, 8 columns
+                    pf_ldmatrix_x2_trans(vb, v_s + (ks * 16) * lay.v_pitch + v_lane + nt * 16);
+                    pf_ldmatrix_x4(ph, p_hi_s + p_lane + ks * 32);
+                    pf_ldmatrix_x4(pl, p_lo_s + p_lane + ks * 32);
+                    pf_mma(acc[t], ph, vb[0], vb[1]);
+                    pf_mma(acc[t], pl, vb[0], vb[1]);
                 }
             }
         }
-        // the next iteration's barrier separates these reads from the following writes
+        pf_group_barrier(grp);                // before the next chunk overwrites V, scores and weights
     }
 
-    // ---- normalise and store: accumulator rows lane/4 and lane/4 + 8, columns 2*(lane%4) + {0,1} ----
+    // ---- merge the two halves: M = max, l and O rescaled (accumulator rows lane/4 and lane/4 + 8) ----
+    __syncthreads();
+    float *xch = reinterpret_cast<float *>(smem + lay.v);             // the copy areas are free now
+    const float *m_a = reinterpret_cast<const float *>(smem + lay.state);
+    const float *m_b = reinterpret_cast<const float *>(smem + lay.state + lay.state_bytes);
     const int r0 = lane >> 2, r1 = r0 + 8, col = 2 * (lane & 3);
+    if (grp == 1) {
 #pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        const int nt = warp + t * kPfWarps;
-        if (nt < n_tiles) {
-            float *o = a.out + (((size_t)b * a.H_q + hq) * a.L_q + q0) * a.d_v + nt * 8 + col;
-            if (r0 < nq) {
-                const float inv = 1.f / l_run[r0];                    // token 0 is always visible: l > 0
-                *reinterpret_cast<float2 *>(o + (size_t)r0 * a.d_v) = make_float2(acc[t][0] * inv, acc[t][1] * inv);
-            }
-            if (r1 < nq) {
-                const float inv = 1.f / l_run[r1];
-                *reinterpret_cast<float2 *>(o + (size_t)r1 * a.d_v) = make_float2(acc[t][2] * inv, acc[t][3] * inv);
+        for (int t = 0; t < kPfMaxSlices; ++t)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) xch[((gw * kPfMaxSlices + t) * 4 + k) * 32 + lane] = acc[t][k];
+    }
+    __syncthreads();
+    if (grp == 0) {
+        const float M0 = fmaxf(m_a[r0], m_b[r0]), M1 = fmaxf(m_a[r1], m_b[r1]);
+        const float fa0 = ex2_approx(m_a[r0] - M0), fb0 = ex2_approx(m_b[r0] - M0);
+        const float fa1 = ex2_approx(m_a[r1] - M1), fb1 = ex2_approx(m_b[r1] - M1);
+        const float l0 = fa0 * m_a[16 + r0] + fb0 * m_b[16 + r0];     // l_run sits 16 floats after m_run
+        const float l1 = fa1 * m_a[16 + r1] + fb1 * m_b[16 + r1];
+#pragma unroll
+        for (int t = 0; t < kPfMaxSlices; ++t) {
+            const int nt = gw + t * kPfGroupWarps;
+            if (nt < n_slices) {
+                float o[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float other = xch[((gw * kPfMaxSlices + t) * 4 + k) * 32 + lane];
+                    o[k] = (k < 2 ? fa0 : fa1) * acc[t][k] + (k < 2 ? fb0 : fb1) * other;
+                }
+                float *dst = a.out + (((size_t)b * a.H_q + hq) * a.L_q + q0) * a.d_v + nt * 8 + col;
+                if (r0 < nq)                                          // token 0 is always visible: l > 0
+                    *reinterpret_cast<float2 *>(dst + (size_t)r0 * a.d_v) = make_float2(o[0] / l0, o[1] / l0);
+                if (r1 < nq)
+                    *reinterpret_cast<float2 *>(dst + (size_t)r1 * a.d_v) = make_float2(o[2] / l1, o[3] / l1);
             }
         }
     }
 }
 
-template <int TQ>
+template <int TQ, int CHUNK>
 lookat_status launch_pf(Ctx *ctx, const PrefillArgs &a)
 {
-    const PfLayout lay = pf_layout(TQ, a.d_k, a.d_v, a.m, a.K);
-    auto kern = attend_prefill_kernel<TQ>;
+    const PfLayout lay = pf_layout(TQ, CHUNK, a.d_k, a.d_v, a.m, a.K);
+    auto kern = attend_prefill_kernel<TQ, CHUNK>;
     if (lay.total > 48 * 1024 &&
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lay.total) != cudaSuccess)
         return check_launch(ctx, "prefill: shared-memory opt-in");
@@ -316,13 +372,14 @@ lookat_status launch_pf(Ctx *ctx, const PrefillArgs &a)
 
 lookat_status launch_prefill(Ctx *ctx, const PrefillArgs &a)
 {
-    if (a.d_v % 8 != 0 || a.d_v > 256 || ((uintptr_t)a.v & 15) != 0)
+    if (a.d_v % 8 != 0 || a.d_v > 256 || ((uintptr_t)a.v & 15) != 0 || ((uintptr_t)a.codes & 3) != 0)
         return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "attend_prefill: d_v must be a multiple of 8, at most 256");
-    // 16 queries per tile when their tables fit in shared memory, else 8
-    for (int tq : {16, 8}) {
-        if (pf_layout(tq, a.d_k, a.d_v, a.m, a.K).total > (size_t)ctx->max_smem_optin) continue;
-        return tq == 16 ? launch_pf<16>(ctx, a) : launch_pf<8>(ctx, a);
-    }
+    // 16 queries per tile when their tables fit in shared memory, else 8; 128-token chunks when they fit
+    const size_t cap = (size_t)ctx->max_smem_optin;
+    if (pf_layout(16, 128, a.d_k, a.d_v, a.m, a.K).total <= cap) return launch_pf<16, 128>(ctx, a);
+    if (pf_layout(16, 64, a.d_k, a.d_v, a.m, a.K).total <= cap) return launch_pf<16, 64>(ctx, a);
+    if (pf_layout(8, 128, a.d_k, a.d_v, a.m, a.K).total <= cap) return launch_pf<8, 128>(ctx, a);
+    if (pf_layout(8, 64, a.d_k, a.d_v, a.m, a.K).total <= cap) return launch_pf<8, 64>(ctx, a);
     return set_error(ctx, LOOKAT_ERR_UNSUPPORTED,
                      "attend_prefill: the tables of 8 queries (m*K*32 bytes) do not fit in shared memory");
 }
