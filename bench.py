@@ -229,6 +229,42 @@ def workload_config(w):
 
 
 # ----------------------------------------------------------------------------- GPU leg
+def time_prefill(device_index: int, steps: int = 5):
+    """Causal multi-query attention (lookat_attend_prefill) on the prefill_4k_m16 shape: batch 4, 32 heads,
+    4096 queries over 4096 cached tokens, d = 128, m = 16.  Bound: the m gathers per (query, token) pair
+    from shared memory, 4 bytes each, against 128 bytes per clock and SM."""
+    import torch
+
+    from paper_2601_10155_b200.binding import Lookat
+    w = synth.WORKLOADS["prefill_4k_m16"]
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K, device=device_index)
+    keys = dev(synth.make_keys(w))
+    v = dev(synth.make_values(w))
+    q = dev(synth.make_prefill_queries(w, w.L))
+    books = lk.lookat_fit_codebooks(keys, w.fit_iters, seed=w.seed)          # per head, on its 16,384 keys
+    codes = lk.lookat_encode_keys(keys, books)
+    out = torch.empty((w.B, w.n_q_heads, w.L, w.d_v), dtype=torch.float32, device="cuda")
+    for _ in range(2):
+        lk.lookat_attend_prefill(q, books, codes, v, out=out)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        lk.lookat_attend_prefill(q, books, codes, v, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    pairs = w.B * w.n_q_heads * w.L * (w.L + 1) // 2
+    props = torch.cuda.get_device_properties(device_index)
+    smem_peak = props.multi_processor_count * 128 * 1.965e9 / 1e9          # GB/s at the maximum SM clock
+    achieved = pairs * w.m * 4 / (ms * 1e-3) / 1e9
+    return {"workload": w.name, "ms": ms, "pairs_per_s": pairs / (ms * 1e-3), "steps": steps,
+            "roofline": {"bound": "smem", "achieved": achieved, "peak": smem_peak, "unit": "GB/s",
+                         "frac": achieved / smem_peak,
+                         "note": "gather bytes (m x 4 B per pair) over 128 B/clk/SM x SMs x 1965 MHz"}}
+
+
 def run_lookat(args, w):
     import torch
     import torch.distributed as dist
@@ -366,6 +402,13 @@ def run_lookat(args, w):
         }
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = time_oracle(w)
+        if world == 1 and args.prefill:
+            del keys, v, codes, code_sets, v_sets
+            torch.cuda.empty_cache()
+            try:
+                line["prefill"] = time_prefill(local_rank)
+            except Exception as exc:                      # the decode line stands on its own
+                line["prefill"] = {"error": str(exc)[:200]}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
@@ -381,6 +424,8 @@ def main():
     ap.add_argument("--workload", default="gqa_32k_m8", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--splits", type=int, default=0, help="sequence chunks per row (0: library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", dest="prefill", action="store_false",
+                    help="skip the extra timing of the causal multi-query kernel")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size (smaller cases for profiler captures)")
     args = ap.parse_args()
