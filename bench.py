@@ -229,7 +229,7 @@ def workload_config(w):
 
 
 # ----------------------------------------------------------------------------- GPU leg
-def time_prefill(device_index: int, steps: int = 5):
+def time_prefill(device_index: int, steps: int = 5, batch: int = 0, heads: int = 0):
     """Causal multi-query attention (lookat_attend_prefill) on the prefill_4k_m16 shape: batch 4, 32 heads,
     4096 queries over 4096 cached tokens, d = 128, m = 16.  Bound: the m gathers per (query, token) pair
     from shared memory, 4 bytes each, against 128 bytes per clock and SM."""
@@ -237,6 +237,10 @@ def time_prefill(device_index: int, steps: int = 5):
 
     from paper_2601_10155_b200.binding import Lookat
     w = synth.WORKLOADS["prefill_4k_m16"]
+    if batch > 0 or heads > 0:                             # smaller cases for profiler captures
+        w = synth.Workload(**{**w.__dict__, "B": batch or w.B, "n_q_heads": heads or w.n_q_heads,
+                              "n_kv_heads": heads or w.n_kv_heads,
+                              "name": f"{w.name}_b{batch or w.B}_h{heads or w.n_q_heads}"})
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
     lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K, device=device_index)
     keys = dev(synth.make_keys(w))
@@ -426,13 +430,20 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", dest="prefill", action="store_false",
                     help="skip the extra timing of the causal multi-query kernel")
+    ap.add_argument("--only-prefill", action="store_true",
+                    help="time only the causal multi-query kernel (prints its object alone)")
+    ap.add_argument("--prefill-batch", type=int, default=0, help="smaller prefill case: batch rows")
+    ap.add_argument("--prefill-heads", type=int, default=0, help="smaller prefill case: heads")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size (smaller cases for profiler captures)")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.batch > 0:
         w = synth.Workload(**{**w.__dict__, "B": args.batch, "name": f"{w.name}_b{args.batch}"})
-    if args.impl == "reference":
+    if args.only_prefill:
+        print(json.dumps(time_prefill(int(os.environ.get("LOCAL_RANK", "0")), steps=max(1, min(args.steps, 5)),
+                                      batch=args.prefill_batch, heads=args.prefill_heads)), flush=True)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_lookat(args, w)
