@@ -39,8 +39,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per (token, KV head) pair of one
 # attend_stream_kernel launch, from an ncu capture of the batch-4 case of gqa_32k_m8
-# (284,259,328 bytes over 1,048,576 pairs; traffic grows in proportion to the pairs).
-ATTEND_DRAM_BYTES_PER_PAIR = {"gqa_32k_m8": 284259328 / 1048576}
+# (283,105,792 bytes over 1,048,576 pairs; traffic grows in proportion to the pairs).
+ATTEND_DRAM_BYTES_PER_PAIR = {"gqa_32k_m8": 283105792 / 1048576}
 
 
 def measured_peak_gbs():
