@@ -127,6 +127,9 @@ struct EncodeArgs {
     int distortion_stride;
 };
 lookat_status launch_encode(Ctx *ctx, const EncodeArgs &a);
+// bulk encoding with the key-by-centroid products on the tensor cores (d_sub 8, 16, 32)
+bool encode_mma_covers(const Ctx *ctx, const EncodeArgs &a);
+lookat_status launch_encode_mma(Ctx *ctx, const EncodeArgs &a);
 
 lookat_status launch_fit_init(Ctx *ctx, const __half *keys, int B, long long n, uint64_t seed,
                               const float *init, float *codebooks);

@@ -211,6 +211,7 @@ lookat_status launch_encode(Ctx *ctx, const EncodeArgs &a)
             a, c.n_kv_heads, c.d_k, c.m, c.K, n_tasks);
         return check_launch(ctx, "encode_warp_kernel");
     }
+    if (encode_mma_covers(ctx, a)) return launch_encode_mma(ctx, a);
     switch (d_sub) {
         case 4: return launch_tile<4, 4>(ctx, a);
         case 8: return launch_tile<8, 4>(ctx, a);
