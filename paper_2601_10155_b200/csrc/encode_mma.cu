@@ -1,17 +1,21 @@
 // Bulk nearest-centroid encoding on the tensor cores (Section 3.4 "Encoding", and the assignment
 // step of "Prototype Learning").  The batched key-by-centroid inner products are the dense
 // contraction of this step:
-//     || x - c ||^2 = ||x||^2 + ( ||c||^2 - 2 x.c ),     argmin_c of the bracket.
-// x (fp16) is exact as an MMA operand; every fp32 centroid is split into two fp16 planes (its
-// rounding and what the rounding left over), so x.c is carried to ~22 bits with fp32 accumulation:
-// two mma.sync.m16n8k16 per 16 keys x 8 centroids.  The winner of this fast search is accepted only
-// when its margin over the runner-up exceeds a bound on the search's own error; every other key
-// (near ties, duplicate centroids) is decided again by the exact rule of encode_warp.cuh (fp32
-// difference form, fp64 inside its band), so the codes equal the fp64 argmin with lowest index on ties.
+//     || x - c ||^2 = ||x||^2 + s(c),     s(c) = ||c||^2 - 2 x.c,     argmin_c s(c).
+// x (fp16) is exact as an MMA operand; -2c (fp32) is split into two fp16 planes (its rounding and
+// what the rounding left over), and ||c||^2 enters as the accumulator's initial value, so one chain
+// of mma.sync.m16n8k16 per 16 keys x 8 centroids leaves s(c) itself in the accumulators.  The low 8
+// bits of every score are then replaced by the centroid's index, which turns the search for the two
+// smallest scores into plain float min/max.  The winner of this fast search is accepted only when
+// its margin over the runner-up exceeds a bound on the search's own error; every other key (near
+// ties, duplicate centroids, non-finite input) is decided again by the exact rule of encode_warp.cuh
+// (fp32 difference form, fp64 inside its band), so the codes equal the fp64 argmin with lowest index
+// on ties.
 //
 // One CTA: one (batch row, KV head), one subspace, up to 1024 keys; its 8 warps take 32 keys at a time
-// (two 16-row operand tiles share each centroid fragment).  The centroid planes sit in shared memory,
-// centroid-major with a row pitch chosen so that the fragment reads are bank-conflict free.
+// (two 16-row operand tiles share each centroid fragment).  Shared memory holds, per centroid and
+// lane-in-group t, the words that lane needs as one 16-byte (d_sub 8: 8-byte) fragment, and per
+// 8-centroid tile the four initial accumulator values of each t.
 #include "common.cuh"
 #include "encode_warp.cuh"
 
@@ -24,20 +28,38 @@ constexpr int kMmaThreads = kMmaWarps * 32;
 constexpr int kMmaKeysPerWarpStep = 32;
 constexpr int kMmaStepsPerCta = 4;
 constexpr int kMmaKeysPerCta = kMmaWarps * kMmaKeysPerWarpStep * kMmaStepsPerCta;   // 1024
-// Margin below which the fast winner is not trusted: kMmaBand * ||x|| * (||x|| + ||c_best||).
-// A fast score errs by at most e(c) = 2 * 64 * 2^-23 * ||x|| ||c|| < 1.6e-5 ||x|| ||c|| (up to 64 exact
-// products accumulated in fp32, plus the 2^-22 split error).  A centroid with ||c|| > 2||x|| + ||c_best||
-// is farther than the winner whatever its error; for all others e(c) + e(c_best) stays below
-// 1.6e-5 * ||x|| * (2||x|| + 2||c_best||) < the margin required here.
-constexpr float kMmaBand = 6.0e-5f;
+
+// Error of a fast score, for the winner w and for the true nearest centroid c* (both have
+// ||c|| <= R = ||x|| + dist(x, w), and |s| <= Q = max(||x||^2, dist(x, w)^2)):
+//   ||c||^2 summed in fp32                      <= 32 * 2^-24 ||c||^2          <= 2^-19 R^2
+//   what the two fp16 planes of -2c leave out   <= 2^-22 ||x|| ||c||           <= 2^-22 R^2
+//                                                  + 2^-25 per term (fp16 subnormal floor)
+//   up to 4 chained MMAs, each taken to err by 8 units in the last place of the largest partial sum
+//                                               <= 2^-18 (||c||^2 + 2 ||x|| ||c||) <= 3 * 2^-18 R^2
+//   the 8 bits given to the index               <= 2^-15 |s|                   <= 2^-15 Q
+// in total < 1.4e-5 R^2 + 3.1e-5 Q + 1e-6 ||x||.  The winner is accepted when its margin exceeds twice
+// that, with a tenth added because R and Q are themselves computed from the fast score.
+constexpr float kMmaErrR2 = 3.1e-5f;
+constexpr float kMmaErrQ = 6.9e-5f;
+constexpr float kMmaErrX = 2.2e-6f;
+constexpr float kMmaMaxCentroid = 30000.f;   // |-2c| must stay inside fp16 range
 
 template <int D_SUB>
 struct MmaShape {
     static constexpr int kSteps = D_SUB >= 16 ? D_SUB / 16 : 1;            // k-steps of 16 dims
-    static constexpr int kWords = D_SUB / 2;                               // 32-bit words per centroid row
-    // row pitch in words: 8 rows x 4 lanes must land in 32 different banks
-    static constexpr int kPitch = D_SUB == 8 ? 4 : (D_SUB == 16 ? 12 : 20);
+    static constexpr int kFragWords = D_SUB >= 16 ? 4 : 2;                 // words per (centroid, t) fragment
 };
+
+// D = A.B + C, C given as its own four registers
+__device__ __forceinline__ void enc_mma_init(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1,
+                                             const float4 &c)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%10,%11,%12,%13};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(c.x), "f"(c.y), "f"(c.z), "f"(c.w));
+}
 
 __device__ __forceinline__ void enc_mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
@@ -46,6 +68,19 @@ __device__ __forceinline__ void enc_mma(float (&c)[4], const uint32_t (&a)[4], u
         "{%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ float min3(float a, float b, float c)
+{
+    float r;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// score with its low 8 mantissa bits replaced by the centroid index
+__device__ __forceinline__ float tag(float s, int c)
+{
+    return __uint_as_float((__float_as_uint(s) & 0xffffff00u) | (uint32_t)c);
 }
 
 // The exact rule for one (key, subspace), by the whole warp; out of line (it is the rare path).
@@ -58,18 +93,6 @@ __device__ __noinline__ int exact_code_warp(const __half *x, const float *book, 
     return code;
 }
 
-// smaller distance wins, then smaller index; the loser's best is a runner-up
-__device__ __forceinline__ void merge_best(Best &r, float ob, float os, int oi)
-{
-    const bool other_wins = ob < r.best || (ob == r.best && oi < r.idx);
-    const float loser = other_wins ? r.best : ob;
-    r.second = fminf(fminf(r.second, os), loser);
-    if (other_wins) {
-        r.best = ob;
-        r.idx = oi;
-    }
-}
-
 template <int D_SUB>
 __global__ void __launch_bounds__(kMmaThreads)
 encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
@@ -77,9 +100,8 @@ encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
     using S = MmaShape<D_SUB>;
     extern __shared__ __align__(16) uint32_t sm_words[];
     const int n_cols = (K + 7) & ~7;                                   // centroid columns, whole n-tiles
-    uint32_t *c_hi = sm_words;                                         // [n_cols][kPitch]
-    uint32_t *c_lo = c_hi + n_cols * S::kPitch;
-    float *c_norm = reinterpret_cast<float *>(c_lo + n_cols * S::kPitch);   // [n_cols], +inf beyond K
+    uint32_t *frag = sm_words;                                         // [kSteps][n_cols][4 t][kFragWords]
+    float *cn4 = reinterpret_cast<float *>(frag + S::kSteps * n_cols * 4 * S::kFragWords);   // [n_cols/8][4 t][4]
     __shared__ int s_force_exact;
     __shared__ double s_red[kMmaWarps];
 
@@ -89,26 +111,44 @@ encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
     const int problem = h * m + j;
     const float *book = a.codebooks + (size_t)problem * K * D_SUB;
 
-    // ---- centroid planes and norms ----
+    // ---- planes of -2c in fragment order, and ||c||^2 as initial accumulators ----
     if (tid == 0) s_force_exact = 0;
     __syncthreads();
     for (int c = tid; c < n_cols; c += kMmaThreads) {
         float norm = 0.f;
         bool bad = false;
-        for (int w = 0; w < S::kWords; ++w) {
+        for (int w = 0; w < D_SUB / 2; ++w) {
             float v0 = 0.f, v1 = 0.f;
             if (c < K) {
                 v0 = book[(size_t)c * D_SUB + 2 * w];
                 v1 = book[(size_t)c * D_SUB + 2 * w + 1];
             }
             norm = fmaf(v0, v0, fmaf(v1, v1, norm));
+            bad = bad || !(fabsf(v0) < kMmaMaxCentroid) || !(fabsf(v1) < kMmaMaxCentroid);
+            v0 *= -2.f;
+            v1 *= -2.f;
             const __half h0 = __float2half_rn(v0), h1 = __float2half_rn(v1);
             const __half l0 = __float2half_rn(v0 - __half2float(h0)), l1 = __float2half_rn(v1 - __half2float(h1));
-            bad = bad || !(fabsf(v0) < 60000.f) || !(fabsf(v1) < 60000.f);
-            c_hi[c * S::kPitch + w] = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
-            c_lo[c * S::kPitch + w] = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
+            const uint32_t hi = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
+            const uint32_t lo = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
+            if (D_SUB >= 16) {
+                // lane t of a group takes words t and t+4 of each k-step: {hi, hi+4, lo, lo+4}
+                const int ks = w >> 3, r = w & 7;
+                uint32_t *f = frag + ((size_t)(ks * n_cols + c) * 4 + (r & 3)) * 4 + (r >> 2);
+                f[0] = hi;
+                f[2] = lo;
+            } else {
+                // d_sub 8: one k-step holds both planes, {hi, lo} of word t
+                uint32_t *f = frag + ((size_t)c * 4 + w) * 2;
+                f[0] = hi;
+                f[1] = lo;
+            }
         }
-        c_norm[c] = c < K ? norm : INFINITY;
+        // columns beyond K keep a large finite score (an infinity would turn into a NaN when tagged)
+        const float cn = c < K ? norm : 3.0e38f;
+        float *q = cn4 + ((c >> 3) * 4 + ((c & 7) >> 1)) * 4 + (c & 1);
+        q[0] = cn;
+        q[2] = cn;
         if (bad) s_force_exact = 1;                       // outside fp16 range: every key takes the exact path
     }
     __syncthreads();
@@ -134,74 +174,82 @@ encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
 #pragma unroll
                 for (int ks = 0; ks < S::kSteps; ++ks) {
                     const uint32_t w0 = *reinterpret_cast<const uint32_t *>(rowp[u][rr] + ks * 16 + 2 * t);
-                    uint32_t w1 = 0u;
+                    // d_sub 8: the second half of the k-step meets the remainder plane, so it repeats x
+                    uint32_t w1 = w0;
                     if (D_SUB >= 16) w1 = *reinterpret_cast<const uint32_t *>(rowp[u][rr] + ks * 16 + 2 * t + 8);
                     xa[u][ks][rr] = w0;                     // a0 (row g) / a1 (row g+8)
-                    xa[u][ks][2 + rr] = w1;                 // a2 / a3: dims +8
+                    xa[u][ks][2 + rr] = w1;                 // a2 / a3
                     const float2 f0 = __half22float2(*reinterpret_cast<const __half2 *>(&w0));
-                    const float2 f1 = __half22float2(*reinterpret_cast<const __half2 *>(&w1));
-                    nn += f0.x * f0.x + f0.y * f0.y + f1.x * f1.x + f1.y * f1.y;
+                    nn += f0.x * f0.x + f0.y * f0.y;
+                    if (D_SUB >= 16) {
+                        const float2 f1 = __half22float2(*reinterpret_cast<const __half2 *>(&w1));
+                        nn += f1.x * f1.x + f1.y * f1.y;
+                    }
                 }
                 nn += __shfl_xor_sync(0xffffffffu, nn, 1);
                 nn += __shfl_xor_sync(0xffffffffu, nn, 2);
                 xnorm[u][rr] = nn;
             }
 
-        Best best[2][2];
+        float best[2][2], second[2][2];                     // tagged scores
 #pragma unroll
         for (int u = 0; u < 2; ++u)
 #pragma unroll
-            for (int rr = 0; rr < 2; ++rr) {
-                best[u][rr].best = INFINITY;
-                best[u][rr].second = INFINITY;
-                best[u][rr].idx = 0x7fffffff;
-            }
+            for (int rr = 0; rr < 2; ++rr) best[u][rr] = second[u][rr] = INFINITY;
 
         // ---- all centroids, 8 at a time ----
         for (int nt = 0; nt < n_cols / 8; ++nt) {
             float acc[2][4];
+            const float4 cq = *reinterpret_cast<const float4 *>(cn4 + (nt * 4 + t) * 4);
+            if (D_SUB >= 16) {
 #pragma unroll
-            for (int u = 0; u < 2; ++u) acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
-            const uint32_t *bh_row = c_hi + (nt * 8 + g) * S::kPitch + t;
-            const uint32_t *bl_row = c_lo + (nt * 8 + g) * S::kPitch + t;
+                for (int ks = 0; ks < S::kSteps; ++ks) {
+                    const uint4 f = *reinterpret_cast<const uint4 *>(frag + ((size_t)(ks * n_cols + nt * 8 + g) * 4 + t) * 4);
 #pragma unroll
-            for (int ks = 0; ks < S::kSteps; ++ks) {
-                const uint32_t h0 = bh_row[ks * 8], l0 = bl_row[ks * 8];
-                const uint32_t h1 = D_SUB >= 16 ? bh_row[ks * 8 + 4] : 0u, l1 = D_SUB >= 16 ? bl_row[ks * 8 + 4] : 0u;
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    enc_mma(acc[u], xa[u][ks], h0, h1);
-                    enc_mma(acc[u], xa[u][ks], l0, l1);
+                    for (int u = 0; u < 2; ++u) {
+                        if (ks == 0) enc_mma_init(acc[u], xa[u][0], f.x, f.y, cq);
+                        else enc_mma(acc[u], xa[u][ks], f.x, f.y);
+                        enc_mma(acc[u], xa[u][ks], f.z, f.w);
+                    }
                 }
+            } else {
+                const uint2 f = *reinterpret_cast<const uint2 *>(frag + ((size_t)(nt * 8 + g) * 4 + t) * 2);
+#pragma unroll
+                for (int u = 0; u < 2; ++u) enc_mma_init(acc[u], xa[u][0], f.x, f.y, cq);
             }
-            const float2 cn = *reinterpret_cast<const float2 *>(c_norm + nt * 8 + 2 * t);
             const int c0 = nt * 8 + 2 * t;
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                consider(best[u][0], fmaf(-2.f, acc[u][0], cn.x), c0);
-                consider(best[u][0], fmaf(-2.f, acc[u][1], cn.y), c0 + 1);
-                consider(best[u][1], fmaf(-2.f, acc[u][2], cn.x), c0);
-                consider(best[u][1], fmaf(-2.f, acc[u][3], cn.y), c0 + 1);
-            }
+            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int rr = 0; rr < 2; ++rr) {
+                    const float d0 = tag(acc[u][2 * rr], c0), d1 = tag(acc[u][2 * rr + 1], c0 + 1);
+                    const float lo = fminf(d0, d1), hi = fmaxf(d0, d1);
+                    second[u][rr] = min3(second[u][rr], hi, fmaxf(best[u][rr], lo));
+                    best[u][rr] = fminf(best[u][rr], lo);
+                }
         }
 
         // ---- the 4 lanes of a row merge; rows whose margin is inside the error bound are redone exactly ----
+        int code[2][2];
         unsigned redo[2][2];
 #pragma unroll
         for (int u = 0; u < 2; ++u)
 #pragma unroll
             for (int rr = 0; rr < 2; ++rr) {
-                Best &r = best[u][rr];
+                float b = best[u][rr], s = second[u][rr];
 #pragma unroll
-                for (int s = 1; s <= 2; s <<= 1) {
-                    const float ob = __shfl_xor_sync(0xffffffffu, r.best, s);
-                    const float os = __shfl_xor_sync(0xffffffffu, r.second, s);
-                    const int oi = __shfl_xor_sync(0xffffffffu, r.idx, s);
-                    merge_best(r, ob, os, oi);
+                for (int sh = 1; sh <= 2; sh <<= 1) {
+                    const float ob = __shfl_xor_sync(0xffffffffu, b, sh);
+                    const float os = __shfl_xor_sync(0xffffffffu, s, sh);
+                    s = min3(s, os, fmaxf(b, ob));
+                    b = fminf(b, ob);
                 }
-                const float xn = sqrtf(xnorm[u][rr]);
-                const float cb = sqrtf(c_norm[r.idx < n_cols ? r.idx : 0]);
-                const bool unsure = force_exact || !(r.second - r.best > kMmaBand * xn * (xn + cb));
+                code[u][rr] = (int)(__float_as_uint(b) & 0xffu);
+                const float x2 = xnorm[u][rr];
+                const float dw2 = fmaxf(b + x2, 0.f);       // squared distance to the winner
+                const float r = sqrtf(x2) + sqrtf(dw2);
+                const float err = kMmaErrR2 * r * r + kMmaErrQ * fmaxf(x2, dw2) + kMmaErrX * sqrtf(x2);
+                const bool unsure = force_exact || !(s - b > err);      // also true when anything is not a number
                 redo[u][rr] = __ballot_sync(0xffffffffu, unsure && t == 0);
             }
         int tie_count = 0;
@@ -216,10 +264,10 @@ encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
                     const unsigned long long p =
                         __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)rowp[u][rr], src);
                     int tie;
-                    const int code = exact_code_warp(reinterpret_cast<const __half *>((uintptr_t)p), book, K, D_SUB,
-                                                     lane, &tie);
+                    const int exact = exact_code_warp(reinterpret_cast<const __half *>((uintptr_t)p), book, K, D_SUB,
+                                                      lane, &tie);
                     if (lane == src) {
-                        best[u][rr].idx = code;
+                        code[u][rr] = exact;
                         tie_count += tie;
                     }
                 }
@@ -233,16 +281,16 @@ encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
                 for (int rr = 0; rr < 2; ++rr) {
                     const long long key = key0 + u * 16 + g + rr * 8;
                     if (key >= a.n) continue;
-                    const int code = best[u][rr].idx;
-                    a.codes[((size_t)bh * a.L_max + a.pos + key) * m + j] = (uint8_t)code;
+                    const int cd = code[u][rr];
+                    a.codes[((size_t)bh * a.L_max + a.pos + key) * m + j] = (uint8_t)cd;
                     if (a.sums) {
                         const __half *x = rowp[u][rr];
-                        unsigned long long *s = a.sums + ((size_t)problem * K + code) * D_SUB;
+                        unsigned long long *s = a.sums + ((size_t)problem * K + cd) * D_SUB;
 #pragma unroll
                         for (int i = 0; i < D_SUB; ++i)
                             atomicAdd(s + i, (unsigned long long)half_to_fixed24(x[i]));
-                        atomicAdd(a.cnt + (size_t)problem * K + code, 1ull);
-                        if (a.distortion) dsum += dist_fp64(x, book + (size_t)code * D_SUB, D_SUB);
+                        atomicAdd(a.cnt + (size_t)problem * K + cd, 1ull);
+                        if (a.distortion) dsum += dist_fp64(x, book + (size_t)cd * D_SUB, D_SUB);
                     }
                 }
             if (tie_count && a.near_ties) atomicAdd(a.near_ties, (unsigned long long)tie_count);
@@ -266,7 +314,7 @@ lookat_status launch_mma(Ctx *ctx, const EncodeArgs &a)
 {
     const lookat_config &c = ctx->cfg;
     const int n_cols = (c.K + 7) & ~7;
-    const size_t smem = (size_t)n_cols * (2 * MmaShape<D_SUB>::kPitch + 1) * 4;
+    const size_t smem = (size_t)n_cols * (MmaShape<D_SUB>::kSteps * 4 * MmaShape<D_SUB>::kFragWords + 2) * 4;
     auto kern = encode_mma_kernel<D_SUB>;
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
