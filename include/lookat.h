@@ -228,6 +228,25 @@ lookat_status lookat_decode_step_host(lookat_ctx *ctx, const void *q_host, const
                                       uint8_t *codes, void *v, int64_t L_max, int64_t pos,
                                       int32_t n_splits, float *out_host);
 
+/*
+ * Which of its two kernels lookat_attend_prefill uses.  Both compute Algorithm
+ * 1 for every query; they differ in how the score of Section 3.4 is formed:
+ *   LOOKAT_PREFILL_TABLES       per-query tables built on chip, then m lookups
+ *                               per (query, token) pair (any shape);
+ *   LOOKAT_PREFILL_CONTRACTION  the centroids named by a chunk of codes are
+ *                               gathered once per 128 queries and the scores
+ *                               taken as q . (C_1[c_1], ..., C_m[c_m]) on the
+ *                               tensor cores (d_k and d_v in {64, 128}, d_sub a
+ *                               multiple of 4);
+ *   LOOKAT_PREFILL_AUTO         (default) contraction where it applies and
+ *                               L_q >= 32, tables otherwise.
+ * Asking for the contraction form on a shape it does not cover makes
+ * lookat_attend_prefill return LOOKAT_ERR_UNSUPPORTED.  Returns
+ * LOOKAT_ERR_INVALID_ARG for an unknown value.
+ */
+enum { LOOKAT_PREFILL_AUTO = 0, LOOKAT_PREFILL_TABLES = 1, LOOKAT_PREFILL_CONTRACTION = 2 };
+lookat_status lookat_set_prefill_form(lookat_ctx *ctx, int32_t form);
+
 /* Number of kernels this context has launched since it was created. */
 uint64_t lookat_kernel_launches(const lookat_ctx *ctx);
 

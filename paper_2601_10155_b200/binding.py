@@ -20,7 +20,7 @@ EXPORTS = [
     "lookat_create", "lookat_destroy", "lookat_last_error", "lookat_fit_codebooks",
     "lookat_encode_keys", "lookat_build_lut", "lookat_attend", "lookat_attend_static",
     "lookat_attend_prefill", "lookat_decode_step", "lookat_decode_step_host",
-    "lookat_kernel_launches", "lookat_set_timing", "lookat_attend_kernel_ms",
+    "lookat_kernel_launches", "lookat_set_prefill_form", "lookat_set_timing", "lookat_attend_kernel_ms",
 ]
 
 STATUS = {0: "LOOKAT_OK", 1: "LOOKAT_ERR_INVALID_ARG", 2: "LOOKAT_ERR_UNSUPPORTED",
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
     lib.lookat_decode_step_host.restype = ctypes.c_int
     lib.lookat_kernel_launches.argtypes = [vp]
     lib.lookat_kernel_launches.restype = ctypes.c_uint64
+    lib.lookat_set_prefill_form.argtypes = [vp, i32]
+    lib.lookat_set_prefill_form.restype = i32
     lib.lookat_set_timing.argtypes = [vp, i32]
     lib.lookat_set_timing.restype = None
     lib.lookat_attend_kernel_ms.argtypes = [vp]
@@ -278,6 +280,11 @@ class Lookat:
 
     def lookat_kernel_launches(self) -> int:
         return int(self._lib.lookat_kernel_launches(self._h))
+
+    def lookat_set_prefill_form(self, form):
+        """form: 'auto', 'tables' or 'contraction' (or the header's integer values)."""
+        code = {"auto": 0, "tables": 1, "contraction": 2}.get(form, form)
+        self._check(self._lib.lookat_set_prefill_form(self._h, int(code)))
 
     def lookat_set_timing(self, enabled: bool):
         self._lib.lookat_set_timing(self._h, 1 if enabled else 0)

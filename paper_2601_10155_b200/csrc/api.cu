@@ -244,6 +244,7 @@ lookat_status lookat_create(const lookat_config *cfg, int device, void *cuda_str
     }
     ctx->sm_count = prop.multiProcessorCount;
     ctx->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    ctx->prefill_form = LOOKAT_PREFILL_AUTO;
     for (int i = 0; i < kTimingSlots; ++i) {
         if (cudaEventCreate(&ctx->ev0[i]) != cudaSuccess || cudaEventCreate(&ctx->ev1[i]) != cudaSuccess) {
             cudaGetLastError();
@@ -281,6 +282,16 @@ const char *lookat_last_error(const lookat_ctx *handle)
 uint64_t lookat_kernel_launches(const lookat_ctx *handle)
 {
     return handle ? reinterpret_cast<const Ctx *>(handle)->launches : 0;
+}
+
+lookat_status lookat_set_prefill_form(lookat_ctx *handle, int32_t form)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    if (form != LOOKAT_PREFILL_AUTO && form != LOOKAT_PREFILL_TABLES && form != LOOKAT_PREFILL_CONTRACTION)
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "set_prefill_form: unknown form %d", (int)form);
+    ctx->prefill_form = form;
+    return LOOKAT_OK;
 }
 
 void lookat_set_timing(lookat_ctx *handle, int32_t enabled)

@@ -19,6 +19,7 @@ struct Ctx {
     cudaStream_t stream;
     int sm_count;
     int max_smem_optin;
+    int prefill_form;          // LOOKAT_PREFILL_*
     float scale;           // resolved softmax scale
     char err[512];
     uint64_t launches;
@@ -110,6 +111,9 @@ struct PrefillArgs {
     float scale_log2;
 };
 lookat_status launch_prefill(Ctx *ctx, const PrefillArgs &a);
+// contraction form (prefill_mma.cu): centroids gathered per chunk, scores on the tensor cores
+bool prefill_mma_covers(const Ctx *ctx, const PrefillArgs &a);
+lookat_status launch_prefill_mma(Ctx *ctx, const PrefillArgs &a);
 
 lookat_status launch_build_lut(Ctx *ctx, const __half *q, int B, const float *codebooks, float *lut);
 

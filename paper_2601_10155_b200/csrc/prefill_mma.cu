@@ -1,0 +1,353 @@
+// Multi-query causal attention over the compressed keys, contraction form (Algorithm 1 applied to a
+// tile of queries).  The score of Section 3.4,
+//     s[q][t] = sum_j LUT_j[code[t][j]],   LUT_j[c] = q^(j) . C_j[c],
+// is the inner product of q with the key rebuilt from its codes, k^[t] = (C_1[code[t][1]], ...,
+// C_m[code[t][m]]).  A table pays when one query meets many keys; in prefill many queries meet each
+// key, so this kernel gathers the centroids of a chunk of tokens ONCE per CTA into shared memory (the
+// codes stay the only stored form of the keys; nothing is written back to HBM) and lets 128 queries
+// take their scores from it on the tensor cores: S = Q . K^^T, online softmax, O += P . V, all with
+// mma.sync.m16n8k16 and fp32 accumulation.  q (fp16) is an exact operand; every fp32 centroid is
+// split into two fp16 planes (rounding + remainder), which carries s to ~2^-22 relative.
+//
+// One CTA: one (batch row, query head), 128 consecutive queries (8 warps x 16 rows), 64-token chunks up
+// to the causal limit of the tile.  Per chunk: the next chunk's V rows arrive by cp.async and its
+// centroid rows are gathered (global loads that hit L1/L2; the codebook of a head is <= 128 KB) while
+// this chunk's MMAs run; they are split and stored between the phases; one barrier per chunk.
+#include "common.cuh"
+
+namespace lookat {
+
+namespace {
+
+constexpr int kPmWarps = 8;
+constexpr int kPmThreads = kPmWarps * 32;
+constexpr int kPmRows = kPmWarps * 16;        // queries per CTA
+constexpr int kPmChunk = 64;                  // tokens per chunk
+
+__device__ __forceinline__ void pm_cp_async16(unsigned dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void pm_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void pm_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+__device__ __forceinline__ void pm_ldmatrix_x4(uint32_t (&r)[4], unsigned src)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(src));
+}
+__device__ __forceinline__ void pm_ldmatrix_x4_trans(uint32_t (&r)[4], unsigned src)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(src));
+}
+__device__ __forceinline__ void pm_mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pm_pack(float lo, float hi)
+{
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+
+// Rounding and remainder planes of 8 consecutive fp32 values, as two 16-byte rows.
+__device__ __forceinline__ void pm_split8(const float4 &x, const float4 &y, uint4 &hi, uint4 &lo)
+{
+    const float v[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
+    uint32_t h[4], l[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __half2 hh = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
+        const float2 back = __half22float2(hh);
+        const __half2 ll = __floats2half2_rn(v[2 * i] - back.x, v[2 * i + 1] - back.y);
+        h[i] = *reinterpret_cast<const uint32_t *>(&hh);
+        l[i] = *reinterpret_cast<const uint32_t *>(&ll);
+    }
+    hi = make_uint4(h[0], h[1], h[2], h[3]);
+    lo = make_uint4(l[0], l[1], l[2], l[3]);
+}
+
+template <int D_K, int D_V>
+struct PmLayout {
+    static constexpr int kPitchK = D_K * 2 + 16;                       // bytes per rebuilt key row (one plane)
+    static constexpr int kPitchV = D_V * 2 + 16;
+    static constexpr int kPlane = kPmChunk * kPitchK;
+    static constexpr int kVTile = kPmChunk * kPitchV;
+    static constexpr int kStage = 2 * kPlane + kVTile;                 // hi plane, lo plane, V
+    static constexpr int kBytes = 2 * kStage;
+    static constexpr int kGroups = D_K / 8;                            // 8-dim groups per key row
+    static constexpr int kPieces = kPmChunk * kGroups / kPmThreads;    // groups gathered per thread per chunk
+    static_assert(kPmChunk * kGroups % kPmThreads == 0, "whole pieces per thread");
+};
+
+template <int D_K, int D_V, bool SCORES, bool SPLIT_P>
+__global__ void __launch_bounds__(kPmThreads, 1)
+attend_prefill_mma_kernel(PrefillArgs a)
+{
+    using Lay = PmLayout<D_K, D_V>;
+    extern __shared__ __align__(16) unsigned char pm_smem[];
+    const unsigned smem0 = (unsigned)__cvta_generic_to_shared(pm_smem);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int n_tiles = (int)((a.L_q + kPmRows - 1) / kPmRows);
+    const int tile = n_tiles - 1 - (int)blockIdx.x;            // longest tiles first
+    const int hq = blockIdx.y, b = blockIdx.z, h = hq / a.g;
+    const int d_sub = D_K / a.m;
+
+    const long long row0 = (long long)tile * kPmRows;
+    const long long t_end = a.q_pos0 + (row0 + kPmRows < a.L_q ? row0 + kPmRows : a.L_q);   // tokens the tile sees
+    const int n_chunks = (int)((t_end + kPmChunk - 1) / kPmChunk);
+
+    const float *book = a.codebooks + (size_t)h * a.m * a.K * d_sub;
+    const uint8_t *codes = a.codes + (size_t)(b * a.H_kv + h) * a.L_max * a.m;
+    const __half *vsrc = a.v + (size_t)(b * a.H_kv + h) * a.L_max * D_V;
+
+    // ---- this thread's two query rows (clamped copies beyond L_q are computed and dropped) ----
+    long long row[2], vis_end[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        row[i] = row0 + warp * 16 + g + 8 * i;
+        const long long rc = row[i] < a.L_q ? row[i] : a.L_q - 1;
+        vis_end[i] = a.q_pos0 + rc + 1;
+    }
+    const long long warp_first = row0 + warp * 16, warp_last = warp_first + 15;
+    const long long w_min_end = a.q_pos0 + (warp_first < a.L_q ? warp_first : a.L_q - 1) + 1;
+    const long long w_max_end = a.q_pos0 + (warp_last < a.L_q ? warp_last : a.L_q - 1) + 1;
+
+    uint32_t qa[D_K / 16][4];
+    {
+        const __half *qb = a.q + (size_t)(b * a.H_q + hq) * a.L_q * D_K;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const __half *qr = qb + (size_t)(vis_end[i] - 1 - a.q_pos0) * D_K;
+#pragma unroll
+            for (int ks = 0; ks < D_K / 16; ++ks) {
+                qa[ks][i] = *reinterpret_cast<const uint32_t *>(qr + ks * 16 + 2 * t);
+                qa[ks][2 + i] = *reinterpret_cast<const uint32_t *>(qr + ks * 16 + 2 * t + 8);
+            }
+        }
+    }
+
+    // ---- staging of one chunk: V rows by cp.async; centroid rows gathered to registers, split, stored ----
+    auto stage_v = [&](int c, int buf) {
+        const unsigned vs = smem0 + buf * Lay::kStage + 2 * Lay::kPlane;
+        constexpr int per_row = D_V * 2 / 16;
+#pragma unroll
+        for (int i = 0; i < kPmChunk * per_row / kPmThreads; ++i) {
+            const int p = tid + i * kPmThreads, tl = p / per_row, piece = p % per_row;
+            const long long tok = (long long)c * kPmChunk + tl;
+            if (tok < t_end)
+                pm_cp_async16(vs + tl * Lay::kPitchV + piece * 16, vsrc + (size_t)tok * D_V + piece * 8);
+            else
+                *reinterpret_cast<uint4 *>(pm_smem + buf * Lay::kStage + 2 * Lay::kPlane + tl * Lay::kPitchV + piece * 16) =
+                    make_uint4(0u, 0u, 0u, 0u);
+        }
+        pm_commit();
+    };
+    float4 gx[Lay::kPieces], gy[Lay::kPieces];
+    auto gather = [&](int c) {
+#pragma unroll
+        for (int i = 0; i < Lay::kPieces; ++i) {
+            const int p = tid + i * kPmThreads, tl = p / Lay::kGroups, d0 = (p % Lay::kGroups) * 8;
+            const long long tok = (long long)c * kPmChunk + tl;
+            gx[i] = gy[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (tok < t_end) {
+                const int j0 = d0 / d_sub, j1 = (d0 + 4) / d_sub;
+                const int c0 = codes[(size_t)tok * a.m + j0], c1 = codes[(size_t)tok * a.m + j1];
+                gx[i] = __ldg(reinterpret_cast<const float4 *>(book + ((size_t)j0 * a.K + c0) * d_sub + (d0 - j0 * d_sub)));
+                gy[i] = __ldg(reinterpret_cast<const float4 *>(book + ((size_t)j1 * a.K + c1) * d_sub + (d0 + 4 - j1 * d_sub)));
+            }
+        }
+    };
+    auto store_keys = [&](int buf) {
+#pragma unroll
+        for (int i = 0; i < Lay::kPieces; ++i) {
+            const int p = tid + i * kPmThreads, tl = p / Lay::kGroups, gi = p % Lay::kGroups;
+            uint4 hi, lo;
+            pm_split8(gx[i], gy[i], hi, lo);
+            unsigned char *dst = pm_smem + buf * Lay::kStage + tl * Lay::kPitchK + gi * 16;
+            *reinterpret_cast<uint4 *>(dst) = hi;
+            *reinterpret_cast<uint4 *>(dst + Lay::kPlane) = lo;
+        }
+    };
+
+    stage_v(0, 0);
+    gather(0);
+    store_keys(0);
+    pm_wait_all();
+    __syncthreads();
+
+    float o[D_V / 8][4];
+#pragma unroll
+    for (int nd = 0; nd < D_V / 8; ++nd) o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+
+    // ldmatrix lane addresses: keys (token lane&7, dims 8*(lane>>3)); V (token (lane&7) + 8*((lane>>3)&1), dims 8*(lane>>4))
+    const unsigned k_lane = (lane & 7) * Lay::kPitchK + (lane >> 3) * 16;
+    const unsigned v_lane = ((lane & 7) + ((lane >> 3) & 1) * 8) * Lay::kPitchV + (lane >> 4) * 16;
+
+    for (int c = 0; c < n_chunks; ++c) {
+        const int buf = c & 1;
+        const bool more = c + 1 < n_chunks;
+        const long long tok0 = (long long)c * kPmChunk;
+        const bool active = tok0 < w_max_end;                  // warp-uniform: some row of this warp sees the chunk
+        if (more) stage_v(c + 1, buf ^ 1);
+
+        float s[kPmChunk / 8][4];
+        if (active) {
+            const unsigned kh = smem0 + buf * Lay::kStage + k_lane;
+#pragma unroll
+            for (int nt = 0; nt < kPmChunk / 8; ++nt) {
+                s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+#pragma unroll
+                for (int kp = 0; kp < D_K / 32; ++kp) {
+                    uint32_t bh[4], bl[4];
+                    pm_ldmatrix_x4(bh, kh + nt * 8 * Lay::kPitchK + kp * 64);
+                    pm_ldmatrix_x4(bl, kh + Lay::kPlane + nt * 8 * Lay::kPitchK + kp * 64);
+                    pm_mma(s[nt], qa[2 * kp], bh[0], bh[1]);
+                    pm_mma(s[nt], qa[2 * kp + 1], bh[2], bh[3]);
+                    pm_mma(s[nt], qa[2 * kp], bl[0], bl[1]);
+                    pm_mma(s[nt], qa[2 * kp + 1], bl[2], bl[3]);
+                }
+            }
+        }
+        if (more) gather(c + 1);
+
+        if (active) {
+            // ---- raw scores out (validation), causal mask, online softmax in base 2 ----
+            const bool masked = tok0 + kPmChunk > w_min_end;
+            if (SCORES && a.scores_out) {
+#pragma unroll
+                for (int nt = 0; nt < kPmChunk / 8; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const long long tok = tok0 + nt * 8 + 2 * t + (e & 1);
+                        const int i = e >> 1;
+                        if (row[i] < a.L_q && tok < vis_end[i])
+                            a.scores_out[((size_t)(b * a.H_q + hq) * a.L_q + row[i]) * a.L_max + tok] = s[nt][e];
+                    }
+            }
+            float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+            for (int nt = 0; nt < kPmChunk / 8; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float sc = s[nt][e] * a.scale_log2;
+                    if (masked && tok0 + nt * 8 + 2 * t + (e & 1) >= vis_end[e >> 1]) sc = -INFINITY;
+                    s[nt][e] = sc;
+                    mx[e >> 1] = fmaxf(mx[e >> 1], sc);
+                }
+            float alpha[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 1));
+                mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 2));
+                const float m_new = fmaxf(m_run[i], mx[i]);     // finite from chunk 0 on: token 0 is visible to every row
+                alpha[i] = ex2_approx(m_run[i] - m_new);
+                m_run[i] = m_new;
+                l_run[i] *= alpha[i];
+            }
+#pragma unroll
+            for (int nd = 0; nd < D_V / 8; ++nd) {
+                o[nd][0] *= alpha[0];
+                o[nd][1] *= alpha[0];
+                o[nd][2] *= alpha[1];
+                o[nd][3] *= alpha[1];
+            }
+            // ---- weights as fp16 operands (two planes when SPLIT_P); the row sums use what the MMA will see ----
+            uint32_t ph[kPmChunk / 8][2], pl[SPLIT_P ? kPmChunk / 8 : 1][2];
+#pragma unroll
+            for (int nt = 0; nt < kPmChunk / 8; ++nt)
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const float p0 = ex2_approx(s[nt][2 * i] - m_run[i]), p1 = ex2_approx(s[nt][2 * i + 1] - m_run[i]);
+                    const __half2 hh = __floats2half2_rn(p0, p1);
+                    ph[nt][i] = *reinterpret_cast<const uint32_t *>(&hh);
+                    if (SPLIT_P) {
+                        const float2 back = __half22float2(hh);
+                        pl[nt][i] = pm_pack(p0 - back.x, p1 - back.y);
+                        l_run[i] += p0 + p1;
+                    } else {
+                        const float2 back = __half22float2(hh);
+                        l_run[i] += back.x + back.y;
+                    }
+                }
+            const unsigned vs = smem0 + buf * Lay::kStage + 2 * Lay::kPlane + v_lane;
+#pragma unroll
+            for (int kt = 0; kt < kPmChunk / 16; ++kt) {
+                const uint32_t pa[4] = {ph[2 * kt][0], ph[2 * kt][1], ph[2 * kt + 1][0], ph[2 * kt + 1][1]};
+#pragma unroll
+                for (int np = 0; np < D_V / 16; ++np) {
+                    uint32_t vb[4];
+                    pm_ldmatrix_x4_trans(vb, vs + kt * 16 * Lay::kPitchV + np * 32);
+                    pm_mma(o[2 * np], pa, vb[0], vb[1]);
+                    pm_mma(o[2 * np + 1], pa, vb[2], vb[3]);
+                    if (SPLIT_P) {
+                        const uint32_t pb[4] = {pl[2 * kt][0], pl[2 * kt][1], pl[2 * kt + 1][0], pl[2 * kt + 1][1]};
+                        pm_mma(o[2 * np], pb, vb[0], vb[1]);
+                        pm_mma(o[2 * np + 1], pb, vb[2], vb[3]);
+                    }
+                }
+            }
+        }
+        if (more) store_keys(buf ^ 1);
+        pm_wait_all();
+        __syncthreads();
+    }
+
+    // ---- normalise and store ----
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
+        l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
+        if (row[i] >= a.L_q) continue;
+        const float inv = 1.f / l_run[i];
+        float *dst = a.out + ((size_t)(b * a.H_q + hq) * a.L_q + row[i]) * D_V + 2 * t;
+#pragma unroll
+        for (int nd = 0; nd < D_V / 8; ++nd)
+            *reinterpret_cast<float2 *>(dst + nd * 8) = make_float2(o[nd][2 * i] * inv, o[nd][2 * i + 1] * inv);
+    }
+}
+
+template <int D_K, int D_V>
+lookat_status launch_pm(Ctx *ctx, const PrefillArgs &a)
+{
+    using Lay = PmLayout<D_K, D_V>;
+    const int n_tiles = (int)((a.L_q + kPmRows - 1) / kPmRows);
+    dim3 grid((unsigned)n_tiles, (unsigned)a.H_q, (unsigned)a.B);
+    auto launch = [&](auto kern) -> lookat_status {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kBytes) != cudaSuccess)
+            return check_launch(ctx, "prefill (contraction form): shared-memory opt-in");
+        kern<<<grid, kPmThreads, Lay::kBytes, ctx->stream>>>(a);
+        return check_launch(ctx, "attend_prefill_mma_kernel");
+    };
+    if (a.scores_out) return launch(attend_prefill_mma_kernel<D_K, D_V, true, false>);
+    return launch(attend_prefill_mma_kernel<D_K, D_V, false, false>);
+}
+
+}  // namespace
+
+bool prefill_mma_covers(const Ctx *ctx, const PrefillArgs &a)
+{
+    const int d_sub = a.d_k / a.m;
+    const bool shape = (a.d_k == 64 || a.d_k == 128) && (a.d_v == 64 || a.d_v == 128) && d_sub % 4 == 0;
+    const bool aligned = ((uintptr_t)a.q & 3) == 0 && ((uintptr_t)a.v & 15) == 0 && ((uintptr_t)a.codebooks & 15) == 0;
+    return shape && aligned && a.H_q <= 65535 && a.B <= 65535 &&
+           (size_t)ctx->max_smem_optin >= (size_t)PmLayout<128, 128>::kBytes;
+}
+
+lookat_status launch_prefill_mma(Ctx *ctx, const PrefillArgs &a)
+{
+    if (a.d_k == 128) return a.d_v == 128 ? launch_pm<128, 128>(ctx, a) : launch_pm<128, 64>(ctx, a);
+    return a.d_v == 128 ? launch_pm<64, 128>(ctx, a) : launch_pm<64, 64>(ctx, a);
+}
+
+}  // namespace lookat
