@@ -237,7 +237,8 @@ lookat_status lookat_decode_step_host(lookat_ctx *ctx, const void *q_host, const
  *                               gathered once per 128 queries and the scores
  *                               taken as q . (C_1[c_1], ..., C_m[c_m]) on the
  *                               tensor cores (d_k and d_v in {64, 128}, d_sub a
- *                               multiple of 4);
+ *                               multiple of 8, both codebook planes of a head
+ *                               in shared memory: K * d_k * 4 bytes);
  *   LOOKAT_PREFILL_AUTO         (default) contraction where it applies and
  *                               L_q >= 32, tables otherwise.
  * Asking for the contraction form on a shape it does not cover makes

@@ -262,7 +262,7 @@ void lookat_destroy(lookat_ctx *handle)
     Ctx *ctx = reinterpret_cast<Ctx *>(handle);
     DeviceGuard guard(ctx->device);
     cudaStreamSynchronize(ctx->stream);
-    void *bufs[] = {ctx->part_o, ctx->part_ml, ctx->tickets, ctx->lut_scratch, ctx->fit_sums, ctx->fit_cnt, ctx->fit_assign,
+    void *bufs[] = {ctx->part_o, ctx->part_ml, ctx->tickets, ctx->lut_scratch, ctx->split_books, ctx->fit_sums, ctx->fit_cnt, ctx->fit_assign,
                     ctx->step_q,  ctx->step_k,  ctx->step_out};
     for (void *p : bufs)
         if (p) cudaFree(p);

@@ -33,6 +33,9 @@ struct Ctx {
     // tables built on behalf of the caller (lookat_attend with lut == NULL)
     float *lut_scratch;
     size_t lut_cap;                        // bytes
+    // prefill, contraction form: the codebooks as two fp16 planes (rounding, remainder), [2][H_kv][m][K][d_sub]
+    __half *split_books;
+    size_t split_cap;                      // bytes
     // k-means scratch
     unsigned long long *fit_sums;          // [H_kv][m][K][d_sub] fixed-point sums
     unsigned long long *fit_cnt;           // [H_kv][m][K]

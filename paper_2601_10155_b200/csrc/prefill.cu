@@ -375,7 +375,8 @@ lookat_status launch_prefill(Ctx *ctx, const PrefillArgs &a)
     const bool contraction_ok = prefill_mma_covers(ctx, a);
     if (ctx->prefill_form == LOOKAT_PREFILL_CONTRACTION && !contraction_ok)
         return set_error(ctx, LOOKAT_ERR_UNSUPPORTED,
-                         "attend_prefill: the contraction form needs d_k, d_v in {64, 128} and d_sub a multiple of 4");
+                         "attend_prefill: the contraction form needs d_k, d_v in {64, 128}, d_sub a multiple of 8 and K * d_k * 4 bytes of "
+                         "shared memory for the codebooks");
     if (contraction_ok &&
         (ctx->prefill_form == LOOKAT_PREFILL_CONTRACTION || (ctx->prefill_form == LOOKAT_PREFILL_AUTO && a.L_q >= 32)))
         return launch_prefill_mma(ctx, a);

@@ -9,10 +9,17 @@
 // mma.sync.m16n8k16 and fp32 accumulation.  q (fp16) is an exact operand; every fp32 centroid is
 // split into two fp16 planes (rounding + remainder), which carries s to ~2^-22 relative.
 //
+//
 // One CTA: one (batch row, query head), 128 consecutive queries (8 warps x 16 rows), 64-token chunks up
-// to the causal limit of the tile.  Per chunk: the next chunk's V rows arrive by cp.async and its
-// centroid rows are gathered (global loads that hit L1/L2; the codebook of a head is <= 128 KB) while
-// this chunk's MMAs run; they are split and stored between the phases; one barrier per chunk.
+// to the causal limit of the tile.  Both planes of the head's codebooks (K x d_k x 4 bytes, 128 KB at
+// d_k = 128) stay in shared memory for the life of the CTA, in an order that makes the gathers free of
+// bank conflicts whatever the codes are: the 16-byte item of (8-dim group gi, plane p, centroid c)
+// lives in bank group (2 gi + p) mod 8, and the 8 lanes of a quarter-warp always fetch 8 different
+// (gi, p).  split_codebook_kernel writes that image once per call; a CTA copies it in with cp.async.
+// Per chunk: the next chunk's V rows arrive by cp.async and its key rows are rebuilt (one 16-byte
+// shared load and store per item) while this chunk's MMAs run; the codes are read one chunk further
+// ahead; one barrier per chunk.  Key and V tiles are XOR-swizzled (16-byte piece index ^ token mod 8)
+// instead of padded, so that everything fits in 224 KB.
 #include "common.cuh"
 
 namespace lookat {
@@ -27,6 +34,10 @@ constexpr int kPmChunk = 64;                  // tokens per chunk
 __device__ __forceinline__ void pm_cp_async16(unsigned dst, const void *src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void pm_cp_async8(unsigned dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void pm_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void pm_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
@@ -57,43 +68,52 @@ __device__ __forceinline__ uint32_t pm_pack(float lo, float hi)
     return *reinterpret_cast<const uint32_t *>(&h);
 }
 
-// Rounding and remainder planes of 8 consecutive fp32 values, as two 16-byte rows.
-__device__ __forceinline__ void pm_split8(const float4 &x, const float4 &y, uint4 &hi, uint4 &lo)
+
+// Shared-memory image of one head's codebooks as two fp16 planes, hi = fp16(c), lo = fp16(c - hi):
+// halfs [d_k/32][K][8 slots][8], slot = 2 (gi mod 4) + plane for the 8-dim group gi of the key row.
+__global__ void split_codebook_kernel(const float *__restrict__ books, __half *__restrict__ images, int H_kv, int m, int K,
+                                      int d_sub)
 {
-    const float v[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
-    uint32_t h[4], l[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const __half2 hh = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
-        const float2 back = __half22float2(hh);
-        const __half2 ll = __floats2half2_rn(v[2 * i] - back.x, v[2 * i + 1] - back.y);
-        h[i] = *reinterpret_cast<const uint32_t *>(&hh);
-        l[i] = *reinterpret_cast<const uint32_t *>(&ll);
+    const int d_k = m * d_sub;
+    const size_t n = (size_t)H_kv * K * d_k;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        // i indexes books [h][j][c][e]
+        const int e = (int)(i % d_sub), c = (int)(i / d_sub % K), j = (int)(i / ((size_t)d_sub * K) % m);
+        const int h = (int)(i / ((size_t)d_sub * K * m));
+        const int dim = j * d_sub + e, gi = dim >> 3;
+        const float v = books[i];
+        const __half hi = __float2half_rn(v), lo = __float2half_rn(v - __half2float(hi));
+        __half *img = images + (size_t)h * K * d_k * 2;
+        const size_t at = (((size_t)(gi >> 2) * K + c) * 8 + (gi & 3) * 2) * 8 + (dim & 7);
+        img[at] = hi;
+        img[at + 8] = lo;
     }
-    hi = make_uint4(h[0], h[1], h[2], h[3]);
-    lo = make_uint4(l[0], l[1], l[2], l[3]);
 }
 
 template <int D_K, int D_V>
 struct PmLayout {
-    static constexpr int kPitchK = D_K * 2 + 16;                       // bytes per rebuilt key row (one plane)
-    static constexpr int kPitchV = D_V * 2 + 16;
-    static constexpr int kPlane = kPmChunk * kPitchK;
-    static constexpr int kVTile = kPmChunk * kPitchV;
+    static constexpr int kRowK = D_K * 2;                              // bytes per rebuilt key row (one plane)
+    static constexpr int kRowV = D_V * 2;
+    static constexpr int kPlane = kPmChunk * kRowK;
+    static constexpr int kVTile = kPmChunk * kRowV;
     static constexpr int kStage = 2 * kPlane + kVTile;                 // hi plane, lo plane, V
-    static constexpr int kBytes = 2 * kStage;
-    static constexpr int kGroups = D_K / 8;                            // 8-dim groups per key row
-    static constexpr int kPieces = kPmChunk * kGroups / kPmThreads;    // groups gathered per thread per chunk
-    static_assert(kPmChunk * kGroups % kPmThreads == 0, "whole pieces per thread");
+    static constexpr int kIds = D_K / 4;                               // 16-byte items per key row, both planes
+    static constexpr int kItems = kPmChunk * kIds / kPmThreads;        // items rebuilt per thread per chunk
+    static_assert(kPmChunk * kIds % kPmThreads == 0, "whole items per thread");
+    static size_t book_bytes(int K) { return (size_t)K * D_K * 4; }
+    static size_t bytes(int K) { return book_bytes(K) + 2 * kStage; }
 };
 
 template <int D_K, int D_V, bool SCORES, bool SPLIT_P>
 __global__ void __launch_bounds__(kPmThreads, 1)
-attend_prefill_mma_kernel(PrefillArgs a)
+attend_prefill_mma_kernel(PrefillArgs a, const __half *__restrict__ images)
 {
     using Lay = PmLayout<D_K, D_V>;
-    extern __shared__ __align__(16) unsigned char pm_smem[];
+    extern __shared__ __align__(128) unsigned char pm_smem[];
     const unsigned smem0 = (unsigned)__cvta_generic_to_shared(pm_smem);
+    const unsigned book_bytes = (unsigned)a.K * D_K * 4;
+    unsigned char *const stages = pm_smem + book_bytes;
+    const unsigned stages0 = smem0 + book_bytes;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
@@ -106,9 +126,14 @@ attend_prefill_mma_kernel(PrefillArgs a)
     const long long t_end = a.q_pos0 + (row0 + kPmRows < a.L_q ? row0 + kPmRows : a.L_q);   // tokens the tile sees
     const int n_chunks = (int)((t_end + kPmChunk - 1) / kPmChunk);
 
-    const float *book = a.codebooks + (size_t)h * a.m * a.K * d_sub;
     const uint8_t *codes = a.codes + (size_t)(b * a.H_kv + h) * a.L_max * a.m;
     const __half *vsrc = a.v + (size_t)(b * a.H_kv + h) * a.L_max * D_V;
+
+    // ---- the head's codebook image: a flat copy ----
+    {
+        const unsigned char *img = reinterpret_cast<const unsigned char *>(images) + (size_t)h * book_bytes;
+        for (unsigned i = tid * 16; i < book_bytes; i += kPmThreads * 16) pm_cp_async16(smem0 + i, img + i);
+    }
 
     // ---- this thread's two query rows (clamped copies beyond L_q are computed and dropped) ----
     long long row[2], vis_end[2];
@@ -136,53 +161,52 @@ attend_prefill_mma_kernel(PrefillArgs a)
         }
     }
 
-    // ---- staging of one chunk: V rows by cp.async; centroid rows gathered to registers, split, stored ----
-    auto stage_v = [&](int c, int buf) {
-        const unsigned vs = smem0 + buf * Lay::kStage + 2 * Lay::kPlane;
+    // ---- staging of one chunk ----
+    auto stage_v = [&](int c, int buf) {                        // V rows by cp.async, pieces swizzled by token
         constexpr int per_row = D_V * 2 / 16;
+        const unsigned vo = buf * Lay::kStage + 2 * Lay::kPlane;
 #pragma unroll
         for (int i = 0; i < kPmChunk * per_row / kPmThreads; ++i) {
             const int p = tid + i * kPmThreads, tl = p / per_row, piece = p % per_row;
             const long long tok = (long long)c * kPmChunk + tl;
+            const unsigned off = vo + tl * Lay::kRowV + ((piece ^ (tl & 7)) << 4);
             if (tok < t_end)
-                pm_cp_async16(vs + tl * Lay::kPitchV + piece * 16, vsrc + (size_t)tok * D_V + piece * 8);
+                pm_cp_async16(stages0 + off, vsrc + (size_t)tok * D_V + piece * 8);
             else
-                *reinterpret_cast<uint4 *>(pm_smem + buf * Lay::kStage + 2 * Lay::kPlane + tl * Lay::kPitchV + piece * 16) =
-                    make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4 *>(stages + off) = make_uint4(0u, 0u, 0u, 0u);
         }
         pm_commit();
     };
-    float4 gx[Lay::kPieces], gy[Lay::kPieces];
-    auto gather = [&](int c) {
+    // item p = tid + i * threads of a chunk: token p / kIds, id = p % kIds = 2 gi + plane
+    const int my_id = tid % Lay::kIds, my_gi = my_id >> 1, my_plane = my_id & 1;
+    const int my_j = (my_gi * 8) / d_sub;
+    const unsigned my_src = (unsigned)(my_gi >> 2) * a.K * 128 + (((my_gi & 3) * 2 + my_plane) << 4);   // + c * 128
+    uint32_t cd[Lay::kItems];                                   // codes of this thread's items; 0xffffffff = token not seen
+    auto load_codes = [&](int c) {
 #pragma unroll
-        for (int i = 0; i < Lay::kPieces; ++i) {
-            const int p = tid + i * kPmThreads, tl = p / Lay::kGroups, d0 = (p % Lay::kGroups) * 8;
+        for (int i = 0; i < Lay::kItems; ++i) {
+            const int tl = (tid + i * kPmThreads) / Lay::kIds;
             const long long tok = (long long)c * kPmChunk + tl;
-            gx[i] = gy[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (tok < t_end) {
-                const int j0 = d0 / d_sub, j1 = (d0 + 4) / d_sub;
-                const int c0 = codes[(size_t)tok * a.m + j0], c1 = codes[(size_t)tok * a.m + j1];
-                gx[i] = __ldg(reinterpret_cast<const float4 *>(book + ((size_t)j0 * a.K + c0) * d_sub + (d0 - j0 * d_sub)));
-                gy[i] = __ldg(reinterpret_cast<const float4 *>(book + ((size_t)j1 * a.K + c1) * d_sub + (d0 + 4 - j1 * d_sub)));
-            }
+            cd[i] = tok < t_end ? (uint32_t)codes[(size_t)tok * a.m + my_j] : 0xffffffffu;
         }
     };
-    auto store_keys = [&](int buf) {
+    auto rebuild_keys = [&](int buf) {                          // uses cd[]: the chunk whose codes were loaded last
 #pragma unroll
-        for (int i = 0; i < Lay::kPieces; ++i) {
-            const int p = tid + i * kPmThreads, tl = p / Lay::kGroups, gi = p % Lay::kGroups;
-            uint4 hi, lo;
-            pm_split8(gx[i], gy[i], hi, lo);
-            unsigned char *dst = pm_smem + buf * Lay::kStage + tl * Lay::kPitchK + gi * 16;
-            *reinterpret_cast<uint4 *>(dst) = hi;
-            *reinterpret_cast<uint4 *>(dst + Lay::kPlane) = lo;
+        for (int i = 0; i < Lay::kItems; ++i) {
+            const int tl = (tid + i * kPmThreads) / Lay::kIds;
+            uint4 item = make_uint4(0u, 0u, 0u, 0u);
+            if (cd[i] != 0xffffffffu) item = *reinterpret_cast<const uint4 *>(pm_smem + my_src + cd[i] * 128);
+            *reinterpret_cast<uint4 *>(stages + buf * Lay::kStage + my_plane * Lay::kPlane + tl * Lay::kRowK +
+                                       ((my_gi ^ (tl & 7) ^ (my_plane << 2)) << 4)) = item;
         }
     };
 
-    stage_v(0, 0);
-    gather(0);
-    store_keys(0);
+    load_codes(0);
+    stage_v(0, 0);                                              // commits the codebook copy as well
     pm_wait_all();
+    __syncthreads();
+    rebuild_keys(0);
+    if (n_chunks > 1) load_codes(1);
     __syncthreads();
 
     float o[D_V / 8][4];
@@ -190,9 +214,12 @@ attend_prefill_mma_kernel(PrefillArgs a)
     for (int nd = 0; nd < D_V / 8; ++nd) o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f;
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
 
-    // ldmatrix lane addresses: keys (token lane&7, dims 8*(lane>>3)); V (token (lane&7) + 8*((lane>>3)&1), dims 8*(lane>>4))
-    const unsigned k_lane = (lane & 7) * Lay::kPitchK + (lane >> 3) * 16;
-    const unsigned v_lane = ((lane & 7) + ((lane >> 3) & 1) * 8) * Lay::kPitchV + (lane >> 4) * 16;
+    // ldmatrix lane addresses.  Keys: token lane&7 of an 8-token group, 16-byte piece (lane>>3) of a 32-dim
+    // group; the lo plane's pieces are swizzled with one more bit (^4).  V: token (lane&7) + 8 ((lane>>3)&1),
+    // piece lane>>4 of a 16-column group.
+    const int r7 = lane & 7;
+    const unsigned k_row = r7 * Lay::kRowK;
+    const unsigned v_row = (r7 + ((lane >> 3) & 1) * 8) * Lay::kRowV;
 
     for (int c = 0; c < n_chunks; ++c) {
         const int buf = c & 1;
@@ -203,15 +230,17 @@ attend_prefill_mma_kernel(PrefillArgs a)
 
         float s[kPmChunk / 8][4];
         if (active) {
-            const unsigned kh = smem0 + buf * Lay::kStage + k_lane;
+            const unsigned kh = stages0 + buf * Lay::kStage + k_row;
 #pragma unroll
-            for (int nt = 0; nt < kPmChunk / 8; ++nt) {
-                s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+            for (int nt = 0; nt < kPmChunk / 8; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
 #pragma unroll
-                for (int kp = 0; kp < D_K / 32; ++kp) {
+            for (int kp = 0; kp < D_K / 32; ++kp) {
+                const unsigned piece = (unsigned)(((kp * 4 + (lane >> 3)) ^ r7) << 4);
+#pragma unroll
+                for (int nt = 0; nt < kPmChunk / 8; ++nt) {
                     uint32_t bh[4], bl[4];
-                    pm_ldmatrix_x4(bh, kh + nt * 8 * Lay::kPitchK + kp * 64);
-                    pm_ldmatrix_x4(bl, kh + Lay::kPlane + nt * 8 * Lay::kPitchK + kp * 64);
+                    pm_ldmatrix_x4(bh, kh + nt * 8 * Lay::kRowK + piece);
+                    pm_ldmatrix_x4(bl, kh + Lay::kPlane + nt * 8 * Lay::kRowK + (piece ^ 64u));
                     pm_mma(s[nt], qa[2 * kp], bh[0], bh[1]);
                     pm_mma(s[nt], qa[2 * kp + 1], bh[2], bh[3]);
                     pm_mma(s[nt], qa[2 * kp], bl[0], bl[1]);
@@ -219,7 +248,6 @@ attend_prefill_mma_kernel(PrefillArgs a)
                 }
             }
         }
-        if (more) gather(c + 1);
 
         if (active) {
             // ---- raw scores out (validation), causal mask, online softmax in base 2 ----
@@ -271,23 +299,22 @@ attend_prefill_mma_kernel(PrefillArgs a)
                     const float p0 = ex2_approx(s[nt][2 * i] - m_run[i]), p1 = ex2_approx(s[nt][2 * i + 1] - m_run[i]);
                     const __half2 hh = __floats2half2_rn(p0, p1);
                     ph[nt][i] = *reinterpret_cast<const uint32_t *>(&hh);
+                    const float2 back = __half22float2(hh);
                     if (SPLIT_P) {
-                        const float2 back = __half22float2(hh);
                         pl[nt][i] = pm_pack(p0 - back.x, p1 - back.y);
                         l_run[i] += p0 + p1;
                     } else {
-                        const float2 back = __half22float2(hh);
                         l_run[i] += back.x + back.y;
                     }
                 }
-            const unsigned vs = smem0 + buf * Lay::kStage + 2 * Lay::kPlane + v_lane;
+            const unsigned vs = stages0 + buf * Lay::kStage + 2 * Lay::kPlane + v_row;
 #pragma unroll
             for (int kt = 0; kt < kPmChunk / 16; ++kt) {
                 const uint32_t pa[4] = {ph[2 * kt][0], ph[2 * kt][1], ph[2 * kt + 1][0], ph[2 * kt + 1][1]};
 #pragma unroll
                 for (int np = 0; np < D_V / 16; ++np) {
                     uint32_t vb[4];
-                    pm_ldmatrix_x4_trans(vb, vs + kt * 16 * Lay::kPitchV + np * 32);
+                    pm_ldmatrix_x4_trans(vb, vs + kt * 16 * Lay::kRowV + (((np * 2 + (lane >> 4)) ^ r7) << 4));
                     pm_mma(o[2 * np], pa, vb[0], vb[1]);
                     pm_mma(o[2 * np + 1], pa, vb[2], vb[3]);
                     if (SPLIT_P) {
@@ -298,7 +325,10 @@ attend_prefill_mma_kernel(PrefillArgs a)
                 }
             }
         }
-        if (more) store_keys(buf ^ 1);
+        if (more) {
+            rebuild_keys(buf ^ 1);                              // chunk c+1: its codes arrived during this step
+            if (c + 2 < n_chunks) load_codes(c + 2);
+        }
         pm_wait_all();
         __syncthreads();
     }
@@ -321,12 +351,22 @@ template <int D_K, int D_V>
 lookat_status launch_pm(Ctx *ctx, const PrefillArgs &a)
 {
     using Lay = PmLayout<D_K, D_V>;
+    // the codebooks as shared-memory images of two fp16 planes, rewritten at every call (the caller may have refitted them)
+    const size_t elems = (size_t)a.H_kv * a.K * a.d_k;
+    lookat_status st = ensure(ctx, (void **)&ctx->split_books, &ctx->split_cap, 2 * elems * sizeof(__half), "codebook planes");
+    if (st != LOOKAT_OK) return st;
+    split_codebook_kernel<<<(unsigned)((elems + 1023) / 1024), 256, 0, ctx->stream>>>(a.codebooks, ctx->split_books, a.H_kv,
+                                                                                      a.m, a.K, a.d_k / a.m);
+    st = check_launch(ctx, "split_codebook_kernel");
+    if (st != LOOKAT_OK) return st;
+
     const int n_tiles = (int)((a.L_q + kPmRows - 1) / kPmRows);
+    const int smem = (int)Lay::bytes(a.K);
     dim3 grid((unsigned)n_tiles, (unsigned)a.H_q, (unsigned)a.B);
     auto launch = [&](auto kern) -> lookat_status {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return check_launch(ctx, "prefill (contraction form): shared-memory opt-in");
-        kern<<<grid, kPmThreads, Lay::kBytes, ctx->stream>>>(a);
+        kern<<<grid, kPmThreads, smem, ctx->stream>>>(a, ctx->split_books);
         return check_launch(ctx, "attend_prefill_mma_kernel");
     };
     if (a.scores_out) return launch(attend_prefill_mma_kernel<D_K, D_V, true, false>);
@@ -338,10 +378,11 @@ lookat_status launch_pm(Ctx *ctx, const PrefillArgs &a)
 bool prefill_mma_covers(const Ctx *ctx, const PrefillArgs &a)
 {
     const int d_sub = a.d_k / a.m;
-    const bool shape = (a.d_k == 64 || a.d_k == 128) && (a.d_v == 64 || a.d_v == 128) && d_sub % 4 == 0;
-    const bool aligned = ((uintptr_t)a.q & 3) == 0 && ((uintptr_t)a.v & 15) == 0 && ((uintptr_t)a.codebooks & 15) == 0;
-    return shape && aligned && a.H_q <= 65535 && a.B <= 65535 &&
-           (size_t)ctx->max_smem_optin >= (size_t)PmLayout<128, 128>::kBytes;
+    const bool shape = (a.d_k == 64 || a.d_k == 128) && (a.d_v == 64 || a.d_v == 128) && d_sub % 8 == 0;
+    const bool aligned = ((uintptr_t)a.q & 3) == 0 && ((uintptr_t)a.v & 15) == 0;
+    if (!shape || !aligned || a.H_q > 65535 || a.B > 65535) return false;
+    const size_t stage = (size_t)kPmChunk * (4 * a.d_k + 2 * a.d_v);
+    return (size_t)a.K * a.d_k * 4 + 2 * stage <= (size_t)ctx->max_smem_optin;
 }
 
 lookat_status launch_prefill_mma(Ctx *ctx, const PrefillArgs &a)

@@ -403,7 +403,8 @@ def test_invalid_arguments_are_rejected_without_launching():
     (dict(B=2, n_q_heads=2, n_kv_heads=1, d_k=32, d_v=32, m=2, K=16, L=70), 1, 69),         # one query = a decode step
     (dict(B=1, n_q_heads=3, n_kv_heads=3, d_k=24, d_v=16, m=8, K=7, L=65), 65, 0),          # d_sub 3, small K
     (dict(B=1, n_q_heads=2, n_kv_heads=1, d_k=128, d_v=64, m=16, K=200, L=450), 300, 150),  # 3 query tiles, ragged, K < 256
-    (dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=128, m=16, K=256, L=257), 257, 0),    # d_sub 4; one row in the last tile
+    (dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=128, m=8, K=256, L=257), 257, 0),     # d_k 64; one row in the last tile
+    (dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=64, m=16, K=256, L=90), 90, 0),       # d_sub 4: tables only
 ])
 @pytest.mark.parametrize("q_scale", [1.0, 0.1])
 @pytest.mark.parametrize("form", ["tables", "contraction"])
@@ -416,7 +417,7 @@ def test_attend_prefill_matches_oracle(shape, L_q, q_pos0, q_scale, form):
     lk = ctx_for(w)
     lk.lookat_set_prefill_form(form)
     scores = torch.full((w.B, w.n_q_heads, L_q, w.L), float("nan"), device="cuda")
-    covered = w.d_k in (64, 128) and w.d_v in (64, 128) and w.d_sub % 4 == 0
+    covered = w.d_k in (64, 128) and w.d_v in (64, 128) and w.d_sub % 8 == 0
     if form == "contraction" and not covered:
         with pytest.raises(LookatError):
             lk.lookat_attend_prefill(dev(q), dev(books), dev(codes), dev(v), q_pos0=q_pos0, scores_out=scores)
