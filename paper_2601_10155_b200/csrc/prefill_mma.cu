@@ -212,7 +212,9 @@ attend_prefill_mma_kernel(PrefillArgs a, const __half *__restrict__ images)
     float o[D_V / 8][4];
 #pragma unroll
     for (int nd = 0; nd < D_V / 8; ++nd) o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f;
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    float m_run[2] = {-INFINITY, -INFINITY};                    // running maxima, in units of the base-2 exponent
+    float l_acc[4] = {0.f, 0.f, 0.f, 0.f};                      // running row sums: P times a block of ones
+    constexpr uint32_t kOnes = 0x3c003c00u;                     // half2(1, 1)
 
     // ldmatrix lane addresses.  Keys: token lane&7 of an 8-token group, 16-byte piece (lane>>3) of a 32-dim
     // group; the lo plane's pieces are swizzled with one more bit (^4).  V: token (lane&7) + 8 ((lane>>3)&1),
@@ -226,8 +228,6 @@ attend_prefill_mma_kernel(PrefillArgs a, const __half *__restrict__ images)
         const bool more = c + 1 < n_chunks;
         const long long tok0 = (long long)c * kPmChunk;
         const bool active = tok0 < w_max_end;                  // warp-uniform: some row of this warp sees the chunk
-        if (more) stage_v(c + 1, buf ^ 1);
-
         float s[kPmChunk / 8][4];
         if (active) {
             const unsigned kh = stages0 + buf * Lay::kStage + k_row;
@@ -249,6 +249,8 @@ attend_prefill_mma_kernel(PrefillArgs a, const __half *__restrict__ images)
             }
         }
 
+        if (more) stage_v(c + 1, buf ^ 1);                     // issued while the score MMAs drain
+
         if (active) {
             // ---- raw scores out (validation), causal mask, online softmax in base 2 ----
             const bool masked = tok0 + kPmChunk > w_min_end;
@@ -263,54 +265,60 @@ attend_prefill_mma_kernel(PrefillArgs a, const __half *__restrict__ images)
                             a.scores_out[((size_t)(b * a.H_q + hq) * a.L_q + row[i]) * a.L_max + tok] = s[nt][e];
                     }
             }
-            float mx[2] = {-INFINITY, -INFINITY};
+            float mx[2] = {-INFINITY, -INFINITY};               // row maxima of the raw scores (scale > 0)
 #pragma unroll
             for (int nt = 0; nt < kPmChunk / 8; ++nt)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    float sc = s[nt][e] * a.scale_log2;
-                    if (masked && tok0 + nt * 8 + 2 * t + (e & 1) >= vis_end[e >> 1]) sc = -INFINITY;
-                    s[nt][e] = sc;
-                    mx[e >> 1] = fmaxf(mx[e >> 1], sc);
+                    if (masked && tok0 + nt * 8 + 2 * t + (e & 1) >= vis_end[e >> 1]) s[nt][e] = -INFINITY;
+                    mx[e >> 1] = fmaxf(mx[e >> 1], s[nt][e]);
                 }
             float alpha[2];
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
                 mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 1));
                 mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 2));
-                const float m_new = fmaxf(m_run[i], mx[i]);     // finite from chunk 0 on: token 0 is visible to every row
+                const float m_new = fmaxf(m_run[i], mx[i] * a.scale_log2);   // finite from chunk 0 on: token 0 is visible to every row
                 alpha[i] = ex2_approx(m_run[i] - m_new);
                 m_run[i] = m_new;
-                l_run[i] *= alpha[i];
             }
+            if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {   // a maximum moved: rescale
 #pragma unroll
-            for (int nd = 0; nd < D_V / 8; ++nd) {
-                o[nd][0] *= alpha[0];
-                o[nd][1] *= alpha[0];
-                o[nd][2] *= alpha[1];
-                o[nd][3] *= alpha[1];
+                for (int nd = 0; nd < D_V / 8; ++nd) {
+                    o[nd][0] *= alpha[0];
+                    o[nd][1] *= alpha[0];
+                    o[nd][2] *= alpha[1];
+                    o[nd][3] *= alpha[1];
+                }
+                l_acc[0] *= alpha[0];
+                l_acc[1] *= alpha[0];
+                l_acc[2] *= alpha[1];
+                l_acc[3] *= alpha[1];
             }
-            // ---- weights as fp16 operands (two planes when SPLIT_P); the row sums use what the MMA will see ----
+            // ---- weights as fp16 operands (two planes when SPLIT_P) ----
             uint32_t ph[kPmChunk / 8][2], pl[SPLIT_P ? kPmChunk / 8 : 1][2];
 #pragma unroll
             for (int nt = 0; nt < kPmChunk / 8; ++nt)
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
-                    const float p0 = ex2_approx(s[nt][2 * i] - m_run[i]), p1 = ex2_approx(s[nt][2 * i + 1] - m_run[i]);
+                    const float p0 = ex2_approx(fmaf(s[nt][2 * i], a.scale_log2, -m_run[i]));
+                    const float p1 = ex2_approx(fmaf(s[nt][2 * i + 1], a.scale_log2, -m_run[i]));
                     const __half2 hh = __floats2half2_rn(p0, p1);
                     ph[nt][i] = *reinterpret_cast<const uint32_t *>(&hh);
-                    const float2 back = __half22float2(hh);
                     if (SPLIT_P) {
+                        const float2 back = __half22float2(hh);
                         pl[nt][i] = pm_pack(p0 - back.x, p1 - back.y);
-                        l_run[i] += p0 + p1;
-                    } else {
-                        l_run[i] += back.x + back.y;
                     }
                 }
             const unsigned vs = stages0 + buf * Lay::kStage + 2 * Lay::kPlane + v_row;
 #pragma unroll
             for (int kt = 0; kt < kPmChunk / 16; ++kt) {
                 const uint32_t pa[4] = {ph[2 * kt][0], ph[2 * kt][1], ph[2 * kt + 1][0], ph[2 * kt + 1][1]};
+                pm_mma(l_acc, pa, kOnes, kOnes);                // row sums of exactly the weights the value sum uses
+                if (SPLIT_P) {
+                    const uint32_t pb[4] = {pl[2 * kt][0], pl[2 * kt][1], pl[2 * kt + 1][0], pl[2 * kt + 1][1]};
+                    pm_mma(l_acc, pb, kOnes, kOnes);
+                }
 #pragma unroll
                 for (int np = 0; np < D_V / 16; ++np) {
                     uint32_t vb[4];
@@ -336,10 +344,8 @@ attend_prefill_mma_kernel(PrefillArgs a, const __half *__restrict__ images)
     // ---- normalise and store ----
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
-        l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
-        l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
         if (row[i] >= a.L_q) continue;
-        const float inv = 1.f / l_run[i];
+        const float inv = 1.f / l_acc[2 * i];                   // every column of the ones block holds the row sum
         float *dst = a.out + ((size_t)(b * a.H_q + hq) * a.L_q + row[i]) * D_V + 2 * t;
 #pragma unroll
         for (int nd = 0; nd < D_V / 8; ++nd)
@@ -380,7 +386,8 @@ bool prefill_mma_covers(const Ctx *ctx, const PrefillArgs &a)
     const int d_sub = a.d_k / a.m;
     const bool shape = (a.d_k == 64 || a.d_k == 128) && (a.d_v == 64 || a.d_v == 128) && d_sub % 8 == 0;
     const bool aligned = ((uintptr_t)a.q & 3) == 0 && ((uintptr_t)a.v & 15) == 0;
-    if (!shape || !aligned || a.H_q > 65535 || a.B > 65535) return false;
+    // the row maxima are taken on the raw scores, which needs a positive softmax scale
+    if (!shape || !aligned || a.H_q > 65535 || a.B > 65535 || !(a.scale_log2 > 0.f)) return false;
     const size_t stage = (size_t)kPmChunk * (4 * a.d_k + 2 * a.d_v);
     return (size_t)a.K * a.d_k * 4 + 2 * stage <= (size_t)ctx->max_smem_optin;
 }
