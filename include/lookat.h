@@ -41,7 +41,7 @@ typedef enum {
     LOOKAT_ERR_UNSUPPORTED = 2,   /* valid but not implemented for this shape */
     LOOKAT_ERR_CUDA = 3,          /* a CUDA runtime call failed; see lookat_last_error */
     LOOKAT_ERR_NOMEM = 4,         /* scratch allocation failed */
-    LOOKAT_ERR_TIMEOUT = 5        /* reserved: a bounded device-side wait expired */
+    LOOKAT_ERR_TIMEOUT = 5        /* a bounded device-side wait expired (reported by the next lookat_attend_prefill) */
 } lookat_status;
 
 typedef struct {
@@ -239,13 +239,22 @@ lookat_status lookat_decode_step_host(lookat_ctx *ctx, const void *q_host, const
  *                               tensor cores (d_k and d_v in {64, 128}, d_sub a
  *                               multiple of 8, both codebook planes of a head
  *                               in shared memory: K * d_k * 4 bytes);
+ *                               tcgen05.mma with accumulators in tensor memory;
+ *   LOOKAT_PREFILL_CONTRACTION_MMA_SYNC  the same contraction on the legacy
+ *                               mma.sync path, kept as the baseline the tcgen05
+ *                               kernel is measured against;
  *   LOOKAT_PREFILL_AUTO         (default) contraction where it applies and
  *                               L_q >= 32, tables otherwise.
  * Asking for the contraction form on a shape it does not cover makes
  * lookat_attend_prefill return LOOKAT_ERR_UNSUPPORTED.  Returns
  * LOOKAT_ERR_INVALID_ARG for an unknown value.
  */
-enum { LOOKAT_PREFILL_AUTO = 0, LOOKAT_PREFILL_TABLES = 1, LOOKAT_PREFILL_CONTRACTION = 2 };
+enum {
+    LOOKAT_PREFILL_AUTO = 0,
+    LOOKAT_PREFILL_TABLES = 1,
+    LOOKAT_PREFILL_CONTRACTION = 2,
+    LOOKAT_PREFILL_CONTRACTION_MMA_SYNC = 3
+};
 lookat_status lookat_set_prefill_form(lookat_ctx *ctx, int32_t form);
 
 /* Number of kernels this context has launched since it was created. */

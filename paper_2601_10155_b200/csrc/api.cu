@@ -245,6 +245,12 @@ lookat_status lookat_create(const lookat_config *cfg, int device, void *cuda_str
     ctx->sm_count = prop.multiProcessorCount;
     ctx->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
     ctx->prefill_form = LOOKAT_PREFILL_AUTO;
+    if (cudaHostAlloc((void **)&ctx->timeout_flag, sizeof(int), cudaHostAllocMapped) == cudaSuccess) {
+        *ctx->timeout_flag = 0;
+    } else {
+        cudaGetLastError();
+        ctx->timeout_flag = nullptr;                       // the tcgen05 prefill kernel is then not used
+    }
     for (int i = 0; i < kTimingSlots; ++i) {
         if (cudaEventCreate(&ctx->ev0[i]) != cudaSuccess || cudaEventCreate(&ctx->ev1[i]) != cudaSuccess) {
             cudaGetLastError();
@@ -266,6 +272,7 @@ void lookat_destroy(lookat_ctx *handle)
                     ctx->step_q,  ctx->step_k,  ctx->step_out};
     for (void *p : bufs)
         if (p) cudaFree(p);
+    if (ctx->timeout_flag) cudaFreeHost(ctx->timeout_flag);
     for (int i = 0; i < kTimingSlots; ++i) {
         if (ctx->ev0[i]) cudaEventDestroy(ctx->ev0[i]);
         if (ctx->ev1[i]) cudaEventDestroy(ctx->ev1[i]);
@@ -288,7 +295,8 @@ lookat_status lookat_set_prefill_form(lookat_ctx *handle, int32_t form)
 {
     if (!handle) return LOOKAT_ERR_INVALID_ARG;
     Ctx *ctx = reinterpret_cast<Ctx *>(handle);
-    if (form != LOOKAT_PREFILL_AUTO && form != LOOKAT_PREFILL_TABLES && form != LOOKAT_PREFILL_CONTRACTION)
+    if (form != LOOKAT_PREFILL_AUTO && form != LOOKAT_PREFILL_TABLES && form != LOOKAT_PREFILL_CONTRACTION &&
+        form != LOOKAT_PREFILL_CONTRACTION_MMA_SYNC)
         return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "set_prefill_form: unknown form %d", (int)form);
     ctx->prefill_form = form;
     return LOOKAT_OK;
@@ -424,6 +432,11 @@ lookat_status lookat_attend_prefill(lookat_ctx *handle, const void *q, const flo
     if (!handle) return LOOKAT_ERR_INVALID_ARG;
     Ctx *ctx = reinterpret_cast<Ctx *>(handle);
     const lookat_config &c = ctx->cfg;
+    if (ctx->timeout_flag && *(volatile int *)ctx->timeout_flag) {
+        *(volatile int *)ctx->timeout_flag = 0;
+        return set_error(ctx, LOOKAT_ERR_TIMEOUT,
+                         "an earlier attend_prefill kernel gave up a bounded barrier wait; its output is not valid");
+    }
     if (B < 1 || B > 65535) return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "B=%d out of range 1..65535", B);
     if (c.n_q_heads > 65535) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "more than 65535 query heads");
     if (L_q < 1 || L_max < 1 || q_pos0 < 0 || q_pos0 + L_q > L_max || L_max > (1ll << 30))

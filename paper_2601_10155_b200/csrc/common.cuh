@@ -20,6 +20,7 @@ struct Ctx {
     int sm_count;
     int max_smem_optin;
     int prefill_form;          // LOOKAT_PREFILL_*
+    int *timeout_flag;         // pinned, device-visible: set by a kernel whose bounded barrier wait ran out
     float scale;           // resolved softmax scale
     char err[512];
     uint64_t launches;
@@ -117,6 +118,9 @@ lookat_status launch_prefill(Ctx *ctx, const PrefillArgs &a);
 // contraction form (prefill_mma.cu): centroids gathered per chunk, scores on the tensor cores
 bool prefill_mma_covers(const Ctx *ctx, const PrefillArgs &a);
 lookat_status launch_prefill_mma(Ctx *ctx, const PrefillArgs &a);
+// the same on tcgen05 with accumulators in tensor memory (prefill_umma.cu)
+bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a);
+lookat_status launch_prefill_umma(Ctx *ctx, const PrefillArgs &a);
 
 lookat_status launch_build_lut(Ctx *ctx, const __half *q, int B, const float *codebooks, float *lut);
 

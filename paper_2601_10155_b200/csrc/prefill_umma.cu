@@ -1,0 +1,454 @@
+// Multi-query causal attention over the compressed keys, contraction form, on the 5th-generation tensor
+// cores (Algorithm 1 applied to a tile of 128 queries).  The score of Section 3.4,
+//     s[q][t] = sum_j LUT_j[code[t][j]],   LUT_j[c] = q^(j) . C_j[c],
+// is the inner product of q with the key rebuilt from its codes, k^[t] = (C_1[code[t][1]], ...,
+// C_m[code[t][m]]).  A table pays when one query meets many keys; in prefill many queries meet each key,
+// so the centroids named by a chunk of 64 tokens are gathered ONCE per CTA into shared memory (the codes
+// stay the only stored form of the keys; nothing is written back to HBM) and all 128 queries take their
+// scores from them with tcgen05.mma: S = Q . K^^T (fp32 in tensor memory), online softmax by one thread
+// per query row, O += P . V with P read from tensor memory.  q (fp16) is an exact operand; every fp32
+// centroid is split into two fp16 planes (rounding + remainder), which carries s to ~2^-22 relative.
+//
+// Roles in a CTA of 9 warps (one CTA per SM; the shared memory is full):
+//   warps 0-3  softmax: thread r owns query row r = tensor-memory lane r;
+//   warps 4-7  producers: rebuild the next chunk's key rows from the codebook image in shared memory
+//              (16-byte items placed so that gathers and stores are free of bank conflicts whatever
+//              the codes are) and fetch its V rows with cp.async;
+//   warp 8     one thread issues every MMA and commits them to mbarriers.
+// Hand-offs go through mbarriers, one per buffer where a buffer is reused, so that no waiter can fall
+// two phases behind; every wait gives up after a bounded number of polls, raises the context's timeout
+// flag and lets the CTA drain and free its tensor memory.
+#include "common.cuh"
+
+namespace lookat {
+
+namespace {
+
+constexpr int kUmRows = 128;                   // queries per CTA = rows of one MMA
+constexpr int kUmChunk = 64;                   // tokens per chunk = columns of the score MMA
+constexpr int kUmSoftmax = 128, kUmProducers = 128;
+constexpr int kUmThreads = kUmSoftmax + kUmProducers + 32;
+constexpr int kUmPolls = 1 << 20;              // bound of every mbarrier wait
+
+__device__ __forceinline__ uint32_t um_smem(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void um_bar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void um_bar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// false after kUmPolls unsuccessful polls
+__device__ __forceinline__ bool um_bar_wait(uint32_t bar, uint32_t parity)
+{
+    for (int it = 0; it < kUmPolls; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void um_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void um_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void um_fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Shared-memory operand descriptor: 128-byte swizzle, start address / leading / stride offsets in 16-byte units.
+__device__ __forceinline__ uint64_t um_desc(uint32_t addr, uint32_t lead_bytes, uint32_t stride_bytes)
+{
+    return (uint64_t)((addr >> 4) & 0x3fff) | ((uint64_t)((lead_bytes >> 4) & 0x3fff) << 16) |
+           ((uint64_t)((stride_bytes >> 4) & 0x3fff) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void um_mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+        "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void um_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void um_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void um_cp_async16(unsigned dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
+// 32 consecutive 32-bit columns of this thread's tensor-memory lane
+__device__ __forceinline__ void um_ld32(uint32_t (&r)[32], uint32_t taddr)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void um_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(
+            taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+        "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+        "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),
+        "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void um_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory image of one head's codebooks as two fp16 planes, hi = fp16(c), lo = fp16(c - hi):
+// halfs [plane][d_k/64][K][8 pieces][8]: the 16-byte piece of 8-dim group gi sits in bank group gi mod 8.
+__global__ void um_codebook_image_kernel(const float *__restrict__ books, __half *__restrict__ images, int H_kv, int m, int K,
+                                         int d_sub)
+{
+    const int d_k = m * d_sub;
+    const size_t n = (size_t)H_kv * K * d_k;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int e = (int)(i % d_sub), c = (int)(i / d_sub % K), j = (int)(i / ((size_t)d_sub * K) % m);
+        const int h = (int)(i / ((size_t)d_sub * K * m));
+        const int dim = j * d_sub + e, gi = dim >> 3, blocks = d_k / 64;
+        const float v = books[i];
+        const __half hi = __float2half_rn(v), lo = __float2half_rn(v - __half2float(hi));
+        __half *img = images + (size_t)h * K * d_k * 2;
+        const size_t at = (((size_t)(gi >> 3) * K + c) * 8 + (gi & 7)) * 8 + (dim & 7);
+        img[at] = hi;
+        img[at + (size_t)blocks * K * 64] = lo;
+    }
+}
+
+template <int D_K, int D_V>
+struct UmLayout {
+    static constexpr int kKb = D_K / 64, kNb = D_V / 64;               // 128-byte blocks per key row / V row
+    static constexpr int kQ = kKb * kUmRows * 128;                     // [kb][128 rows][128 B]
+    static constexpr int kPlane = kKb * kUmChunk * 128;                // [kb][64 tokens][128 B]
+    static constexpr int kV = kNb * kUmChunk * 128;                    // [nb][64 tokens][128 B]
+    static constexpr int kOffKhi = kQ, kOffKlo = kQ + kPlane, kOffV = kQ + 2 * kPlane, kOffBook = kOffV + 2 * kV;
+    static constexpr int kIds = D_K / 4;                               // 16-byte items per key row, both planes
+    static constexpr int kItems = kUmChunk * kIds / kUmProducers;      // items rebuilt per producer thread per chunk
+    static constexpr int kVPieces = kUmChunk * (D_V / 8) / kUmProducers;
+    static_assert(kUmChunk * kIds % kUmProducers == 0 && kItems % 4 == 0, "whole items per thread, four codes per word");
+    static size_t book_bytes(int K) { return (size_t)K * D_K * 4; }
+    // operands, codebook image, then barriers and the tensor-memory address; 1 KB of slack to align the base
+    static size_t bytes(int K) { return (size_t)kOffBook + book_bytes(K) + 128 + 1024; }
+    static constexpr int kTmemCols = 256;                              // S0, S1: 64 each; O: D_V
+    static constexpr uint32_t kIdescS = (1u << 4) | ((uint32_t)(kUmChunk >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
+    static constexpr uint32_t kIdescO = (1u << 4) | (1u << 16) | ((uint32_t)(D_V >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
+};
+
+template <int D_K, int D_V, bool SCORES>
+__global__ void __launch_bounds__(kUmThreads, 1)
+attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int *__restrict__ timeout_flag)
+{
+    using Lay = UmLayout<D_K, D_V>;
+    extern __shared__ __align__(1024) unsigned char um_raw[];
+    unsigned char *const sm = um_raw + ((1024u - (um_smem(um_raw) & 1023u)) & 1023u);   // operands want 1024-byte alignment
+    const uint32_t sm0 = um_smem(sm);
+    const uint32_t book_bytes = (uint32_t)a.K * D_K * 4;
+    unsigned char *const book = sm + Lay::kOffBook;
+    uint64_t *const bars = reinterpret_cast<uint64_t *>(book + book_bytes);
+    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(bars + 8);
+    // barriers: 0 kv_ready; 1,2 s_full[buf]; 3,4 pv_done[buf]; 5 p_ready
+    const uint32_t bar0 = um_smem(bars);
+    const uint32_t bar_kv = bar0, bar_s = bar0 + 8, bar_pv = bar0 + 24, bar_p = bar0 + 40;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_tiles = (int)((a.L_q + kUmRows - 1) / kUmRows);
+    const int tile = n_tiles - 1 - (int)blockIdx.x;            // longest tiles first
+    const int hq = blockIdx.y, b = blockIdx.z, h = hq / a.g;
+    const int d_sub = D_K / a.m;
+
+    const long long row0 = (long long)tile * kUmRows;
+    const long long t_end = a.q_pos0 + (row0 + kUmRows < a.L_q ? row0 + kUmRows : a.L_q);   // tokens the tile sees
+    const int n_chunks = (int)((t_end + kUmChunk - 1) / kUmChunk);
+
+    // ---- prologue, all threads: codebook image and Q tile into shared memory, barriers, tensor memory ----
+    {
+        const unsigned char *img = reinterpret_cast<const unsigned char *>(images) + (size_t)h * book_bytes;
+        for (uint32_t i = tid * 16; i < book_bytes; i += kUmThreads * 16) um_cp_async16(sm0 + Lay::kOffBook + i, img + i);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        const __half *qb = a.q + (size_t)(b * a.H_q + hq) * a.L_q * D_K;
+        for (int p = tid; p < kUmRows * (D_K / 8); p += kUmThreads) {
+            const int r = p / (D_K / 8), pc = p % (D_K / 8);
+            const long long qr = row0 + r < a.L_q ? row0 + r : a.L_q - 1;      // rows beyond L_q repeat the last one
+            *reinterpret_cast<uint4 *>(sm + (pc >> 3) * (kUmRows * 128) + r * 128 + (((pc & 7) ^ (r & 7)) << 4)) =
+                *reinterpret_cast<const uint4 *>(qb + (size_t)qr * D_K + pc * 8);
+        }
+        if (tid == 0) {
+            um_bar_init(bar_kv, kUmProducers);
+            um_bar_init(bar_s, 1);
+            um_bar_init(bar_s + 8, 1);
+            um_bar_init(bar_pv, 1);
+            um_bar_init(bar_pv + 8, 1);
+            um_bar_init(bar_p, kUmSoftmax);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        if (warp == 0) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(um_smem(tmem_slot)),
+                         "n"(Lay::kTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        um_fence_async_smem();
+        um_fence_before();
+        __syncthreads();
+        um_fence_after();
+    }
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tm_s = tmem, tm_o = tmem + 2 * kUmChunk;    // columns: S0 | S1 | O
+    bool dead = false;                                         // a wait ran out: leave the loops, free, return
+
+    if (warp >= 8) {
+        // =================== the MMA thread ===================
+        if (lane == 0) {
+            auto value_mma = [&](int c) {                      // O += P(c) . V(c), P read from the S columns of its buffer
+                const int buf = c & 1;
+#pragma unroll
+                for (int kt = 0; kt < kUmChunk / 16; ++kt)
+                    um_mma_ts(tm_o, tm_s + buf * kUmChunk + kt * 8,
+                              um_desc(sm0 + Lay::kOffV + buf * Lay::kV + kt * 2048, kUmChunk * 128, 1024), Lay::kIdescO,
+                              (c > 0 || kt > 0) ? 1u : 0u);
+                um_commit(bar_pv + 8 * buf);
+            };
+            for (int c = 0; c < n_chunks && !dead; ++c) {
+                if (!um_bar_wait(bar_kv, c & 1)) { dead = true; break; }
+                um_fence_after();
+                const int buf = c & 1;
+#pragma unroll
+                for (int plane = 0; plane < 2; ++plane)
+#pragma unroll
+                    for (int ks = 0; ks < D_K / 16; ++ks) {
+                        const uint32_t off = (ks >> 2) * (kUmRows * 128) + (ks & 3) * 32;
+                        const uint32_t offk = (plane ? Lay::kOffKlo : Lay::kOffKhi) + (ks >> 2) * (kUmChunk * 128) + (ks & 3) * 32;
+                        um_mma_ss(tm_s + buf * kUmChunk, um_desc(sm0 + off, 16, 1024), um_desc(sm0 + offk, 16, 1024), Lay::kIdescS,
+                                  (plane | ks) ? 1u : 0u);
+                    }
+                um_commit(bar_s + 8 * buf);
+                if (c >= 1) {
+                    if (!um_bar_wait(bar_p, (c - 1) & 1)) { dead = true; break; }
+                    um_fence_after();
+                    value_mma(c - 1);
+                }
+            }
+            if (!dead) {
+                if (um_bar_wait(bar_p, (n_chunks - 1) & 1)) {
+                    um_fence_after();
+                    value_mma(n_chunks - 1);
+                } else {
+                    dead = true;
+                }
+            }
+        }
+    } else if (warp >= 4) {
+        // =================== producers ===================
+        const int ptid = tid - kUmSoftmax;
+        const uint8_t *codes = a.codes + (size_t)(b * a.H_kv + h) * a.L_max * a.m;
+        const __half *vsrc = a.v + (size_t)(b * a.H_kv + h) * a.L_max * D_V;
+        // item p = ptid + i * producers of a chunk: token p / kIds, id = p % kIds = plane * (D_K/8) + gi (fixed per thread)
+        const int my_id = ptid % Lay::kIds, my_plane = my_id / (D_K / 8), my_gi = my_id % (D_K / 8);
+        const int my_j = (my_gi * 8) / d_sub;
+        const uint32_t my_src = (uint32_t)my_plane * (book_bytes / 2) + (uint32_t)(my_gi >> 3) * a.K * 128 + ((my_gi & 7) << 4);
+        const uint32_t my_dst = (my_plane ? Lay::kOffKlo : Lay::kOffKhi) + (my_gi >> 3) * (kUmChunk * 128);
+        uint32_t cd[Lay::kItems / 4];                          // this thread's codes of one chunk, four per word
+        auto load_codes = [&](int c) {
+#pragma unroll
+            for (int i = 0; i < Lay::kItems; ++i) {
+                const long long tok = (long long)c * kUmChunk + (ptid + i * kUmProducers) / Lay::kIds;
+                const uint32_t code = tok < t_end ? (uint32_t)codes[(size_t)tok * a.m + my_j] : 0u;
+                cd[i >> 2] = (i & 3) ? (cd[i >> 2] | (code << (8 * (i & 3)))) : code;
+            }
+        };
+        load_codes(0);
+        for (int c = 0; c < n_chunks; ++c) {
+            const int buf = c & 1;
+            if (c >= 2 && !um_bar_wait(bar_pv + 8 * buf, ((c - 2) >> 1) & 1)) { dead = true; break; }   // V buffer is free
+            // V rows by cp.async: [nb][token][128 B], 16-byte pieces swizzled by token
+#pragma unroll
+            for (int i = 0; i < Lay::kVPieces; ++i) {
+                const int p = ptid + i * kUmProducers, tl = p / (D_V / 8), pc = p % (D_V / 8);
+                const long long tok = (long long)c * kUmChunk + tl;
+                const uint32_t off = Lay::kOffV + buf * Lay::kV + (pc >> 3) * (kUmChunk * 128) + tl * 128 + (((pc & 7) ^ (tl & 7)) << 4);
+                if (tok < t_end)
+                    um_cp_async16(sm0 + off, vsrc + (size_t)tok * D_V + pc * 8);
+                else
+                    *reinterpret_cast<uint4 *>(sm + off) = make_uint4(0u, 0u, 0u, 0u);
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            if (c >= 1 && !um_bar_wait(bar_s + 8 * (buf ^ 1), ((c - 1) >> 1) & 1)) { dead = true; break; }   // key buffer is free
+            // key rows: one 16-byte item of the codebook image per (token, 8-dim group, plane)
+#pragma unroll
+            for (int i = 0; i < Lay::kItems; ++i) {
+                const int tl = (ptid + i * kUmProducers) / Lay::kIds;
+                const uint32_t code = (cd[i >> 2] >> (8 * (i & 3))) & 0xffu;
+                uint4 item = make_uint4(0u, 0u, 0u, 0u);
+                if ((long long)c * kUmChunk + tl < t_end) item = *reinterpret_cast<const uint4 *>(book + my_src + code * 128);
+                *reinterpret_cast<uint4 *>(sm + my_dst + tl * 128 + (((my_gi & 7) ^ (tl & 7)) << 4)) = item;
+            }
+            if (c + 1 < n_chunks) load_codes(c + 1);           // lands while this chunk is consumed
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            um_fence_async_smem();                             // generic-proxy writes before the MMA's reads
+            um_bar_arrive(bar_kv);
+        }
+    } else {
+        // =================== softmax: thread r owns query row r (tensor-memory lane r) ===================
+        const long long row = row0 + tid;
+        const long long vis_end = a.q_pos0 + (row < a.L_q ? row : a.L_q - 1) + 1;    // tokens this row sees
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        float m_run = -INFINITY, l_run = 0.f;                  // running maximum (base-2 exponent units) and row sum
+        for (int c = 0; c < n_chunks; ++c) {
+            const int buf = c & 1;
+            const long long tok0 = (long long)c * kUmChunk;
+            if (!um_bar_wait(bar_s + 8 * buf, (c >> 1) & 1)) { dead = true; break; }
+            um_fence_after();
+            uint32_t s0[32], s1[32];
+            um_ld32(s0, tm_s + buf * kUmChunk + lane_base);
+            um_ld32(s1, tm_s + buf * kUmChunk + 32 + lane_base);
+            if (SCORES && a.scores_out && row < a.L_q) {
+                float *dst = a.scores_out + ((size_t)(b * a.H_q + hq) * a.L_q + row) * a.L_max + tok0;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    if (tok0 + i < vis_end) dst[i] = __uint_as_float(s0[i]);
+                    if (tok0 + 32 + i < vis_end) dst[32 + i] = __uint_as_float(s1[i]);
+                }
+            }
+            // the scale is positive, so the maximum can be taken on the raw scores
+            float mx = -INFINITY;
+            if (tok0 + kUmChunk > vis_end) {                   // the chunk crosses this row's causal limit
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    if (tok0 + i >= vis_end) s0[i] = 0xff800000u;
+                    if (tok0 + 32 + i >= vis_end) s1[i] = 0xff800000u;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
+            const float m_new = fmaxf(m_run, mx * a.scale_log2);   // finite from chunk 0 on: token 0 is visible to every row
+            const float alpha = ex2_approx(m_run - m_new);
+            m_run = m_new;
+            // weights, rounded to fp16 once; the row sum uses the rounded values, as the MMA does
+            uint32_t pk[32];
+            float sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float p0 = ex2_approx(fmaf(__uint_as_float(s0[2 * i]), a.scale_log2, -m_new));
+                const float p1 = ex2_approx(fmaf(__uint_as_float(s0[2 * i + 1]), a.scale_log2, -m_new));
+                const float p2 = ex2_approx(fmaf(__uint_as_float(s1[2 * i]), a.scale_log2, -m_new));
+                const float p3 = ex2_approx(fmaf(__uint_as_float(s1[2 * i + 1]), a.scale_log2, -m_new));
+                const __half2 h01 = __floats2half2_rn(p0, p1), h23 = __floats2half2_rn(p2, p3);
+                pk[i] = *reinterpret_cast<const uint32_t *>(&h01);
+                pk[16 + i] = *reinterpret_cast<const uint32_t *>(&h23);
+                const float2 b01 = __half22float2(h01), b23 = __half22float2(h23);
+                sum += (b01.x + b01.y) + (b23.x + b23.y);
+            }
+            l_run = l_run * alpha + sum;
+            if (c >= 1) {
+                // the previous value MMA must be done before O is rescaled (and it has consumed the other P buffer)
+                if (!um_bar_wait(bar_pv + 8 * (buf ^ 1), ((c - 1) >> 1) & 1)) { dead = true; break; }
+                um_fence_after();
+                if (__any_sync(0xffffffffu, alpha != 1.f)) {   // a maximum moved in this warp's rows: rescale them
+#pragma unroll 1
+                    for (int part = 0; part < D_V / 32; ++part) {
+                        uint32_t o[32];
+                        um_ld32(o, tm_o + part * 32 + lane_base);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        um_st32(tm_o + part * 32 + lane_base, o);
+                    }
+                }
+            }
+            um_st32(tm_s + buf * kUmChunk + lane_base, pk);    // P over the first half of the S columns, two per column
+            um_wait_st();
+            um_fence_before();
+            um_bar_arrive(bar_p);
+        }
+        if (!dead && um_bar_wait(bar_pv + 8 * ((n_chunks - 1) & 1), ((n_chunks - 1) >> 1) & 1)) {
+            um_fence_after();
+            const float inv = 1.f / l_run;
+#pragma unroll 1
+            for (int part = 0; part < D_V / 32; ++part) {
+                uint32_t o[32];
+                um_ld32(o, tm_o + part * 32 + lane_base);
+                if (row < a.L_q) {
+                    float4 *dst = reinterpret_cast<float4 *>(a.out + ((size_t)(b * a.H_q + hq) * a.L_q + row) * D_V + part * 32);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        dst[i] = make_float4(__uint_as_float(o[4 * i]) * inv, __uint_as_float(o[4 * i + 1]) * inv,
+                                             __uint_as_float(o[4 * i + 2]) * inv, __uint_as_float(o[4 * i + 3]) * inv);
+                }
+            }
+        } else {
+            dead = true;
+        }
+    }
+
+    if (dead) atomicExch(timeout_flag, 1);
+    um_fence_before();
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(Lay::kTmemCols) : "memory");
+}
+
+template <int D_K, int D_V>
+lookat_status launch_um(Ctx *ctx, const PrefillArgs &a)
+{
+    using Lay = UmLayout<D_K, D_V>;
+    // the codebooks as shared-memory images of two fp16 planes, rewritten at every call (the caller may have refitted them)
+    const size_t elems = (size_t)a.H_kv * a.K * a.d_k;
+    lookat_status st = ensure(ctx, (void **)&ctx->split_books, &ctx->split_cap, 2 * elems * sizeof(__half), "codebook planes");
+    if (st != LOOKAT_OK) return st;
+    um_codebook_image_kernel<<<(unsigned)((elems + 1023) / 1024), 256, 0, ctx->stream>>>(a.codebooks, ctx->split_books, a.H_kv,
+                                                                                         a.m, a.K, a.d_k / a.m);
+    st = check_launch(ctx, "um_codebook_image_kernel");
+    if (st != LOOKAT_OK) return st;
+
+    const int n_tiles = (int)((a.L_q + kUmRows - 1) / kUmRows);
+    const int smem = (int)Lay::bytes(a.K);
+    dim3 grid((unsigned)n_tiles, (unsigned)a.H_q, (unsigned)a.B);
+    auto launch = [&](auto kern) -> lookat_status {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+            return check_launch(ctx, "prefill (tcgen05 form): shared-memory opt-in");
+        kern<<<grid, kUmThreads, smem, ctx->stream>>>(a, ctx->split_books, ctx->timeout_flag);
+        return check_launch(ctx, "attend_prefill_umma_kernel");
+    };
+    if (a.scores_out) return launch(attend_prefill_umma_kernel<D_K, D_V, true>);
+    return launch(attend_prefill_umma_kernel<D_K, D_V, false>);
+}
+
+}  // namespace
+
+bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a)
+{
+    const int d_sub = a.d_k / a.m;
+    const bool shape = (a.d_k == 64 || a.d_k == 128) && (a.d_v == 64 || a.d_v == 128) && d_sub % 8 == 0;
+    const bool aligned = ((uintptr_t)a.q & 15) == 0 && ((uintptr_t)a.v & 15) == 0;
+    // the row maxima are taken on the raw scores, which needs a positive softmax scale
+    if (!shape || !aligned || a.H_q > 65535 || a.B > 65535 || !(a.scale_log2 > 0.f) || !ctx->timeout_flag) return false;
+    const size_t operands = (size_t)kUmRows * a.d_k * 2 + 2 * (size_t)kUmChunk * a.d_k * 2 + 2 * (size_t)kUmChunk * a.d_v * 2;
+    return operands + (size_t)a.K * a.d_k * 4 + 128 + 1024 <= (size_t)ctx->max_smem_optin;
+}
+
+lookat_status launch_prefill_umma(Ctx *ctx, const PrefillArgs &a)
+{
+    if (a.d_k == 128) return a.d_v == 128 ? launch_um<128, 128>(ctx, a) : launch_um<128, 64>(ctx, a);
+    return a.d_v == 128 ? launch_um<64, 128>(ctx, a) : launch_um<64, 64>(ctx, a);
+}
+
+}  // namespace lookat

@@ -407,7 +407,7 @@ def test_invalid_arguments_are_rejected_without_launching():
     (dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=64, m=16, K=256, L=90), 90, 0),       # d_sub 4: tables only
 ])
 @pytest.mark.parametrize("q_scale", [1.0, 0.1])
-@pytest.mark.parametrize("form", ["tables", "contraction"])
+@pytest.mark.parametrize("form", ["tables", "contraction", "contraction_mma_sync"])
 def test_attend_prefill_matches_oracle(shape, L_q, q_pos0, q_scale, form):
     w = synth.small_workload(**shape)
     keys, v = synth.make_keys(w), synth.make_values(w)
@@ -418,7 +418,7 @@ def test_attend_prefill_matches_oracle(shape, L_q, q_pos0, q_scale, form):
     lk.lookat_set_prefill_form(form)
     scores = torch.full((w.B, w.n_q_heads, L_q, w.L), float("nan"), device="cuda")
     covered = w.d_k in (64, 128) and w.d_v in (64, 128) and w.d_sub % 8 == 0
-    if form == "contraction" and not covered:
+    if form != "tables" and not covered:
         with pytest.raises(LookatError):
             lk.lookat_attend_prefill(dev(q), dev(books), dev(codes), dev(v), q_pos0=q_pos0, scores_out=scores)
         return
