@@ -54,6 +54,17 @@ __device__ __forceinline__ bool um_bar_wait(uint32_t bar, uint32_t parity)
     }
     return false;
 }
+// One thread polls, the named barrier hands its verdict to all producers: nobody leaves a loop alone.
+__device__ __forceinline__ bool um_producers_wait(bool poller, uint32_t bar, uint32_t parity)
+{
+    const uint32_t failed = poller ? (um_bar_wait(bar, parity) ? 0u : 1u) : 0u;
+    uint32_t any;
+    asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, 1, %2, p;\nselp.u32 %0, 1, 0, q;\n}"
+                 : "=r"(any)
+                 : "r"(failed), "n"(kUmProducers)
+                 : "memory");
+    return any == 0;
+}
 __device__ __forceinline__ void um_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void um_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void um_fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -146,8 +157,8 @@ struct UmLayout {
     static constexpr int kVPieces = kUmChunk * (D_V / 8) / kUmProducers;
     static_assert(kUmChunk * kIds % kUmProducers == 0 && kItems % 4 == 0, "whole items per thread, four codes per word");
     static size_t book_bytes(int K) { return (size_t)K * D_K * 4; }
-    // operands, codebook image, then barriers and the tensor-memory address; 1 KB of slack to align the base
-    static size_t bytes(int K) { return (size_t)kOffBook + book_bytes(K) + 128 + 1024; }
+    // operands, codebook image, then barriers, the tensor-memory address and the codes of two chunks
+    static size_t bytes(int K) { return (size_t)kOffBook + book_bytes(K) + 64 + 2048; }
     static constexpr int kTmemCols = 256;                              // S0, S1: 64 each; O: D_V
     static constexpr uint32_t kIdescS = (1u << 4) | ((uint32_t)(kUmChunk >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
     static constexpr uint32_t kIdescO = (1u << 4) | (1u << 16) | ((uint32_t)(D_V >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
@@ -159,12 +170,13 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
 {
     using Lay = UmLayout<D_K, D_V>;
     extern __shared__ __align__(1024) unsigned char um_raw[];
-    unsigned char *const sm = um_raw + ((1024u - (um_smem(um_raw) & 1023u)) & 1023u);   // operands want 1024-byte alignment
+    unsigned char *const sm = um_raw;                          // operands want 1024-byte alignment (checked below)
     const uint32_t sm0 = um_smem(sm);
     const uint32_t book_bytes = (uint32_t)a.K * D_K * 4;
     unsigned char *const book = sm + Lay::kOffBook;
     uint64_t *const bars = reinterpret_cast<uint64_t *>(book + book_bytes);
-    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(bars + 8);
+    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(bars + 6);
+    uint8_t *const codes_s = reinterpret_cast<uint8_t *>(bars + 8);   // [2][1024]: the codes of two chunks
     // barriers: 0 kv_ready; 1,2 s_full[buf]; 3,4 pv_done[buf]; 5 p_ready
     const uint32_t bar0 = um_smem(bars);
     const uint32_t bar_kv = bar0, bar_s = bar0 + 8, bar_pv = bar0 + 24, bar_p = bar0 + 40;
@@ -214,9 +226,11 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
     }
     const uint32_t tmem = *tmem_slot;
     const uint32_t tm_s = tmem, tm_o = tmem + 2 * kUmChunk;    // columns: S0 | S1 | O
-    bool dead = false;                                         // a wait ran out: leave the loops, free, return
+    bool dead = (sm0 & 1023u) != 0;                            // a wait ran out (or the base is misaligned): leave, free, return
 
-    if (warp >= 8) {
+    if (dead) {
+        // misaligned shared-memory base: nothing runs
+    } else if (warp >= 8) {
         // =================== the MMA thread ===================
         if (lane == 0) {
             auto value_mma = [&](int c) {                      // O += P(c) . V(c), P read from the S columns of its buffer
@@ -265,47 +279,56 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         // item p = ptid + i * producers of a chunk: token p / kIds, id = p % kIds = plane * (D_K/8) + gi (fixed per thread)
         const int my_id = ptid % Lay::kIds, my_plane = my_id / (D_K / 8), my_gi = my_id % (D_K / 8);
         const int my_j = (my_gi * 8) / d_sub;
-        const uint32_t my_src = (uint32_t)my_plane * (book_bytes / 2) + (uint32_t)(my_gi >> 3) * a.K * 128 + ((my_gi & 7) << 4);
-        const uint32_t my_dst = (my_plane ? Lay::kOffKlo : Lay::kOffKhi) + (my_gi >> 3) * (kUmChunk * 128);
-        uint32_t cd[Lay::kItems / 4];                          // this thread's codes of one chunk, four per word
-        auto load_codes = [&](int c) {
-#pragma unroll
-            for (int i = 0; i < Lay::kItems; ++i) {
-                const long long tok = (long long)c * kUmChunk + (ptid + i * kUmProducers) / Lay::kIds;
-                const uint32_t code = tok < t_end ? (uint32_t)codes[(size_t)tok * a.m + my_j] : 0u;
-                cd[i >> 2] = (i & 3) ? (cd[i >> 2] | (code << (8 * (i & 3)))) : code;
-            }
+        const unsigned char *my_src = book + (uint32_t)my_plane * (book_bytes / 2) + (uint32_t)(my_gi >> 3) * a.K * 128 + ((my_gi & 7) << 4);
+        unsigned char *my_dst = sm + (my_plane ? Lay::kOffKlo : Lay::kOffKhi) + (my_gi >> 3) * (kUmChunk * 128);
+        const int tl0 = ptid / Lay::kIds;                      // this thread's tokens of a chunk: tl0 + i * (producers / kIds)
+        constexpr int kTokStep = kUmProducers / Lay::kIds;
+        const int code_bytes = kUmChunk * a.m;                 // codes of one chunk, staged in shared memory a chunk ahead
+        auto fetch_codes = [&](int c) {                        // 4-byte cp.async pieces; pieces beyond the tile's tokens stay unread
+            const long long first = (long long)c * code_bytes, limit = t_end * a.m;
+            for (int o = ptid * 4; o < code_bytes; o += kUmProducers * 4)
+                if (first + o + 4 <= limit)
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(um_smem(codes_s) + (c & 1) * 1024 + o),
+                                 "l"(codes + first + o)
+                                 : "memory");
         };
-        load_codes(0);
+        fetch_codes(0);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
-            if (c >= 2 && !um_bar_wait(bar_pv + 8 * buf, ((c - 2) >> 1) & 1)) { dead = true; break; }   // V buffer is free
-            // V rows by cp.async: [nb][token][128 B], 16-byte pieces swizzled by token
+            if (c >= 2 && !um_producers_wait(ptid == 0, bar_pv + 8 * buf, ((c - 2) >> 1) & 1)) { dead = true; break; }   // V buffer is free
+            // V rows by cp.async: [nb][token][128 B], 16-byte pieces swizzled by token; the next chunk's codes
+            const bool whole = (long long)(c + 1) * kUmChunk <= t_end;   // every token of the chunk is visible to the tile
 #pragma unroll
             for (int i = 0; i < Lay::kVPieces; ++i) {
                 const int p = ptid + i * kUmProducers, tl = p / (D_V / 8), pc = p % (D_V / 8);
-                const long long tok = (long long)c * kUmChunk + tl;
                 const uint32_t off = Lay::kOffV + buf * Lay::kV + (pc >> 3) * (kUmChunk * 128) + tl * 128 + (((pc & 7) ^ (tl & 7)) << 4);
-                if (tok < t_end)
-                    um_cp_async16(sm0 + off, vsrc + (size_t)tok * D_V + pc * 8);
+                if (whole || (long long)c * kUmChunk + tl < t_end)
+                    um_cp_async16(sm0 + off, vsrc + ((size_t)c * kUmChunk + tl) * D_V + pc * 8);
                 else
                     *reinterpret_cast<uint4 *>(sm + off) = make_uint4(0u, 0u, 0u, 0u);
             }
+            if (c + 1 < n_chunks) fetch_codes(c + 1);
             asm volatile("cp.async.commit_group;" ::: "memory");
-            if (c >= 1 && !um_bar_wait(bar_s + 8 * (buf ^ 1), ((c - 1) >> 1) & 1)) { dead = true; break; }   // key buffer is free
+            if (c >= 1 && !um_producers_wait(ptid == 0, bar_s + 8 * (buf ^ 1), ((c - 1) >> 1) & 1)) { dead = true; break; }   // key buffer is free
             // key rows: one 16-byte item of the codebook image per (token, 8-dim group, plane)
+            const uint8_t *cs = codes_s + buf * 1024 + my_j;
+            uint32_t code[Lay::kItems];
+#pragma unroll
+            for (int i = 0; i < Lay::kItems; ++i) code[i] = cs[(tl0 + i * kTokStep) * a.m];
 #pragma unroll
             for (int i = 0; i < Lay::kItems; ++i) {
-                const int tl = (ptid + i * kUmProducers) / Lay::kIds;
-                const uint32_t code = (cd[i >> 2] >> (8 * (i & 3))) & 0xffu;
+                const int tl = tl0 + i * kTokStep;
                 uint4 item = make_uint4(0u, 0u, 0u, 0u);
-                if ((long long)c * kUmChunk + tl < t_end) item = *reinterpret_cast<const uint4 *>(book + my_src + code * 128);
-                *reinterpret_cast<uint4 *>(sm + my_dst + tl * 128 + (((my_gi & 7) ^ (tl & 7)) << 4)) = item;
+                if (whole || (long long)c * kUmChunk + tl < t_end) item = *reinterpret_cast<const uint4 *>(my_src + code[i] * 128);
+                *reinterpret_cast<uint4 *>(my_dst + tl * 128 + (((my_gi & 7) ^ (tl & 7)) << 4)) = item;
             }
-            if (c + 1 < n_chunks) load_codes(c + 1);           // lands while this chunk is consumed
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             um_fence_async_smem();                             // generic-proxy writes before the MMA's reads
             um_bar_arrive(bar_kv);
+            asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");   // the next chunk's codes are visible to all producers
         }
     } else {
         // =================== softmax: thread r owns query row r (tensor-memory lane r) ===================
@@ -316,7 +339,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
             const long long tok0 = (long long)c * kUmChunk;
-            if (!um_bar_wait(bar_s + 8 * buf, (c >> 1) & 1)) { dead = true; break; }
+            if (!__all_sync(0xffffffffu, um_bar_wait(bar_s + 8 * buf, (c >> 1) & 1))) { dead = true; break; }   // warp-uniform
             um_fence_after();
             uint32_t s0[32], s1[32];
             um_ld32(s0, tm_s + buf * kUmChunk + lane_base);
@@ -361,7 +384,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             l_run = l_run * alpha + sum;
             if (c >= 1) {
                 // the previous value MMA must be done before O is rescaled (and it has consumed the other P buffer)
-                if (!um_bar_wait(bar_pv + 8 * (buf ^ 1), ((c - 1) >> 1) & 1)) { dead = true; break; }
+                if (!__all_sync(0xffffffffu, um_bar_wait(bar_pv + 8 * (buf ^ 1), ((c - 1) >> 1) & 1))) { dead = true; break; }
                 um_fence_after();
                 if (__any_sync(0xffffffffu, alpha != 1.f)) {   // a maximum moved in this warp's rows: rescale them
 #pragma unroll 1
@@ -379,7 +402,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             um_fence_before();
             um_bar_arrive(bar_p);
         }
-        if (!dead && um_bar_wait(bar_pv + 8 * ((n_chunks - 1) & 1), ((n_chunks - 1) >> 1) & 1)) {
+        if (!dead && __all_sync(0xffffffffu, um_bar_wait(bar_pv + 8 * ((n_chunks - 1) & 1), ((n_chunks - 1) >> 1) & 1))) {
             um_fence_after();
             const float inv = 1.f / l_run;
 #pragma unroll 1
@@ -438,11 +461,12 @@ bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a)
 {
     const int d_sub = a.d_k / a.m;
     const bool shape = (a.d_k == 64 || a.d_k == 128) && (a.d_v == 64 || a.d_v == 128) && d_sub % 8 == 0;
-    const bool aligned = ((uintptr_t)a.q & 15) == 0 && ((uintptr_t)a.v & 15) == 0;
+    const bool aligned = ((uintptr_t)a.q & 15) == 0 && ((uintptr_t)a.v & 15) == 0 && ((uintptr_t)a.codes & 3) == 0 &&
+                         (a.L_max * a.m) % 4 == 0;
     // the row maxima are taken on the raw scores, which needs a positive softmax scale
     if (!shape || !aligned || a.H_q > 65535 || a.B > 65535 || !(a.scale_log2 > 0.f) || !ctx->timeout_flag) return false;
     const size_t operands = (size_t)kUmRows * a.d_k * 2 + 2 * (size_t)kUmChunk * a.d_k * 2 + 2 * (size_t)kUmChunk * a.d_v * 2;
-    return operands + (size_t)a.K * a.d_k * 4 + 128 + 1024 <= (size_t)ctx->max_smem_optin;
+    return operands + (size_t)a.K * a.d_k * 4 + 64 + 2048 <= (size_t)ctx->max_smem_optin;
 }
 
 lookat_status launch_prefill_umma(Ctx *ctx, const PrefillArgs &a)
