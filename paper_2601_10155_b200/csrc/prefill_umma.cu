@@ -54,6 +54,16 @@ __device__ __forceinline__ bool um_bar_wait(uint32_t bar, uint32_t parity)
     }
     return false;
 }
+// one poll
+__device__ __forceinline__ bool um_bar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok)
+                 : "r"(bar), "r"(parity)
+                 : "memory");
+    return ok != 0;
+}
 // One thread polls, the named barrier hands its verdict to all producers: nobody leaves a loop alone.
 __device__ __forceinline__ bool um_producers_wait(bool poller, uint32_t bar, uint32_t parity)
 {
@@ -69,19 +79,6 @@ __device__ __forceinline__ void um_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void um_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void um_fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// Shared-memory operand descriptor: 128-byte swizzle, start address / leading / stride offsets in 16-byte units.
-__device__ __forceinline__ uint64_t um_desc(uint32_t addr, uint32_t lead_bytes, uint32_t stride_bytes)
-{
-    return (uint64_t)((addr >> 4) & 0x3fff) | ((uint64_t)((lead_bytes >> 4) & 0x3fff) << 16) |
-           ((uint64_t)((stride_bytes >> 4) & 0x3fff) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-__device__ __forceinline__ void um_mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
-        "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
 __device__ __forceinline__ void um_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
@@ -148,18 +145,20 @@ __global__ void um_codebook_image_kernel(const float *__restrict__ books, __half
 template <int D_K, int D_V>
 struct UmLayout {
     static constexpr int kKb = D_K / 64, kNb = D_V / 64;               // 128-byte blocks per key row / V row
-    static constexpr int kQ = kKb * kUmRows * 128;                     // [kb][128 rows][128 B]
     static constexpr int kPlane = kKb * kUmChunk * 128;                // [kb][64 tokens][128 B]
     static constexpr int kV = kNb * kUmChunk * 128;                    // [nb][64 tokens][128 B]
-    static constexpr int kOffKhi = kQ, kOffKlo = kQ + kPlane, kOffV = kQ + 2 * kPlane, kOffBook = kOffV + 2 * kV;
+    static constexpr int kKeys = 2 * kPlane;                           // hi plane, lo plane of one chunk
+    static constexpr int kOffKeys = 0, kOffV = 2 * kKeys, kOffBook = kOffV + 2 * kV;   // two key buffers, two V buffers
     static constexpr int kIds = D_K / 4;                               // 16-byte items per key row, both planes
     static constexpr int kItems = kUmChunk * kIds / kUmProducers;      // items rebuilt per producer thread per chunk
     static constexpr int kVPieces = kUmChunk * (D_V / 8) / kUmProducers;
     static_assert(kUmChunk * kIds % kUmProducers == 0 && kItems % 4 == 0, "whole items per thread, four codes per word");
     static size_t book_bytes(int K) { return (size_t)K * D_K * 4; }
     // operands, codebook image, then barriers, the tensor-memory address and the codes of two chunks
-    static size_t bytes(int K) { return (size_t)kOffBook + book_bytes(K) + 64 + 2048; }
-    static constexpr int kTmemCols = 256;                              // S0, S1: 64 each; O: D_V
+    static size_t bytes(int K) { return (size_t)kOffBook + book_bytes(K) + 128 + 2048; }
+    static constexpr int kColO = 2 * kUmChunk, kColQ = kColO + D_V;    // columns: S0, S1 (64 each) | O (D_V) | Q (D_K / 2)
+    static constexpr int kTmemCols = kColQ + D_K / 2 <= 256 ? 256 : 512;
+    // instruction descriptors: fp32 accumulate, fp16 operands, N >> 3 at bit 17, M >> 4 at bit 24; bit 16: B is MN-major
     static constexpr uint32_t kIdescS = (1u << 4) | ((uint32_t)(kUmChunk >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
     static constexpr uint32_t kIdescO = (1u << 4) | (1u << 16) | ((uint32_t)(D_V >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
 };
@@ -175,11 +174,11 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
     const uint32_t book_bytes = (uint32_t)a.K * D_K * 4;
     unsigned char *const book = sm + Lay::kOffBook;
     uint64_t *const bars = reinterpret_cast<uint64_t *>(book + book_bytes);
-    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(bars + 6);
-    uint8_t *const codes_s = reinterpret_cast<uint8_t *>(bars + 8);   // [2][1024]: the codes of two chunks
-    // barriers: 0 kv_ready; 1,2 s_full[buf]; 3,4 pv_done[buf]; 5 p_ready
+    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(bars + 8);
+    uint8_t *const codes_s = reinterpret_cast<uint8_t *>(bars + 16);  // [2][1024]: the codes of two chunks
+    // barriers, one per buffer: kv_ready[2] (keys and V staged), s_full[2] (scores done), pv_done[2] (value MMA done), p_ready[2]
     const uint32_t bar0 = um_smem(bars);
-    const uint32_t bar_kv = bar0, bar_s = bar0 + 8, bar_pv = bar0 + 24, bar_p = bar0 + 40;
+    const uint32_t bar_kv = bar0, bar_s = bar0 + 16, bar_pv = bar0 + 32, bar_p = bar0 + 48;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_tiles = (int)((a.L_q + kUmRows - 1) / kUmRows);
@@ -191,25 +190,18 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
     const long long t_end = a.q_pos0 + (row0 + kUmRows < a.L_q ? row0 + kUmRows : a.L_q);   // tokens the tile sees
     const int n_chunks = (int)((t_end + kUmChunk - 1) / kUmChunk);
 
-    // ---- prologue, all threads: codebook image and Q tile into shared memory, barriers, tensor memory ----
+    // ---- prologue, all threads: codebook image into shared memory, barriers, tensor memory ----
     {
         const unsigned char *img = reinterpret_cast<const unsigned char *>(images) + (size_t)h * book_bytes;
         for (uint32_t i = tid * 16; i < book_bytes; i += kUmThreads * 16) um_cp_async16(sm0 + Lay::kOffBook + i, img + i);
         asm volatile("cp.async.commit_group;" ::: "memory");
-        const __half *qb = a.q + (size_t)(b * a.H_q + hq) * a.L_q * D_K;
-        for (int p = tid; p < kUmRows * (D_K / 8); p += kUmThreads) {
-            const int r = p / (D_K / 8), pc = p % (D_K / 8);
-            const long long qr = row0 + r < a.L_q ? row0 + r : a.L_q - 1;      // rows beyond L_q repeat the last one
-            *reinterpret_cast<uint4 *>(sm + (pc >> 3) * (kUmRows * 128) + r * 128 + (((pc & 7) ^ (r & 7)) << 4)) =
-                *reinterpret_cast<const uint4 *>(qb + (size_t)qr * D_K + pc * 8);
-        }
         if (tid == 0) {
-            um_bar_init(bar_kv, kUmProducers);
-            um_bar_init(bar_s, 1);
-            um_bar_init(bar_s + 8, 1);
-            um_bar_init(bar_pv, 1);
-            um_bar_init(bar_pv + 8, 1);
-            um_bar_init(bar_p, kUmSoftmax);
+            for (int i = 0; i < 2; ++i) {
+                um_bar_init(bar_kv + 8 * i, kUmProducers);
+                um_bar_init(bar_s + 8 * i, 1);
+                um_bar_init(bar_pv + 8 * i, 1);
+                um_bar_init(bar_p + 8 * i, kUmSoftmax);
+            }
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         if (warp == 0) {
@@ -225,50 +217,80 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         um_fence_after();
     }
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tm_s = tmem, tm_o = tmem + 2 * kUmChunk;    // columns: S0 | S1 | O
+    const uint32_t tm_s = tmem, tm_o = tmem + Lay::kColO, tm_q = tmem + Lay::kColQ;   // columns: S0 | S1 | O | Q
     bool dead = (sm0 & 1023u) != 0;                            // a wait ran out (or the base is misaligned): leave, free, return
+
+    // ---- the query rows go to tensor memory as the A operand of the score MMA: lane r = row r, two halfs per column ----
+    if (warp < 4) {
+        const long long qr = row0 + tid < a.L_q ? row0 + tid : a.L_q - 1;       // rows beyond L_q repeat the last one
+        const uint4 *src = reinterpret_cast<const uint4 *>(a.q + ((size_t)(b * a.H_q + hq) * a.L_q + qr) * D_K);
+#pragma unroll
+        for (int part = 0; part < D_K / 64; ++part) {
+            uint32_t w[32];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint4 x = src[part * 8 + i];
+                w[4 * i] = x.x;
+                w[4 * i + 1] = x.y;
+                w[4 * i + 2] = x.z;
+                w[4 * i + 3] = x.w;
+            }
+            um_st32(tm_q + part * 32 + ((uint32_t)(warp * 32) << 16), w);
+        }
+        um_wait_st();
+    }
+    um_fence_before();
+    __syncthreads();
+    um_fence_after();
 
     if (dead) {
         // misaligned shared-memory base: nothing runs
     } else if (warp >= 8) {
         // =================== the MMA thread ===================
         if (lane == 0) {
+            // descriptors: only the start address (low word, 16-byte units) changes from one MMA to the next
+            const uint32_t hi_k = (1024u >> 4) | (1u << 14) | (2u << 29);   // stride 1024 B, version 1, 128-byte swizzle
+            auto desc = [&](uint32_t addr, uint32_t lead_bytes) -> uint64_t {
+                return ((uint64_t)hi_k << 32) | (uint64_t)(((addr >> 4) & 0x3fffu) | ((lead_bytes >> 4) << 16));
+            };
+            auto score_mma = [&](int c) {                      // S[c & 1] = Q . K^(c)^T, both planes
+                const int buf = c & 1;
+                const uint32_t keys = sm0 + Lay::kOffKeys + buf * Lay::kKeys;
+#pragma unroll
+                for (int plane = 0; plane < 2; ++plane)
+#pragma unroll
+                    for (int ks = 0; ks < D_K / 16; ++ks)
+                        um_mma_ts(tm_s + buf * kUmChunk, tm_q + ks * 8,
+                                  desc(keys + plane * Lay::kPlane + (ks >> 2) * (kUmChunk * 128) + (ks & 3) * 32, 16), Lay::kIdescS,
+                                  (plane | ks) ? 1u : 0u);
+                um_commit(bar_s + 8 * buf);
+            };
             auto value_mma = [&](int c) {                      // O += P(c) . V(c), P read from the S columns of its buffer
                 const int buf = c & 1;
 #pragma unroll
                 for (int kt = 0; kt < kUmChunk / 16; ++kt)
-                    um_mma_ts(tm_o, tm_s + buf * kUmChunk + kt * 8,
-                              um_desc(sm0 + Lay::kOffV + buf * Lay::kV + kt * 2048, kUmChunk * 128, 1024), Lay::kIdescO,
-                              (c > 0 || kt > 0) ? 1u : 0u);
+                    um_mma_ts(tm_o, tm_s + buf * kUmChunk + kt * 8, desc(sm0 + Lay::kOffV + buf * Lay::kV + kt * 2048, kUmChunk * 128),
+                              Lay::kIdescO, (c > 0 || kt > 0) ? 1u : 0u);
                 um_commit(bar_pv + 8 * buf);
             };
-            for (int c = 0; c < n_chunks && !dead; ++c) {
-                if (!um_bar_wait(bar_kv, c & 1)) { dead = true; break; }
-                um_fence_after();
-                const int buf = c & 1;
-#pragma unroll
-                for (int plane = 0; plane < 2; ++plane)
-#pragma unroll
-                    for (int ks = 0; ks < D_K / 16; ++ks) {
-                        const uint32_t off = (ks >> 2) * (kUmRows * 128) + (ks & 3) * 32;
-                        const uint32_t offk = (plane ? Lay::kOffKlo : Lay::kOffKhi) + (ks >> 2) * (kUmChunk * 128) + (ks & 3) * 32;
-                        um_mma_ss(tm_s + buf * kUmChunk, um_desc(sm0 + off, 16, 1024), um_desc(sm0 + offk, 16, 1024), Lay::kIdescS,
-                                  (plane | ks) ? 1u : 0u);
-                    }
-                um_commit(bar_s + 8 * buf);
-                if (c >= 1) {
-                    if (!um_bar_wait(bar_p, (c - 1) & 1)) { dead = true; break; }
+            // Whichever is ready goes first: the scores of chunk next_qk (its keys are staged and the value MMA
+            // that read the previous weights of that buffer has been issued) or the value MMA of chunk next_pv.
+            int next_qk = 0, next_pv = 0;
+            long long polls = 0;
+            while (next_pv < n_chunks) {
+                bool progress = false;
+                if (next_qk < n_chunks && next_qk - next_pv < 2 && um_bar_test(bar_kv + 8 * (next_qk & 1), (next_qk >> 1) & 1)) {
                     um_fence_after();
-                    value_mma(c - 1);
+                    score_mma(next_qk++);
+                    progress = true;
                 }
-            }
-            if (!dead) {
-                if (um_bar_wait(bar_p, (n_chunks - 1) & 1)) {
+                if (next_pv < next_qk && um_bar_test(bar_p + 8 * (next_pv & 1), (next_pv >> 1) & 1)) {
                     um_fence_after();
-                    value_mma(n_chunks - 1);
-                } else {
-                    dead = true;
+                    value_mma(next_pv++);
+                    progress = true;
                 }
+                if (progress) polls = 0;
+                else if (++polls > kUmPolls) { dead = true; break; }
             }
         }
     } else if (warp >= 4) {
@@ -280,7 +302,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         const int my_id = ptid % Lay::kIds, my_plane = my_id / (D_K / 8), my_gi = my_id % (D_K / 8);
         const int my_j = (my_gi * 8) / d_sub;
         const unsigned char *my_src = book + (uint32_t)my_plane * (book_bytes / 2) + (uint32_t)(my_gi >> 3) * a.K * 128 + ((my_gi & 7) << 4);
-        unsigned char *my_dst = sm + (my_plane ? Lay::kOffKlo : Lay::kOffKhi) + (my_gi >> 3) * (kUmChunk * 128);
+        unsigned char *my_dst = sm + Lay::kOffKeys + my_plane * Lay::kPlane + (my_gi >> 3) * (kUmChunk * 128);   // + buf * kKeys
         const int tl0 = ptid / Lay::kIds;                      // this thread's tokens of a chunk: tl0 + i * (producers / kIds)
         constexpr int kTokStep = kUmProducers / Lay::kIds;
         const int code_bytes = kUmChunk * a.m;                 // codes of one chunk, staged in shared memory a chunk ahead
@@ -298,7 +320,8 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
-            if (c >= 2 && !um_producers_wait(ptid == 0, bar_pv + 8 * buf, ((c - 2) >> 1) & 1)) { dead = true; break; }   // V buffer is free
+            // both buffers of chunk c - 2 are free once its value MMA is done (its score MMA was done before that)
+            if (c >= 2 && !um_producers_wait(ptid == 0, bar_pv + 8 * buf, ((c - 2) >> 1) & 1)) { dead = true; break; }
             // V rows by cp.async: [nb][token][128 B], 16-byte pieces swizzled by token; the next chunk's codes
             const bool whole = (long long)(c + 1) * kUmChunk <= t_end;   // every token of the chunk is visible to the tile
 #pragma unroll
@@ -312,7 +335,6 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             }
             if (c + 1 < n_chunks) fetch_codes(c + 1);
             asm volatile("cp.async.commit_group;" ::: "memory");
-            if (c >= 1 && !um_producers_wait(ptid == 0, bar_s + 8 * (buf ^ 1), ((c - 1) >> 1) & 1)) { dead = true; break; }   // key buffer is free
             // key rows: one 16-byte item of the codebook image per (token, 8-dim group, plane)
             const uint8_t *cs = codes_s + buf * 1024 + my_j;
             uint32_t code[Lay::kItems];
@@ -323,11 +345,11 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                 const int tl = tl0 + i * kTokStep;
                 uint4 item = make_uint4(0u, 0u, 0u, 0u);
                 if (whole || (long long)c * kUmChunk + tl < t_end) item = *reinterpret_cast<const uint4 *>(my_src + code[i] * 128);
-                *reinterpret_cast<uint4 *>(my_dst + tl * 128 + (((my_gi & 7) ^ (tl & 7)) << 4)) = item;
+                *reinterpret_cast<uint4 *>(my_dst + buf * Lay::kKeys + tl * 128 + (((my_gi & 7) ^ (tl & 7)) << 4)) = item;
             }
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             um_fence_async_smem();                             // generic-proxy writes before the MMA's reads
-            um_bar_arrive(bar_kv);
+            um_bar_arrive(bar_kv + 8 * buf);
             asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");   // the next chunk's codes are visible to all producers
         }
     } else {
@@ -400,7 +422,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             um_st32(tm_s + buf * kUmChunk + lane_base, pk);    // P over the first half of the S columns, two per column
             um_wait_st();
             um_fence_before();
-            um_bar_arrive(bar_p);
+            um_bar_arrive(bar_p + 8 * buf);
         }
         if (!dead && __all_sync(0xffffffffu, um_bar_wait(bar_pv + 8 * ((n_chunks - 1) & 1), ((n_chunks - 1) >> 1) & 1))) {
             um_fence_after();
