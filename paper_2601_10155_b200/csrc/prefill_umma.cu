@@ -9,16 +9,28 @@
 // per query row, O += P . V with P read from tensor memory.  q (fp16) is an exact operand; every fp32
 // centroid is split into two fp16 planes (rounding + remainder), which carries s to ~2^-22 relative.
 //
-// Roles in a CTA of 9 warps (one CTA per SM; the shared memory is full):
+// Roles in a CTA of 13 warps (one CTA per SM; the shared memory is full):
 //   warps 0-3  softmax: thread r owns query row r = tensor-memory lane r;
-//   warps 4-7  producers: rebuild the next chunk's key rows from the codebook image in shared memory
+//   warps 4-11 producers: rebuild the next chunk's key rows from the codebook image in shared memory
 //              (16-byte items placed so that gathers and stores are free of bank conflicts whatever
 //              the codes are) and fetch its V rows with cp.async;
-//   warp 8     one thread issues every MMA and commits them to mbarriers.
+//   warp 12    one thread issues every MMA and commits them to mbarriers.
 // Hand-offs go through mbarriers, one per buffer where a buffer is reused, so that no waiter can fall
 // two phases behind; every wait gives up after a bounded number of polls, raises the context's timeout
 // flag and lets the CTA drain and free its tensor memory.
 #include "common.cuh"
+
+// Tuning aid (-DLOOKAT_PHASE_STAMPS): per role, the cycles spent in each phase of the chunk loop, averaged
+// over the chunks of the first CTA and printed at its end.
+#ifdef LOOKAT_PHASE_STAMPS
+#include <cstdio>
+#define UM_STAMPS(name, n) long long name[n] = {}; long long um_tp_ = clock64();
+#define UM_STAMP(name, k) { const long long um_tn_ = clock64(); name[k] += um_tn_ - um_tp_; um_tp_ = um_tn_; }
+#define UM_FIRST_CTA (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+#else
+#define UM_STAMPS(name, n)
+#define UM_STAMP(name, k)
+#endif
 
 namespace lookat {
 
@@ -26,7 +38,7 @@ namespace {
 
 constexpr int kUmRows = 128;                   // queries per CTA = rows of one MMA
 constexpr int kUmChunk = 64;                   // tokens per chunk = columns of the score MMA
-constexpr int kUmSoftmax = 128, kUmProducers = 128;
+constexpr int kUmSoftmax = 128, kUmProducers = 256;
 constexpr int kUmThreads = kUmSoftmax + kUmProducers + 32;
 constexpr int kUmPolls = 1 << 20;              // bound of every mbarrier wait
 
@@ -79,11 +91,14 @@ __device__ __forceinline__ void um_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void um_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void um_fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-__device__ __forceinline__ void um_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate)
+// D (tensor memory) = or += A (tensor memory) . B (shared memory, descriptor given as its two words)
+template <bool ACCUMULATE>
+__device__ __forceinline__ void um_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc)
 {
     asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
-        "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate)
+        "{\n.reg .pred p;\n.reg .b64 bd;\nsetp.ne.b32 p, %5, 0;\nmov.b64 bd, {%2, %3};\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n}" ::"r"(d_tmem),
+        "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACCUMULATE ? 1 : 0)
         : "memory");
 }
 __device__ __forceinline__ void um_commit(uint32_t bar)
@@ -174,11 +189,12 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
     const uint32_t book_bytes = (uint32_t)a.K * D_K * 4;
     unsigned char *const book = sm + Lay::kOffBook;
     uint64_t *const bars = reinterpret_cast<uint64_t *>(book + book_bytes);
-    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(bars + 8);
+    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(bars + 12);
     uint8_t *const codes_s = reinterpret_cast<uint8_t *>(bars + 16);  // [2][1024]: the codes of two chunks
-    // barriers, one per buffer: kv_ready[2] (keys and V staged), s_full[2] (scores done), pv_done[2] (value MMA done), p_ready[2]
+    // barriers, one per buffer: k_ready[2], v_ready[2] (keys / V staged), s_full[2] (scores done), pv_done[2] (value MMA
+    // done), p_ready[2] (weights stored)
     const uint32_t bar0 = um_smem(bars);
-    const uint32_t bar_kv = bar0, bar_s = bar0 + 16, bar_pv = bar0 + 32, bar_p = bar0 + 48;
+    const uint32_t bar_k = bar0, bar_v = bar0 + 16, bar_s = bar0 + 32, bar_pv = bar0 + 48, bar_p = bar0 + 64;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_tiles = (int)((a.L_q + kUmRows - 1) / kUmRows);
@@ -197,7 +213,8 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         asm volatile("cp.async.commit_group;" ::: "memory");
         if (tid == 0) {
             for (int i = 0; i < 2; ++i) {
-                um_bar_init(bar_kv + 8 * i, kUmProducers);
+                um_bar_init(bar_k + 8 * i, kUmProducers);
+                um_bar_init(bar_v + 8 * i, kUmProducers);
                 um_bar_init(bar_s + 8 * i, 1);
                 um_bar_init(bar_pv + 8 * i, 1);
                 um_bar_init(bar_p + 8 * i, kUmSoftmax);
@@ -245,53 +262,66 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
 
     if (dead) {
         // misaligned shared-memory base: nothing runs
-    } else if (warp >= 8) {
+    } else if (warp >= (kUmSoftmax + kUmProducers) / 32) {
         // =================== the MMA thread ===================
         if (lane == 0) {
-            // descriptors: only the start address (low word, 16-byte units) changes from one MMA to the next
-            const uint32_t hi_k = (1024u >> 4) | (1u << 14) | (2u << 29);   // stride 1024 B, version 1, 128-byte swizzle
-            auto desc = [&](uint32_t addr, uint32_t lead_bytes) -> uint64_t {
-                return ((uint64_t)hi_k << 32) | (uint64_t)(((addr >> 4) & 0x3fffu) | ((lead_bytes >> 4) << 16));
-            };
+            // descriptors: stride 1024 B, version 1, 128-byte swizzle in the high word; the low word holds the start
+            // address and the leading offset (16-byte units) and is all that changes from one MMA to the next
+            const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+            const uint32_t keys_lo = ((sm0 + Lay::kOffKeys) >> 4) | (1u << 16);                    // leading offset unused (16 B)
+            const uint32_t v_lo = ((sm0 + Lay::kOffV) >> 4) | ((uint32_t)(kUmChunk * 128 / 16) << 16);   // between 64-column blocks
             auto score_mma = [&](int c) {                      // S[c & 1] = Q . K^(c)^T, both planes
                 const int buf = c & 1;
-                const uint32_t keys = sm0 + Lay::kOffKeys + buf * Lay::kKeys;
+                const uint32_t lo = keys_lo + buf * (Lay::kKeys >> 4), d = tm_s + buf * kUmChunk;
 #pragma unroll
                 for (int plane = 0; plane < 2; ++plane)
 #pragma unroll
-                    for (int ks = 0; ks < D_K / 16; ++ks)
-                        um_mma_ts(tm_s + buf * kUmChunk, tm_q + ks * 8,
-                                  desc(keys + plane * Lay::kPlane + (ks >> 2) * (kUmChunk * 128) + (ks & 3) * 32, 16), Lay::kIdescS,
-                                  (plane | ks) ? 1u : 0u);
+                    for (int ks = 0; ks < D_K / 16; ++ks) {
+                        const uint32_t off = (plane * Lay::kPlane + (ks >> 2) * (kUmChunk * 128) + (ks & 3) * 32) >> 4;
+                        if (plane == 0 && ks == 0) um_mma_ts<false>(d, tm_q + ks * 8, lo + off, desc_hi, Lay::kIdescS);
+                        else um_mma_ts<true>(d, tm_q + ks * 8, lo + off, desc_hi, Lay::kIdescS);
+                    }
                 um_commit(bar_s + 8 * buf);
             };
             auto value_mma = [&](int c) {                      // O += P(c) . V(c), P read from the S columns of its buffer
                 const int buf = c & 1;
+                const uint32_t lo = v_lo + buf * (Lay::kV >> 4), pa = tm_s + buf * kUmChunk;
 #pragma unroll
-                for (int kt = 0; kt < kUmChunk / 16; ++kt)
-                    um_mma_ts(tm_o, tm_s + buf * kUmChunk + kt * 8, desc(sm0 + Lay::kOffV + buf * Lay::kV + kt * 2048, kUmChunk * 128),
-                              Lay::kIdescO, (c > 0 || kt > 0) ? 1u : 0u);
+                for (int kt = 0; kt < kUmChunk / 16; ++kt) {   // 16 tokens: 8 columns of weights, two 8-token groups of V
+                    if (kt == 0 && c == 0) um_mma_ts<false>(tm_o, pa + kt * 8, lo + kt * (2048 >> 4), desc_hi, Lay::kIdescO);
+                    else um_mma_ts<true>(tm_o, pa + kt * 8, lo + kt * (2048 >> 4), desc_hi, Lay::kIdescO);
+                }
                 um_commit(bar_pv + 8 * buf);
             };
             // Whichever is ready goes first: the scores of chunk next_qk (its keys are staged and the value MMA
-            // that read the previous weights of that buffer has been issued) or the value MMA of chunk next_pv.
+            // that read the previous weights of that buffer has been issued) or the value MMA of chunk next_pv
+            // (its weights are stored and its V rows have landed).
             int next_qk = 0, next_pv = 0;
             long long polls = 0;
+            UM_STAMPS(mm, 3)
             while (next_pv < n_chunks) {
                 bool progress = false;
-                if (next_qk < n_chunks && next_qk - next_pv < 2 && um_bar_test(bar_kv + 8 * (next_qk & 1), (next_qk >> 1) & 1)) {
+                if (next_qk < n_chunks && next_qk - next_pv < 2 && um_bar_test(bar_k + 8 * (next_qk & 1), (next_qk >> 1) & 1)) {
+                    UM_STAMP(mm, 0)
                     um_fence_after();
                     score_mma(next_qk++);
                     progress = true;
+                    UM_STAMP(mm, 1)
                 }
-                if (next_pv < next_qk && um_bar_test(bar_p + 8 * (next_pv & 1), (next_pv >> 1) & 1)) {
+                if (next_pv < next_qk && um_bar_test(bar_p + 8 * (next_pv & 1), (next_pv >> 1) & 1) &&
+                    um_bar_test(bar_v + 8 * (next_pv & 1), (next_pv >> 1) & 1)) {
+                    UM_STAMP(mm, 0)
                     um_fence_after();
                     value_mma(next_pv++);
                     progress = true;
+                    UM_STAMP(mm, 2)
                 }
                 if (progress) polls = 0;
                 else if (++polls > kUmPolls) { dead = true; break; }
             }
+#ifdef LOOKAT_PHASE_STAMPS
+            if (UM_FIRST_CTA) printf("mma thread: idle %lld, score issue %lld, value issue %lld cycles per chunk\n", mm[0] / n_chunks, mm[1] / n_chunks, mm[2] / n_chunks);
+#endif
         }
     } else if (warp >= 4) {
         // =================== producers ===================
@@ -314,16 +344,45 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                                  "l"(codes + first + o)
                                  : "memory");
         };
+        // key rows of chunk c into key buffer c & 1: one 16-byte item of the codebook image per (token, 8-dim group, plane)
+        auto rebuild_keys = [&](int c) {
+            const int buf = c & 1;
+            const bool whole = (long long)(c + 1) * kUmChunk <= t_end;   // every token of the chunk is visible to the tile
+            const uint8_t *cs = codes_s + buf * 1024 + my_j;
+            uint32_t code[Lay::kItems];
+            uint4 item[Lay::kItems];
+#pragma unroll
+            for (int i = 0; i < Lay::kItems; ++i) code[i] = cs[(tl0 + i * kTokStep) * a.m];
+#pragma unroll
+            for (int i = 0; i < Lay::kItems; ++i) {            // all loads before any store: they overlap
+                item[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (whole || (long long)c * kUmChunk + tl0 + i * kTokStep < t_end)
+                    item[i] = *reinterpret_cast<const uint4 *>(my_src + code[i] * 128);
+            }
+#pragma unroll
+            for (int i = 0; i < Lay::kItems; ++i) {
+                const int tl = tl0 + i * kTokStep;
+                *reinterpret_cast<uint4 *>(my_dst + buf * Lay::kKeys + tl * 128 + (((my_gi & 7) ^ (tl & 7)) << 4)) = item[i];
+            }
+            um_fence_async_smem();                             // generic-proxy writes before the MMA's reads
+            um_bar_arrive(bar_k + 8 * buf);
+        };
         fetch_codes(0);
+        if (n_chunks > 1) fetch_codes(1);
         asm volatile("cp.async.commit_group;" ::: "memory");
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");
+        rebuild_keys(0);
+        // Iteration c fetches V(c) (and the codes of chunk c + 2), rebuilds the keys of chunk c + 1 while those land,
+        // then hands V(c) over: the key rows run one chunk ahead of the V rows.
+        UM_STAMPS(pp, 5)
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
-            // both buffers of chunk c - 2 are free once its value MMA is done (its score MMA was done before that)
+            // the V buffer of chunk c - 2 is free once its value MMA is done
             if (c >= 2 && !um_producers_wait(ptid == 0, bar_pv + 8 * buf, ((c - 2) >> 1) & 1)) { dead = true; break; }
-            // V rows by cp.async: [nb][token][128 B], 16-byte pieces swizzled by token; the next chunk's codes
-            const bool whole = (long long)(c + 1) * kUmChunk <= t_end;   // every token of the chunk is visible to the tile
+            UM_STAMP(pp, 0)
+            // V rows by cp.async: [nb][token][128 B], 16-byte pieces swizzled by token
+            const bool whole = (long long)(c + 1) * kUmChunk <= t_end;
 #pragma unroll
             for (int i = 0; i < Lay::kVPieces; ++i) {
                 const int p = ptid + i * kUmProducers, tl = p / (D_V / 8), pc = p % (D_V / 8);
@@ -333,36 +392,38 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                 else
                     *reinterpret_cast<uint4 *>(sm + off) = make_uint4(0u, 0u, 0u, 0u);
             }
-            if (c + 1 < n_chunks) fetch_codes(c + 1);
+            if (c + 2 < n_chunks) fetch_codes(c + 2);          // into the code buffer the keys of chunk c were built from
             asm volatile("cp.async.commit_group;" ::: "memory");
-            // key rows: one 16-byte item of the codebook image per (token, 8-dim group, plane)
-            const uint8_t *cs = codes_s + buf * 1024 + my_j;
-            uint32_t code[Lay::kItems];
-#pragma unroll
-            for (int i = 0; i < Lay::kItems; ++i) code[i] = cs[(tl0 + i * kTokStep) * a.m];
-#pragma unroll
-            for (int i = 0; i < Lay::kItems; ++i) {
-                const int tl = tl0 + i * kTokStep;
-                uint4 item = make_uint4(0u, 0u, 0u, 0u);
-                if (whole || (long long)c * kUmChunk + tl < t_end) item = *reinterpret_cast<const uint4 *>(my_src + code[i] * 128);
-                *reinterpret_cast<uint4 *>(my_dst + buf * Lay::kKeys + tl * 128 + (((my_gi & 7) ^ (tl & 7)) << 4)) = item;
+            UM_STAMP(pp, 1)
+            if (c + 1 < n_chunks) {
+                // the key buffer of chunk c - 1 is free once its score MMA is done
+                if (c >= 1 && !um_producers_wait(ptid == 0, bar_s + 8 * (buf ^ 1), ((c - 1) >> 1) & 1)) { dead = true; break; }
+                UM_STAMP(pp, 2)
+                rebuild_keys(c + 1);
             }
+            UM_STAMP(pp, 3)
             asm volatile("cp.async.wait_group 0;" ::: "memory");
-            um_fence_async_smem();                             // generic-proxy writes before the MMA's reads
-            um_bar_arrive(bar_kv + 8 * buf);
-            asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");   // the next chunk's codes are visible to all producers
+            um_fence_async_smem();
+            um_bar_arrive(bar_v + 8 * buf);
+            asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");   // the codes of chunk c + 2 are visible to all producers
+            UM_STAMP(pp, 4)
         }
+#ifdef LOOKAT_PHASE_STAMPS
+        if (UM_FIRST_CTA && ptid == 0) printf("producers: wait V buffer %lld, issue V %lld, wait key buffer %lld, rebuild %lld, land + sync %lld\n", pp[0] / n_chunks, pp[1] / n_chunks, pp[2] / n_chunks, pp[3] / n_chunks, pp[4] / n_chunks);
+#endif
     } else {
         // =================== softmax: thread r owns query row r (tensor-memory lane r) ===================
         const long long row = row0 + tid;
         const long long vis_end = a.q_pos0 + (row < a.L_q ? row : a.L_q - 1) + 1;    // tokens this row sees
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         float m_run = -INFINITY, l_run = 0.f;                  // running maximum (base-2 exponent units) and row sum
+        UM_STAMPS(ss, 5)
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
             const long long tok0 = (long long)c * kUmChunk;
             if (!__all_sync(0xffffffffu, um_bar_wait(bar_s + 8 * buf, (c >> 1) & 1))) { dead = true; break; }   // warp-uniform
             um_fence_after();
+            UM_STAMP(ss, 0)
             uint32_t s0[32], s1[32];
             um_ld32(s0, tm_s + buf * kUmChunk + lane_base);
             um_ld32(s1, tm_s + buf * kUmChunk + 32 + lane_base);
@@ -404,10 +465,12 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                 sum += (b01.x + b01.y) + (b23.x + b23.y);
             }
             l_run = l_run * alpha + sum;
+            UM_STAMP(ss, 1)
             if (c >= 1) {
                 // the previous value MMA must be done before O is rescaled (and it has consumed the other P buffer)
                 if (!__all_sync(0xffffffffu, um_bar_wait(bar_pv + 8 * (buf ^ 1), ((c - 1) >> 1) & 1))) { dead = true; break; }
                 um_fence_after();
+                UM_STAMP(ss, 2)
                 if (__any_sync(0xffffffffu, alpha != 1.f)) {   // a maximum moved in this warp's rows: rescale them
 #pragma unroll 1
                     for (int part = 0; part < D_V / 32; ++part) {
@@ -419,11 +482,16 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                     }
                 }
             }
+            UM_STAMP(ss, 3)
             um_st32(tm_s + buf * kUmChunk + lane_base, pk);    // P over the first half of the S columns, two per column
             um_wait_st();
             um_fence_before();
             um_bar_arrive(bar_p + 8 * buf);
+            UM_STAMP(ss, 4)
         }
+#ifdef LOOKAT_PHASE_STAMPS
+        if (UM_FIRST_CTA && tid == 0) printf("softmax: wait scores %lld, load + exp %lld, wait value MMA %lld, rescale %lld, store %lld (%d chunks)\n", ss[0] / n_chunks, ss[1] / n_chunks, ss[2] / n_chunks, ss[3] / n_chunks, ss[4] / n_chunks, n_chunks);
+#endif
         if (!dead && __all_sync(0xffffffffu, um_bar_wait(bar_pv + 8 * ((n_chunks - 1) & 1), ((n_chunks - 1) >> 1) & 1))) {
             um_fence_after();
             const float inv = 1.f / l_run;
