@@ -40,6 +40,7 @@ constexpr int kUmRows = 128;                   // queries per CTA = rows of one 
 constexpr int kUmChunk = 64;                   // tokens per chunk = columns of the score MMA
 constexpr int kUmSoftmax = 128, kUmProducers = 256;
 constexpr int kUmThreads = kUmSoftmax + kUmProducers + 32;
+constexpr float kUmSlack = 8.f;                // how far a row maximum may run ahead of the softmax reference point
 constexpr int kUmPolls = 1 << 20;              // bound of every mbarrier wait
 
 __device__ __forceinline__ uint32_t um_smem(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -446,10 +447,14 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             }
 #pragma unroll
             for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
-            const float m_new = fmaxf(m_run, mx * a.scale_log2);   // finite from chunk 0 on: token 0 is visible to every row
-            const float alpha = ex2_approx(m_run - m_new);
+            // The reference point m_run of the exponentials follows the row maximum lazily: it moves only when the
+            // maximum has grown by more than kUmSlack (base-2 units), so weights stay below 2^kUmSlack (fine in fp16
+            // and in the fp32 sums) and O is rescaled rarely.  Any reference gives the same normalised result.
+            const float m_cand = mx * a.scale_log2;             // finite in chunk 0: token 0 is visible to every row
+            const bool move = m_cand > m_run + kUmSlack;
+            const float alpha = move ? ex2_approx(m_run - m_cand) : 1.f;
+            const float m_new = move ? m_cand : m_run;
             m_run = m_new;
-            // weights, rounded to fp16 once; the row sum uses the rounded values, as the MMA does
             uint32_t pk[32];
             float sum = 0.f;
 #pragma unroll
@@ -461,8 +466,8 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                 const __half2 h01 = __floats2half2_rn(p0, p1), h23 = __floats2half2_rn(p2, p3);
                 pk[i] = *reinterpret_cast<const uint32_t *>(&h01);
                 pk[16 + i] = *reinterpret_cast<const uint32_t *>(&h23);
-                const float2 b01 = __half22float2(h01), b23 = __half22float2(h23);
-                sum += (b01.x + b01.y) + (b23.x + b23.y);
+                const float2 b01 = __half22float2(h01), b23 = __half22float2(h23);   // the row sum takes the weights as
+                sum += (b01.x + b01.y) + (b23.x + b23.y);                              // the MMA sees them: rounding cancels
             }
             l_run = l_run * alpha + sum;
             UM_STAMP(ss, 1)
