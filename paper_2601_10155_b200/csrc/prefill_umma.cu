@@ -67,11 +67,12 @@ __device__ __forceinline__ bool um_bar_wait(uint32_t bar, uint32_t parity)
     }
     return false;
 }
-// one poll
+// one poll that never suspends the thread (try_wait may park it for a while, which would starve the other condition
+// the MMA thread is watching)
 __device__ __forceinline__ bool um_bar_test(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
                  : "=r"(ok)
                  : "r"(bar), "r"(parity)
                  : "memory");
@@ -111,7 +112,7 @@ __device__ __forceinline__ void um_cp_async16(unsigned dst, const void *src)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 
-// 32 consecutive 32-bit columns of this thread's tensor-memory lane
+// 32 consecutive 32-bit columns of this thread's tensor-memory lane; the registers are valid after um_wait_ld()
 __device__ __forceinline__ void um_ld32(uint32_t (&r)[32], uint32_t taddr)
 {
     asm volatile(
@@ -122,8 +123,8 @@ __device__ __forceinline__ void um_ld32(uint32_t (&r)[32], uint32_t taddr)
           "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
           "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void um_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void um_st32(uint32_t taddr, const uint32_t (&r)[32])
 {
     asm volatile(
@@ -161,9 +162,8 @@ __global__ void um_codebook_image_kernel(const float *__restrict__ books, __half
 template <int D_K, int D_V>
 struct UmLayout {
     static constexpr int kKb = D_K / 64, kNb = D_V / 64;               // 128-byte blocks per key row / V row
-    static constexpr int kPlane = kKb * kUmChunk * 128;                // [kb][64 tokens][128 B]
+    static constexpr int kKeys = kKb * 2 * kUmChunk * 128;             // [kb][64 hi rows, 64 lo rows][128 B]: one operand of 128 rows
     static constexpr int kV = kNb * kUmChunk * 128;                    // [nb][64 tokens][128 B]
-    static constexpr int kKeys = 2 * kPlane;                           // hi plane, lo plane of one chunk
     static constexpr int kOffKeys = 0, kOffV = 2 * kKeys, kOffBook = kOffV + 2 * kV;   // two key buffers, two V buffers
     static constexpr int kIds = D_K / 4;                               // 16-byte items per key row, both planes
     static constexpr int kItems = kUmChunk * kIds / kUmProducers;      // items rebuilt per producer thread per chunk
@@ -171,11 +171,14 @@ struct UmLayout {
     static_assert(kUmChunk * kIds % kUmProducers == 0 && kItems % 4 == 0, "whole items per thread, four codes per word");
     static size_t book_bytes(int K) { return (size_t)K * D_K * 4; }
     // operands, codebook image, then barriers, the tensor-memory address and the codes of two chunks
-    static size_t bytes(int K) { return (size_t)kOffBook + book_bytes(K) + 128 + 2048; }
-    static constexpr int kColO = 2 * kUmChunk, kColQ = kColO + D_V;    // columns: S0, S1 (64 each) | O (D_V) | Q (D_K / 2)
+    // ... then barriers (256 B) and the codes of two chunks (2 KB)
+    static size_t bytes(int K) { return (size_t)kOffBook + book_bytes(K) + 256 + 2048; }
+    static constexpr int kColS = 2 * kUmChunk;                         // one score buffer: hi-plane sums | lo-plane sums
+    static constexpr int kColP = 2 * kColS;                            // weights of one chunk: 64 fp16, two per column
+    static constexpr int kColO = kColP + 2 * (kUmChunk / 2), kColQ = kColO + D_V;   // columns: S0 | S1 | P0 | P1 | O (D_V) | Q (D_K / 2)
     static constexpr int kTmemCols = kColQ + D_K / 2 <= 256 ? 256 : 512;
     // instruction descriptors: fp32 accumulate, fp16 operands, N >> 3 at bit 17, M >> 4 at bit 24; bit 16: B is MN-major
-    static constexpr uint32_t kIdescS = (1u << 4) | ((uint32_t)(kUmChunk >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
+    static constexpr uint32_t kIdescS = (1u << 4) | ((uint32_t)(2 * kUmChunk >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
     static constexpr uint32_t kIdescO = (1u << 4) | (1u << 16) | ((uint32_t)(D_V >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
 };
 
@@ -190,8 +193,8 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
     const uint32_t book_bytes = (uint32_t)a.K * D_K * 4;
     unsigned char *const book = sm + Lay::kOffBook;
     uint64_t *const bars = reinterpret_cast<uint64_t *>(book + book_bytes);
-    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(bars + 12);
-    uint8_t *const codes_s = reinterpret_cast<uint8_t *>(bars + 16);  // [2][1024]: the codes of two chunks
+    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(bars + 30);
+    uint8_t *const codes_s = reinterpret_cast<uint8_t *>(bars + 32);  // [2][1024]: the codes of two chunks
     // barriers, one per buffer: k_ready[2], v_ready[2] (keys / V staged), s_full[2] (scores done), pv_done[2] (value MMA
     // done), p_ready[2] (weights stored)
     const uint32_t bar0 = um_smem(bars);
@@ -235,11 +238,11 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         um_fence_after();
     }
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tm_s = tmem, tm_o = tmem + Lay::kColO, tm_q = tmem + Lay::kColQ;   // columns: S0 | S1 | O | Q
+    const uint32_t tm_s = tmem, tm_p = tmem + Lay::kColP, tm_o = tmem + Lay::kColO, tm_q = tmem + Lay::kColQ;
     bool dead = (sm0 & 1023u) != 0;                            // a wait ran out (or the base is misaligned): leave, free, return
 
     // ---- the query rows go to tensor memory as the A operand of the score MMA: lane r = row r, two halfs per column ----
-    if (warp < 4) {
+    if (warp < 4) {                                            // one thread per row
         const long long qr = row0 + tid < a.L_q ? row0 + tid : a.L_q - 1;       // rows beyond L_q repeat the last one
         const uint4 *src = reinterpret_cast<const uint4 *>(a.q + ((size_t)(b * a.H_q + hq) * a.L_q + qr) * D_K);
 #pragma unroll
@@ -271,22 +274,20 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
             const uint32_t keys_lo = ((sm0 + Lay::kOffKeys) >> 4) | (1u << 16);                    // leading offset unused (16 B)
             const uint32_t v_lo = ((sm0 + Lay::kOffV) >> 4) | ((uint32_t)(kUmChunk * 128 / 16) << 16);   // between 64-column blocks
-            auto score_mma = [&](int c) {                      // S[c & 1] = Q . K^(c)^T, both planes
+            auto score_mma = [&](int c) {                      // S[c & 1] = Q . [K^hi(c); K^lo(c)]^T: 64 + 64 columns
                 const int buf = c & 1;
-                const uint32_t lo = keys_lo + buf * (Lay::kKeys >> 4), d = tm_s + buf * kUmChunk;
+                const uint32_t lo = keys_lo + buf * (Lay::kKeys >> 4), d = tm_s + buf * Lay::kColS;
 #pragma unroll
-                for (int plane = 0; plane < 2; ++plane)
-#pragma unroll
-                    for (int ks = 0; ks < D_K / 16; ++ks) {
-                        const uint32_t off = (plane * Lay::kPlane + (ks >> 2) * (kUmChunk * 128) + (ks & 3) * 32) >> 4;
-                        if (plane == 0 && ks == 0) um_mma_ts<false>(d, tm_q + ks * 8, lo + off, desc_hi, Lay::kIdescS);
-                        else um_mma_ts<true>(d, tm_q + ks * 8, lo + off, desc_hi, Lay::kIdescS);
-                    }
+                for (int ks = 0; ks < D_K / 16; ++ks) {            // 128 operand rows: the hi and the lo plane of 64 tokens
+                    const uint32_t off = ((ks >> 2) * (2 * kUmChunk * 128) + (ks & 3) * 32) >> 4;
+                    if (ks == 0) um_mma_ts<false>(d, tm_q + ks * 8, lo + off, desc_hi, Lay::kIdescS);
+                    else um_mma_ts<true>(d, tm_q + ks * 8, lo + off, desc_hi, Lay::kIdescS);
+                }
                 um_commit(bar_s + 8 * buf);
             };
-            auto value_mma = [&](int c) {                      // O += P(c) . V(c), P read from the S columns of its buffer
+            auto value_mma = [&](int c) {                      // O += P(c) . V(c), P read from tensor memory
                 const int buf = c & 1;
-                const uint32_t lo = v_lo + buf * (Lay::kV >> 4), pa = tm_s + buf * kUmChunk;
+                const uint32_t lo = v_lo + buf * (Lay::kV >> 4), pa = tm_p + buf * (kUmChunk / 2);
 #pragma unroll
                 for (int kt = 0; kt < kUmChunk / 16; ++kt) {   // 16 tokens: 8 columns of weights, two 8-token groups of V
                     if (kt == 0 && c == 0) um_mma_ts<false>(tm_o, pa + kt * 8, lo + kt * (2048 >> 4), desc_hi, Lay::kIdescO);
@@ -324,7 +325,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             if (UM_FIRST_CTA) printf("mma thread: idle %lld, score issue %lld, value issue %lld cycles per chunk\n", mm[0] / n_chunks, mm[1] / n_chunks, mm[2] / n_chunks);
 #endif
         }
-    } else if (warp >= 4) {
+    } else if (warp >= kUmSoftmax / 32) {
         // =================== producers ===================
         const int ptid = tid - kUmSoftmax;
         const uint8_t *codes = a.codes + (size_t)(b * a.H_kv + h) * a.L_max * a.m;
@@ -333,7 +334,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         const int my_id = ptid % Lay::kIds, my_plane = my_id / (D_K / 8), my_gi = my_id % (D_K / 8);
         const int my_j = (my_gi * 8) / d_sub;
         const unsigned char *my_src = book + (uint32_t)my_plane * (book_bytes / 2) + (uint32_t)(my_gi >> 3) * a.K * 128 + ((my_gi & 7) << 4);
-        unsigned char *my_dst = sm + Lay::kOffKeys + my_plane * Lay::kPlane + (my_gi >> 3) * (kUmChunk * 128);   // + buf * kKeys
+        unsigned char *my_dst = sm + Lay::kOffKeys + (my_gi >> 3) * (2 * kUmChunk * 128) + my_plane * (kUmChunk * 128);   // + buf * kKeys
         const int tl0 = ptid / Lay::kIds;                      // this thread's tokens of a chunk: tl0 + i * (producers / kIds)
         constexpr int kTokStep = kUmProducers / Lay::kIds;
         const int code_bytes = kUmChunk * a.m;                 // codes of one chunk, staged in shared memory a chunk ahead
@@ -417,7 +418,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         const long long row = row0 + tid;
         const long long vis_end = a.q_pos0 + (row < a.L_q ? row : a.L_q - 1) + 1;    // tokens this row sees
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        float m_run = -INFINITY, l_run = 0.f;                  // running maximum (base-2 exponent units) and row sum
+        float m_run = -INFINITY, l_run = 0.f;                  // reference point (base-2 exponent units) and row sum
         UM_STAMPS(ss, 5)
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
@@ -425,62 +426,66 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             if (!__all_sync(0xffffffffu, um_bar_wait(bar_s + 8 * buf, (c >> 1) & 1))) { dead = true; break; }   // warp-uniform
             um_fence_after();
             UM_STAMP(ss, 0)
-            uint32_t s0[32], s1[32];
-            um_ld32(s0, tm_s + buf * kUmChunk + lane_base);
-            um_ld32(s1, tm_s + buf * kUmChunk + 32 + lane_base);
+            float sc[kUmChunk];                                // raw scores: hi-plane sum + lo-plane sum
+            {
+                uint32_t h0[32], l0[32], h1[32], l1[32];
+                const uint32_t at = tm_s + buf * Lay::kColS + lane_base;
+                um_ld32(h0, at);
+                um_ld32(l0, at + kUmChunk);
+                um_ld32(h1, at + 32);
+                um_ld32(l1, at + kUmChunk + 32);
+                um_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    sc[i] = __uint_as_float(h0[i]) + __uint_as_float(l0[i]);
+                    sc[32 + i] = __uint_as_float(h1[i]) + __uint_as_float(l1[i]);
+                }
+            }
             if (SCORES && a.scores_out && row < a.L_q) {
                 float *dst = a.scores_out + ((size_t)(b * a.H_q + hq) * a.L_q + row) * a.L_max + tok0;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    if (tok0 + i < vis_end) dst[i] = __uint_as_float(s0[i]);
-                    if (tok0 + 32 + i < vis_end) dst[32 + i] = __uint_as_float(s1[i]);
-                }
+                for (int i = 0; i < kUmChunk; ++i)
+                    if (tok0 + i < vis_end) dst[i] = sc[i];
             }
-            // the scale is positive, so the maximum can be taken on the raw scores
-            float mx = -INFINITY;
             if (tok0 + kUmChunk > vis_end) {                   // the chunk crosses this row's causal limit
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    if (tok0 + i >= vis_end) s0[i] = 0xff800000u;
-                    if (tok0 + 32 + i >= vis_end) s1[i] = 0xff800000u;
-                }
+                for (int i = 0; i < kUmChunk; ++i)
+                    if (tok0 + i >= vis_end) sc[i] = -INFINITY;
             }
+            float mx = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
+            for (int i = 0; i < kUmChunk; ++i) mx = fmaxf(mx, sc[i]);
             // The reference point m_run of the exponentials follows the row maximum lazily: it moves only when the
             // maximum has grown by more than kUmSlack (base-2 units), so weights stay below 2^kUmSlack (fine in fp16
             // and in the fp32 sums) and O is rescaled rarely.  Any reference gives the same normalised result.
-            const float m_cand = mx * a.scale_log2;             // finite in chunk 0: token 0 is visible to every row
+            const float m_cand = mx * a.scale_log2;             // the scale is positive; finite in chunk 0 (token 0 is visible)
             const bool move = m_cand > m_run + kUmSlack;
             const float alpha = move ? ex2_approx(m_run - m_cand) : 1.f;
-            const float m_new = move ? m_cand : m_run;
-            m_run = m_new;
+            m_run = move ? m_cand : m_run;
             uint32_t pk[32];
             float sum = 0.f;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float p0 = ex2_approx(fmaf(__uint_as_float(s0[2 * i]), a.scale_log2, -m_new));
-                const float p1 = ex2_approx(fmaf(__uint_as_float(s0[2 * i + 1]), a.scale_log2, -m_new));
-                const float p2 = ex2_approx(fmaf(__uint_as_float(s1[2 * i]), a.scale_log2, -m_new));
-                const float p3 = ex2_approx(fmaf(__uint_as_float(s1[2 * i + 1]), a.scale_log2, -m_new));
-                const __half2 h01 = __floats2half2_rn(p0, p1), h23 = __floats2half2_rn(p2, p3);
+            for (int i = 0; i < 32; ++i) {
+                const float p0 = ex2_approx(fmaf(sc[2 * i], a.scale_log2, -m_run));
+                const float p1 = ex2_approx(fmaf(sc[2 * i + 1], a.scale_log2, -m_run));
+                const __half2 h01 = __floats2half2_rn(p0, p1);
                 pk[i] = *reinterpret_cast<const uint32_t *>(&h01);
-                pk[16 + i] = *reinterpret_cast<const uint32_t *>(&h23);
-                const float2 b01 = __half22float2(h01), b23 = __half22float2(h23);   // the row sum takes the weights as
-                sum += (b01.x + b01.y) + (b23.x + b23.y);                              // the MMA sees them: rounding cancels
+                const float2 b01 = __half22float2(h01);        // the row sum takes the weights as the MMA sees them:
+                sum += b01.x + b01.y;                          // their rounding cancels in the normalised result
             }
             l_run = l_run * alpha + sum;
             UM_STAMP(ss, 1)
             if (c >= 1) {
-                // the previous value MMA must be done before O is rescaled (and it has consumed the other P buffer)
+                // the previous value MMA must be done before O is rescaled; the one before it has released this P buffer
                 if (!__all_sync(0xffffffffu, um_bar_wait(bar_pv + 8 * (buf ^ 1), ((c - 1) >> 1) & 1))) { dead = true; break; }
                 um_fence_after();
                 UM_STAMP(ss, 2)
-                if (__any_sync(0xffffffffu, alpha != 1.f)) {   // a maximum moved in this warp's rows: rescale them
+                if (__any_sync(0xffffffffu, alpha != 1.f)) {   // a reference point moved in this warp's rows: rescale them
 #pragma unroll 1
                     for (int part = 0; part < D_V / 32; ++part) {
                         uint32_t o[32];
                         um_ld32(o, tm_o + part * 32 + lane_base);
+                        um_wait_ld();
 #pragma unroll
                         for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
                         um_st32(tm_o + part * 32 + lane_base, o);
@@ -488,7 +493,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                 }
             }
             UM_STAMP(ss, 3)
-            um_st32(tm_s + buf * kUmChunk + lane_base, pk);    // P over the first half of the S columns, two per column
+            um_st32(tm_p + buf * (kUmChunk / 2) + lane_base, pk);   // the 64 weights, two per column
             um_wait_st();
             um_fence_before();
             um_bar_arrive(bar_p + 8 * buf);
@@ -504,6 +509,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             for (int part = 0; part < D_V / 32; ++part) {
                 uint32_t o[32];
                 um_ld32(o, tm_o + part * 32 + lane_base);
+                um_wait_ld();
                 if (row < a.L_q) {
                     float4 *dst = reinterpret_cast<float4 *>(a.out + ((size_t)(b * a.H_q + hq) * a.L_q + row) * D_V + part * 32);
 #pragma unroll
@@ -561,7 +567,7 @@ bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a)
     // the row maxima are taken on the raw scores, which needs a positive softmax scale
     if (!shape || !aligned || a.H_q > 65535 || a.B > 65535 || !(a.scale_log2 > 0.f) || !ctx->timeout_flag) return false;
     const size_t operands = (size_t)kUmRows * a.d_k * 2 + 2 * (size_t)kUmChunk * a.d_k * 2 + 2 * (size_t)kUmChunk * a.d_v * 2;
-    return operands + (size_t)a.K * a.d_k * 4 + 64 + 2048 <= (size_t)ctx->max_smem_optin;
+    return operands + (size_t)a.K * a.d_k * 4 + 256 + 2048 <= (size_t)ctx->max_smem_optin;
 }
 
 lookat_status launch_prefill_umma(Ctx *ctx, const PrefillArgs &a)
