@@ -43,13 +43,19 @@ FALLBACK_HBM_GBS = 6650.0
 ATTEND_DRAM_BYTES_PER_PAIR = {"gqa_32k_m8": 283105792 / 1048576}
 
 
-def measured_peak_gbs():
+def measured_peak(key: str, fallback: float):
+    """A figure of MEASURED_PEAKS.json ("of measured"), else the stated fallback ("of fallback")."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
+            return float(json.load(f)[key]), "of measured"
     except Exception:
-        return FALLBACK_HBM_GBS, "fallback"
+        return fallback, "of fallback"
+
+
+def measured_peak_gbs():
+    peak, which = measured_peak("hbm_gbs", FALLBACK_HBM_GBS)
+    return peak, which[3:]
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -229,10 +235,11 @@ def workload_config(w):
 
 
 # ----------------------------------------------------------------------------- GPU leg
-def time_prefill(device_index: int, steps: int = 5, batch: int = 0, heads: int = 0):
+def time_prefill(device_index: int, steps: int = 5, batch: int = 0, heads: int = 0, form: str = "auto"):
     """Causal multi-query attention (lookat_attend_prefill) on the prefill_4k_m16 shape: batch 4, 32 heads,
-    4096 queries over 4096 cached tokens, d = 128, m = 16.  Bound: the m gathers per (query, token) pair
-    from shared memory, 4 bytes each, against 128 bytes per clock and SM."""
+    4096 queries over 4096 cached tokens, d = 128, m = 16.  The contraction forms are bound by the tensor
+    cores: per visible (query, token) pair 2 * d_k MACs of scores (two fp16 planes of each centroid) and
+    d_v MACs of the value sum; the table form by its m shared-memory gathers per pair."""
     import torch
 
     from paper_2601_10155_b200.binding import Lookat
@@ -243,6 +250,7 @@ def time_prefill(device_index: int, steps: int = 5, batch: int = 0, heads: int =
                               "name": f"{w.name}_b{batch or w.B}_h{heads or w.n_q_heads}"})
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
     lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K, device=device_index)
+    lk.lookat_set_prefill_form(form)
     keys = dev(synth.make_keys(w))
     v = dev(synth.make_values(w))
     q = dev(synth.make_prefill_queries(w, w.L))
@@ -260,13 +268,21 @@ def time_prefill(device_index: int, steps: int = 5, batch: int = 0, heads: int =
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
     pairs = w.B * w.n_q_heads * w.L * (w.L + 1) // 2
-    props = torch.cuda.get_device_properties(device_index)
-    smem_peak = props.multi_processor_count * 128 * 1.965e9 / 1e9          # GB/s at the maximum SM clock
-    achieved = pairs * w.m * 4 / (ms * 1e-3) / 1e9
-    return {"workload": w.name, "ms": ms, "pairs_per_s": pairs / (ms * 1e-3), "steps": steps,
-            "roofline": {"bound": "smem", "achieved": achieved, "peak": smem_peak, "unit": "GB/s",
-                         "frac": achieved / smem_peak,
-                         "note": "gather bytes (m x 4 B per pair) over 128 B/clk/SM x SMs x 1965 MHz"}}
+    res = {"workload": w.name, "form": form, "ms": ms, "pairs_per_s": pairs / (ms * 1e-3), "steps": steps}
+    if form == "tables":
+        props = torch.cuda.get_device_properties(device_index)
+        smem_peak = props.multi_processor_count * 128 * 1.965e9 / 1e9      # GB/s at the maximum SM clock
+        achieved = pairs * w.m * 4 / (ms * 1e-3) / 1e9
+        res["roofline"] = {"bound": "smem", "achieved": achieved, "peak": smem_peak, "unit": "GB/s",
+                           "frac": achieved / smem_peak,
+                           "note": "gather bytes (m x 4 B per pair) over 128 B/clk/SM x SMs x 1965 MHz"}
+    else:
+        peak, which = measured_peak("bf16_tflops", 1590.0)                 # fp16 and bf16 run at the same rate
+        achieved = pairs * 2.0 * (2 * w.d_k + w.d_v) / (ms * 1e-3) / 1e12
+        res["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                           "frac": achieved / peak,
+                           "note": f"2 x (2 d_k + d_v) flop per visible pair; peak: cuBLAS bf16 burst, {which}"}
+    return res
 
 
 def run_lookat(args, w):
@@ -434,6 +450,8 @@ def main():
                     help="time only the causal multi-query kernel (prints its object alone)")
     ap.add_argument("--prefill-batch", type=int, default=0, help="smaller prefill case: batch rows")
     ap.add_argument("--prefill-heads", type=int, default=0, help="smaller prefill case: heads")
+    ap.add_argument("--prefill-form", default="auto", choices=["auto", "tables", "contraction", "contraction_mma_sync"],
+                    help="which kernel lookat_attend_prefill uses in the prefill timing")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size (smaller cases for profiler captures)")
     args = ap.parse_args()
@@ -442,7 +460,7 @@ def main():
         w = synth.Workload(**{**w.__dict__, "B": args.batch, "name": f"{w.name}_b{args.batch}"})
     if args.only_prefill:
         print(json.dumps(time_prefill(int(os.environ.get("LOCAL_RANK", "0")), steps=max(1, min(args.steps, 5)),
-                                      batch=args.prefill_batch, heads=args.prefill_heads)), flush=True)
+                                      batch=args.prefill_batch, heads=args.prefill_heads, form=args.prefill_form)), flush=True)
     elif args.impl == "reference":
         run_reference(args, w)
     else:
