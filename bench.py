@@ -317,12 +317,13 @@ def run_lookat(args, w):
     per_row = max(1, n_fit // w.B)
     fit_keys = keys[:, :, :per_row].contiguous()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-    ev[0].record()
-    books = lk.lookat_fit_codebooks(fit_keys, w.fit_iters, seed=w.seed)
-    ev[1].record()
-    ties = torch.zeros(1, dtype=torch.int64, device="cuda")
-    codes = lk.lookat_encode_keys(keys, books, near_ties=ties)
-    ev[2].record()
+    for attempt in range(2):                               # the second pass is timed: no first-call allocations, clocks up
+        ev[0].record()
+        books = lk.lookat_fit_codebooks(fit_keys, w.fit_iters, seed=w.seed)
+        ev[1].record()
+        ties = torch.zeros(1, dtype=torch.int64, device="cuda")
+        codes = lk.lookat_encode_keys(keys, books, near_ties=ties)
+        ev[2].record()
     torch.cuda.synchronize()
     fit_ms, enc_ms = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
     del fit_keys
