@@ -1,7 +1,8 @@
 """Parity at the full size of the benchmark workload (`gqa_32k_m8`: batch 16, 32 query heads on 8 KV
 heads, d = 128, 32768 cached tokens, m = 8), in the launch configuration bench.py times
 (`lookat_decode_step`, library-chosen chunking), on sampled rows the oracle can compute one by one;
-plus properties that hold at any size.  Also the 1M-key encode shape on a subset the oracle can do.
+plus properties that hold at any size.  Also the 1M-key encode shape on a subset the oracle can do,
+and the causal prefill launch of config 4 in its three forms on sampled queries.
 """
 import numpy as np
 import pytest
@@ -127,3 +128,47 @@ def test_encode_shape_of_the_1m_key_workload_on_a_subset():
     near = (gap > 0) & (gap < 1e-6)
     assert not ((codes != ref) & ~near).any()
     assert int(ties.item()) == int(near.sum())
+
+
+# ------------------------------------------------------------------ causal prefill at the config-4 size
+@pytest.fixture(scope="module")
+def prefill_4k():
+    w = synth.WORKLOADS["prefill_4k_m16"]
+    keys, v = synth.make_keys(w), synth.make_values(w)
+    q = synth.make_prefill_queries(w, w.L)
+    books, _ = oracle.fit_codebooks(synth.make_calibration_keys(w, 2048), w.m, w.K, iters=2, seed=w.seed)
+    lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K)
+    codes_d = lk.lookat_encode_keys(dev(keys), dev(books))
+    torch.cuda.synchronize()
+    return dict(w=w, keys=keys, v=v, q=q, books=books, lk=lk, codes_d=codes_d)
+
+
+@pytest.mark.parametrize("form", ["contraction", "contraction_mma_sync", "tables"])
+def test_full_size_prefill_on_sampled_rows(prefill_4k, form):
+    """The whole config-4 launch (batch 4, 32 heads, 4096 causal queries over 4096 tokens) as bench.py times it;
+    sampled (row, head, query) triples against the oracle, tile and chunk edges among them; and a closed form
+    for every head: the first query sees one token, so its output is that token's value row."""
+    s = prefill_4k
+    w, lk = s["w"], s["lk"]
+    heads = [(0, 0), (1, 13), (3, 31)]
+    queries = [0, 1, 63, 64, 127, 128, 129, 1000, 2047, 2048, 4032, 4095]
+    # hand-off: the sampled heads get the oracle's codes (the GPU's are checked against them first)
+    for b, h in heads:
+        ref_codes, gap = oracle.encode_keys(s["keys"][b:b + 1, h:h + 1], s["books"][h:h + 1], want_gap=True)
+        got = s["codes_d"][b, h].cpu().numpy()
+        near = (gap[0, 0] > 0) & (gap[0, 0] < 1e-6)
+        assert not ((got != ref_codes[0, 0]) & ~near).any()
+        s["codes_d"][b, h] = dev(ref_codes[0, 0])
+    lk.lookat_set_prefill_form(form)
+    out = lk.lookat_attend_prefill(dev(s["q"]), dev(s["books"]), s["codes_d"], dev(s["v"]))
+    torch.cuda.synchronize()
+    lk.lookat_set_prefill_form("auto")
+    out = out.cpu().numpy()
+    assert np.isfinite(out).all()
+    assert np.abs(out[:, :, 0] - s["v"][:, :, 0].astype(np.float32)).max() <= 1e-3
+    for b, h in heads:
+        codes_row = s["codes_d"][b, h].cpu().numpy()[None, None]
+        for i in queries:
+            ref = oracle.attend_prefill(s["q"][b:b + 1, h:h + 1, i:i + 1], s["books"][h:h + 1], codes_row,
+                                        s["v"][b:b + 1, h:h + 1], q_pos0=i)
+            assert np.abs(out[b, h, i] - ref[0, 0, 0]).max() <= OUT_TOL, (form, b, h, i)
