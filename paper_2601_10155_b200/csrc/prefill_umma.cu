@@ -9,12 +9,13 @@
 // per query row, O += P . V with P read from tensor memory.  q (fp16) is an exact operand; every fp32
 // centroid is split into two fp16 planes (rounding + remainder), which carries s to ~2^-22 relative.
 //
-// Roles in a CTA of 13 warps (one CTA per SM; the shared memory is full):
+// Roles in a CTA of 15 warps (one CTA per SM; the shared memory is full):
 //   warps 0-3  softmax: thread r owns query row r = tensor-memory lane r;
 //   warps 4-11 producers: rebuild the next chunk's key rows from the codebook image in shared memory
 //              (16-byte items placed so that gathers and stores are free of bank conflicts whatever
 //              the codes are) and fetch its V rows with cp.async;
-//   warp 12    one thread issues every MMA and commits them to mbarriers.
+//   warps 12-13 fetch the V rows of the chunk after next with cp.async, on their own schedule;
+//   warp 14    one thread issues every MMA and commits them to mbarriers.
 // Hand-offs go through mbarriers, one per buffer where a buffer is reused, so that no waiter can fall
 // two phases behind; every wait gives up after a bounded number of polls, raises the context's timeout
 // flag and lets the CTA drain and free its tensor memory.
@@ -38,8 +39,8 @@ namespace {
 
 constexpr int kUmRows = 128;                   // queries per CTA = rows of one MMA
 constexpr int kUmChunk = 64;                   // tokens per chunk = columns of the score MMA
-constexpr int kUmSoftmax = 128, kUmProducers = 256;
-constexpr int kUmThreads = kUmSoftmax + kUmProducers + 32;
+constexpr int kUmSoftmax = 128, kUmProducers = 256, kUmVLoaders = 64;
+constexpr int kUmThreads = kUmSoftmax + kUmProducers + kUmVLoaders + 32;
 constexpr float kUmSlack = 8.f;                // how far a row maximum may run ahead of the softmax reference point
 constexpr int kUmPolls = 1 << 20;              // bound of every mbarrier wait
 
@@ -78,14 +79,16 @@ __device__ __forceinline__ bool um_bar_test(uint32_t bar, uint32_t parity)
                  : "memory");
     return ok != 0;
 }
-// One thread polls, the named barrier hands its verdict to all producers: nobody leaves a loop alone.
-__device__ __forceinline__ bool um_producers_wait(bool poller, uint32_t bar, uint32_t parity)
+// One thread polls, the named barrier hands its verdict to the whole group (key producers: barrier 1, V loaders:
+// barrier 2): nobody leaves a loop alone.
+template <int BARRIER, int THREADS>
+__device__ __forceinline__ bool um_group_wait(bool poller, uint32_t bar, uint32_t parity)
 {
     const uint32_t failed = poller ? (um_bar_wait(bar, parity) ? 0u : 1u) : 0u;
     uint32_t any;
-    asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, 1, %2, p;\nselp.u32 %0, 1, 0, q;\n}"
+    asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, %2, %3, p;\nselp.u32 %0, 1, 0, q;\n}"
                  : "=r"(any)
-                 : "r"(failed), "n"(kUmProducers)
+                 : "r"(failed), "n"(BARRIER), "n"(THREADS)
                  : "memory");
     return any == 0;
 }
@@ -167,7 +170,6 @@ struct UmLayout {
     static constexpr int kOffKeys = 0, kOffV = 2 * kKeys, kOffBook = kOffV + 2 * kV;   // two key buffers, two V buffers
     static constexpr int kIds = D_K / 4;                               // 16-byte items per key row, both planes
     static constexpr int kItems = kUmChunk * kIds / kUmProducers;      // items rebuilt per producer thread per chunk
-    static constexpr int kVPieces = kUmChunk * (D_V / 8) / kUmProducers;
     static_assert(kUmChunk * kIds % kUmProducers == 0 && kItems % 4 == 0, "whole items per thread, four codes per word");
     static size_t book_bytes(int K) { return (size_t)K * D_K * 4; }
     // operands, codebook image, then barriers, the tensor-memory address and the codes of two chunks
@@ -218,7 +220,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         if (tid == 0) {
             for (int i = 0; i < 2; ++i) {
                 um_bar_init(bar_k + 8 * i, kUmProducers);
-                um_bar_init(bar_v + 8 * i, kUmProducers);
+                um_bar_init(bar_v + 8 * i, kUmVLoaders);
                 um_bar_init(bar_s + 8 * i, 1);
                 um_bar_init(bar_pv + 8 * i, 1);
                 um_bar_init(bar_p + 8 * i, kUmSoftmax);
@@ -266,7 +268,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
 
     if (dead) {
         // misaligned shared-memory base: nothing runs
-    } else if (warp >= (kUmSoftmax + kUmProducers) / 32) {
+    } else if (warp >= (kUmSoftmax + kUmProducers + kUmVLoaders) / 32) {
         // =================== the MMA thread ===================
         if (lane == 0) {
             // descriptors: stride 1024 B, version 1, 128-byte swizzle in the high word; the low word holds the start
@@ -325,11 +327,10 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             if (UM_FIRST_CTA) printf("mma thread: idle %lld, score issue %lld, value issue %lld cycles per chunk\n", mm[0] / n_chunks, mm[1] / n_chunks, mm[2] / n_chunks);
 #endif
         }
-    } else if (warp >= kUmSoftmax / 32) {
-        // =================== producers ===================
+    } else if (warp >= kUmSoftmax / 32 && warp < (kUmSoftmax + kUmProducers) / 32) {
+        // =================== key producers ===================
         const int ptid = tid - kUmSoftmax;
         const uint8_t *codes = a.codes + (size_t)(b * a.H_kv + h) * a.L_max * a.m;
-        const __half *vsrc = a.v + (size_t)(b * a.H_kv + h) * a.L_max * D_V;
         // item p = ptid + i * producers of a chunk: token p / kIds, id = p % kIds = plane * (D_K/8) + gi (fixed per thread)
         const int my_id = ptid % Lay::kIds, my_plane = my_id / (D_K / 8), my_gi = my_id % (D_K / 8);
         const int my_j = (my_gi * 8) / d_sub;
@@ -375,43 +376,54 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");
         rebuild_keys(0);
-        // Iteration c fetches V(c) (and the codes of chunk c + 2), rebuilds the keys of chunk c + 1 while those land,
-        // then hands V(c) over: the key rows run one chunk ahead of the V rows.
-        UM_STAMPS(pp, 5)
+        asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");   // everyone is done with the codes of chunk 0
+        // keys of chunk c into the buffer that the score MMA of chunk c - 2 has released; codes two chunks ahead
+        UM_STAMPS(pp, 3)
+        for (int c = 1; c < n_chunks; ++c) {
+            if (c >= 2 && !um_group_wait<1, kUmProducers>(ptid == 0, bar_s + 8 * (c & 1), ((c - 2) >> 1) & 1)) { dead = true; break; }
+            UM_STAMP(pp, 0)
+            rebuild_keys(c);
+            UM_STAMP(pp, 1)
+            if (c + 1 < n_chunks) fetch_codes(c + 1);          // into the code buffer the keys of chunk c - 1 were built from
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");   // those codes are visible to all key producers
+            UM_STAMP(pp, 2)
+        }
+#ifdef LOOKAT_PHASE_STAMPS
+        if (UM_FIRST_CTA && ptid == 0) printf("key producers: wait key buffer %lld, rebuild %lld, codes + sync %lld\n", pp[0] / n_chunks, pp[1] / n_chunks, pp[2] / n_chunks);
+#endif
+    } else if (warp >= (kUmSoftmax + kUmProducers) / 32) {
+        // =================== V loaders ===================
+        const int vtid = tid - kUmSoftmax - kUmProducers;
+        const __half *vsrc = a.v + (size_t)(b * a.H_kv + h) * a.L_max * D_V;
+        constexpr int kPieces = kUmChunk * (D_V / 8) / kUmVLoaders;
+        UM_STAMPS(vv, 3)
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
             // the V buffer of chunk c - 2 is free once its value MMA is done
-            if (c >= 2 && !um_producers_wait(ptid == 0, bar_pv + 8 * buf, ((c - 2) >> 1) & 1)) { dead = true; break; }
-            UM_STAMP(pp, 0)
+            if (c >= 2 && !um_group_wait<2, kUmVLoaders>(vtid == 0, bar_pv + 8 * buf, ((c - 2) >> 1) & 1)) { dead = true; break; }
+            UM_STAMP(vv, 0)
             // V rows by cp.async: [nb][token][128 B], 16-byte pieces swizzled by token
             const bool whole = (long long)(c + 1) * kUmChunk <= t_end;
 #pragma unroll
-            for (int i = 0; i < Lay::kVPieces; ++i) {
-                const int p = ptid + i * kUmProducers, tl = p / (D_V / 8), pc = p % (D_V / 8);
+            for (int i = 0; i < kPieces; ++i) {
+                const int p = vtid + i * kUmVLoaders, tl = p / (D_V / 8), pc = p % (D_V / 8);
                 const uint32_t off = Lay::kOffV + buf * Lay::kV + (pc >> 3) * (kUmChunk * 128) + tl * 128 + (((pc & 7) ^ (tl & 7)) << 4);
                 if (whole || (long long)c * kUmChunk + tl < t_end)
                     um_cp_async16(sm0 + off, vsrc + ((size_t)c * kUmChunk + tl) * D_V + pc * 8);
                 else
                     *reinterpret_cast<uint4 *>(sm + off) = make_uint4(0u, 0u, 0u, 0u);
             }
-            if (c + 2 < n_chunks) fetch_codes(c + 2);          // into the code buffer the keys of chunk c were built from
             asm volatile("cp.async.commit_group;" ::: "memory");
-            UM_STAMP(pp, 1)
-            if (c + 1 < n_chunks) {
-                // the key buffer of chunk c - 1 is free once its score MMA is done
-                if (c >= 1 && !um_producers_wait(ptid == 0, bar_s + 8 * (buf ^ 1), ((c - 1) >> 1) & 1)) { dead = true; break; }
-                UM_STAMP(pp, 2)
-                rebuild_keys(c + 1);
-            }
-            UM_STAMP(pp, 3)
+            UM_STAMP(vv, 1)
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             um_fence_async_smem();
             um_bar_arrive(bar_v + 8 * buf);
-            asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");   // the codes of chunk c + 2 are visible to all producers
-            UM_STAMP(pp, 4)
+            UM_STAMP(vv, 2)
         }
 #ifdef LOOKAT_PHASE_STAMPS
-        if (UM_FIRST_CTA && ptid == 0) printf("producers: wait V buffer %lld, issue V %lld, wait key buffer %lld, rebuild %lld, land + sync %lld\n", pp[0] / n_chunks, pp[1] / n_chunks, pp[2] / n_chunks, pp[3] / n_chunks, pp[4] / n_chunks);
+        if (UM_FIRST_CTA && vtid == 0) printf("V loaders: wait V buffer %lld, issue %lld, land %lld\n", vv[0] / n_chunks, vv[1] / n_chunks, vv[2] / n_chunks);
 #endif
     } else {
         // =================== softmax: thread r owns query row r (tensor-memory lane r) ===================
