@@ -438,3 +438,36 @@ def test_attend_prefill_matches_oracle(shape, L_q, q_pos0, q_scale, form):
         dec = lk.lookat_attend(dev(codes), dev(v), q=dev(np.ascontiguousarray(q[:, :, -1])), codebooks=dev(books))
         # the contraction form rounds each weight to fp16 once (relative 2^-12) where decode keeps two planes
         assert float((dec - out[:, :, -1]).abs().max()) <= (2e-5 if form == "tables" else 3e-4)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_attend_prefill_contraction_on_random_shapes(seed):
+    """Shapes drawn at random inside what the tensor-core forms cover: grouped heads, codebooks small enough for two
+    CTAs per SM, query slices that start and end anywhere; both contraction kernels against the oracle, twice
+    (the second call reuses the context's scratch)."""
+    rng = np.random.default_rng(9000 + seed)
+    d_k, d_v = int(rng.choice([64, 128])), int(rng.choice([64, 128]))
+    d_sub = int(rng.choice([8, 16, 32]))
+    H_kv = int(rng.choice([1, 2, 3]))
+    g = int(rng.choice([1, 2, 4]))
+    K = int(rng.choice([16, 64, 200, 256]))
+    L = int(rng.integers(70, 700))
+    L_q = int(rng.integers(1, L + 1))
+    q_pos0 = int(rng.integers(0, L - L_q + 1))
+    B = int(rng.choice([1, 2, 3]))
+    w = synth.small_workload(B=B, n_q_heads=H_kv * g, n_kv_heads=H_kv, d_k=d_k, d_v=d_v, m=d_k // d_sub, K=K, L=L)
+    keys, v = synth.make_keys(w), synth.make_values(w)
+    q = synth.make_prefill_queries(w, L_q, float(rng.choice([1.0, 0.2])))
+    books, _ = oracle.fit_codebooks(keys[:, :, :min(w.L, 300)], w.m, w.K, iters=1, seed=3)
+    codes = oracle.encode_keys(keys, books)
+    ref = oracle.attend_prefill(q, books, codes, v, q_pos0=q_pos0)
+    lk = ctx_for(w)
+    for form in ("contraction", "contraction_mma_sync"):
+        lk.lookat_set_prefill_form(form)
+        for _ in range(2):
+            out = lk.lookat_attend_prefill(dev(q), dev(books), dev(codes), dev(v), q_pos0=q_pos0)
+            assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL, (form, shape_of(w), L_q, q_pos0)
+
+
+def shape_of(w):
+    return dict(B=w.B, H_q=w.n_q_heads, H_kv=w.n_kv_heads, d_k=w.d_k, d_v=w.d_v, m=w.m, K=w.K, L=w.L)
