@@ -1,24 +1,27 @@
 // Multi-query causal attention over the compressed keys, contraction form, on the 5th-generation tensor
-// cores (Algorithm 1 applied to a tile of 128 queries).  The score of Section 3.4,
+// cores (Algorithm 1 applied to two tiles of 128 queries at a time).  The score of Section 3.4,
 //     s[q][t] = sum_j LUT_j[code[t][j]],   LUT_j[c] = q^(j) . C_j[c],
 // is the inner product of q with the key rebuilt from its codes, k^[t] = (C_1[code[t][1]], ...,
 // C_m[code[t][m]]).  A table pays when one query meets many keys; in prefill many queries meet each key,
 // so the centroids named by a chunk of 64 tokens are gathered ONCE per CTA into shared memory (the codes
-// stay the only stored form of the keys; nothing is written back to HBM) and all 128 queries take their
+// stay the only stored form of the keys; nothing is written back to HBM) and all 256 queries take their
 // scores from them with tcgen05.mma: S = Q . K^^T (fp32 in tensor memory), online softmax by one thread
 // per query row, O += P . V with P read from tensor memory.  q (fp16) is an exact operand; every fp32
 // centroid is split into two fp16 planes (rounding + remainder), which carries s to ~2^-22 relative.
 //
+// A CTA works on two tiles of 128 queries against the same chunks, one behind the other: while the softmax
+// threads of one tile work, the tensor pipe runs the other tile's MMAs, and every rebuilt chunk serves 256 queries.
 // Roles in a CTA of 15 warps (one CTA per SM; the shared memory is full):
-//   warps 0-3  softmax: thread r owns query row r = tensor-memory lane r;
-//   warps 4-11 producers: rebuild the next chunk's key rows from the codebook image in shared memory
-//              (16-byte items placed so that gathers and stores are free of bank conflicts whatever
-//              the codes are) and fetch its V rows with cp.async;
+//   warps 0-3 / 4-7  softmax of tile 0 / tile 1: thread r owns query row r of its tile = tensor-memory lane r;
+//   warps 8-11  key producers: rebuild the next chunk's key rows from the codebook image in shared memory
+//               (16-byte items placed so that gathers and stores are free of bank conflicts whatever the codes are);
 //   warps 12-13 fetch the V rows of the chunk after next with cp.async, on their own schedule;
-//   warp 14    one thread issues every MMA and commits them to mbarriers.
-// Hand-offs go through mbarriers, one per buffer where a buffer is reused, so that no waiter can fall
-// two phases behind; every wait gives up after a bounded number of polls, raises the context's timeout
-// flag and lets the CTA drain and free its tensor memory.
+//   warp 14     one thread issues every MMA and commits them to mbarriers.
+// Tensor memory (512 columns): per tile the scores of one chunk (64; the fp16 weights overwrite their first
+// half), O (d_v) and the query rows as the A operand of the score MMA (d_k / 2).
+// Hand-offs go through mbarriers, one per buffer where a buffer is reused, so that no waiter can fall two
+// phases behind; every wait gives up after a bounded number of polls, raises the context's timeout flag and
+// lets the CTA drain and free its tensor memory.
 #include "common.cuh"
 
 // Tuning aid (-DLOOKAT_PHASE_STAMPS): per role, the cycles spent in each phase of the chunk loop, averaged
@@ -39,7 +42,8 @@ namespace {
 
 constexpr int kUmRows = 128;                   // queries per CTA = rows of one MMA
 constexpr int kUmChunk = 64;                   // tokens per chunk = columns of the score MMA
-constexpr int kUmSoftmax = 128, kUmProducers = 256, kUmVLoaders = 64;
+constexpr int kUmTiles = 2;                    // query tiles per CTA
+constexpr int kUmSoftmax = kUmTiles * kUmRows, kUmProducers = 128, kUmVLoaders = 64;
 constexpr int kUmThreads = kUmSoftmax + kUmProducers + kUmVLoaders + 32;
 constexpr float kUmSlack = 8.f;                // how far a row maximum may run ahead of the softmax reference point
 constexpr int kUmPolls = 1 << 20;              // bound of every mbarrier wait
@@ -165,22 +169,21 @@ __global__ void um_codebook_image_kernel(const float *__restrict__ books, __half
 template <int D_K, int D_V>
 struct UmLayout {
     static constexpr int kKb = D_K / 64, kNb = D_V / 64;               // 128-byte blocks per key row / V row
-    static constexpr int kKeys = kKb * 2 * kUmChunk * 128;             // [kb][64 hi rows, 64 lo rows][128 B]: one operand of 128 rows
+    static constexpr int kKeys = kKb * 2 * kUmChunk * 128;             // [kb][64 hi rows, 64 lo rows][128 B]
     static constexpr int kV = kNb * kUmChunk * 128;                    // [nb][64 tokens][128 B]
     static constexpr int kOffKeys = 0, kOffV = 2 * kKeys, kOffBook = kOffV + 2 * kV;   // two key buffers, two V buffers
     static constexpr int kIds = D_K / 4;                               // 16-byte items per key row, both planes
     static constexpr int kItems = kUmChunk * kIds / kUmProducers;      // items rebuilt per producer thread per chunk
-    static_assert(kUmChunk * kIds % kUmProducers == 0 && kItems % 4 == 0, "whole items per thread, four codes per word");
+    static_assert(kUmChunk * kIds % kUmProducers == 0, "whole items per thread");
     static size_t book_bytes(int K) { return (size_t)K * D_K * 4; }
-    // operands, codebook image, then barriers, the tensor-memory address and the codes of two chunks
-    // ... then barriers (256 B) and the codes of two chunks (2 KB)
+    // operands, codebook image, then barriers (256 B) and the codes of two chunks (2 KB)
     static size_t bytes(int K) { return (size_t)kOffBook + book_bytes(K) + 256 + 2048; }
-    static constexpr int kColS = 2 * kUmChunk;                         // one score buffer: hi-plane sums | lo-plane sums
-    static constexpr int kColP = 2 * kColS;                            // weights of one chunk: 64 fp16, two per column
-    static constexpr int kColO = kColP + 2 * (kUmChunk / 2), kColQ = kColO + D_V;   // columns: S0 | S1 | P0 | P1 | O (D_V) | Q (D_K / 2)
-    static constexpr int kTmemCols = kColQ + D_K / 2 <= 256 ? 256 : 512;
+    // tensor-memory columns: S of tile 0, 1 (64 each; P over their first halves) | O of tile 0, 1 | Q of tile 0, 1
+    static constexpr int kColO = kUmTiles * kUmChunk, kColQ = kColO + kUmTiles * D_V;
+    static constexpr int kTmemCols = kColQ + kUmTiles * (D_K / 2) <= 256 ? 256 : 512;
+    static_assert(kColQ + kUmTiles * (D_K / 2) <= 512, "tensor memory");
     // instruction descriptors: fp32 accumulate, fp16 operands, N >> 3 at bit 17, M >> 4 at bit 24; bit 16: B is MN-major
-    static constexpr uint32_t kIdescS = (1u << 4) | ((uint32_t)(2 * kUmChunk >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
+    static constexpr uint32_t kIdescS = (1u << 4) | ((uint32_t)(kUmChunk >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
     static constexpr uint32_t kIdescO = (1u << 4) | (1u << 16) | ((uint32_t)(D_V >> 3) << 17) | ((uint32_t)(kUmRows >> 4) << 24);
 };
 
@@ -197,20 +200,20 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
     uint64_t *const bars = reinterpret_cast<uint64_t *>(book + book_bytes);
     uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(bars + 30);
     uint8_t *const codes_s = reinterpret_cast<uint8_t *>(bars + 32);  // [2][1024]: the codes of two chunks
-    // barriers, one per buffer: k_ready[2], v_ready[2] (keys / V staged), s_full[2] (scores done), pv_done[2] (value MMA
-    // done), p_ready[2] (weights stored)
+    // barriers: k_ready[buf], v_ready[buf] (keys / V of a chunk staged); per tile s_full[t][buf] (scores done),
+    // pv_done[t][buf] (value MMA done), p_ready[t] (weights stored)
     const uint32_t bar0 = um_smem(bars);
-    const uint32_t bar_k = bar0, bar_v = bar0 + 16, bar_s = bar0 + 32, bar_pv = bar0 + 48, bar_p = bar0 + 64;
+    const uint32_t bar_k = bar0, bar_v = bar0 + 16, bar_s = bar0 + 32, bar_pv = bar0 + 64, bar_p = bar0 + 96;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int n_tiles = (int)((a.L_q + kUmRows - 1) / kUmRows);
-    const int tile = n_tiles - 1 - (int)blockIdx.x;            // longest tiles first
+    const int n_super = (int)((a.L_q + kUmTiles * kUmRows - 1) / (kUmTiles * kUmRows));
+    const int super = n_super - 1 - (int)blockIdx.x;           // longest first
     const int hq = blockIdx.y, b = blockIdx.z, h = hq / a.g;
     const int d_sub = D_K / a.m;
 
-    const long long row0 = (long long)tile * kUmRows;
-    const long long t_end = a.q_pos0 + (row0 + kUmRows < a.L_q ? row0 + kUmRows : a.L_q);   // tokens the tile sees
-    const int n_chunks = (int)((t_end + kUmChunk - 1) / kUmChunk);
+    const long long row0 = (long long)super * (kUmTiles * kUmRows);
+    const long long t_end = a.q_pos0 + (row0 + kUmTiles * kUmRows < a.L_q ? row0 + kUmTiles * kUmRows : a.L_q);   // tokens the CTA sees
+    const int n_chunks = (int)((t_end + kUmChunk - 1) / kUmChunk);     // both tiles walk all of them (tile 0: up to two all masked)
 
     // ---- prologue, all threads: codebook image into shared memory, barriers, tensor memory ----
     {
@@ -221,9 +224,11 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             for (int i = 0; i < 2; ++i) {
                 um_bar_init(bar_k + 8 * i, kUmProducers);
                 um_bar_init(bar_v + 8 * i, kUmVLoaders);
-                um_bar_init(bar_s + 8 * i, 1);
-                um_bar_init(bar_pv + 8 * i, 1);
-                um_bar_init(bar_p + 8 * i, kUmSoftmax);
+                for (int t = 0; t < kUmTiles; ++t) {
+                    um_bar_init(bar_s + 16 * t + 8 * i, 1);
+                    um_bar_init(bar_pv + 16 * t + 8 * i, 1);
+                }
+                um_bar_init(bar_p + 8 * i, kUmRows);           // i as the tile index here
             }
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
@@ -240,12 +245,13 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         um_fence_after();
     }
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tm_s = tmem, tm_p = tmem + Lay::kColP, tm_o = tmem + Lay::kColO, tm_q = tmem + Lay::kColQ;
     bool dead = (sm0 & 1023u) != 0;                            // a wait ran out (or the base is misaligned): leave, free, return
 
     // ---- the query rows go to tensor memory as the A operand of the score MMA: lane r = row r, two halfs per column ----
-    if (warp < 4) {                                            // one thread per row
-        const long long qr = row0 + tid < a.L_q ? row0 + tid : a.L_q - 1;       // rows beyond L_q repeat the last one
+    if (warp < kUmSoftmax / 32) {                              // one thread per row of each tile
+        const int t = warp >> 2, r = (warp & 3) * 32 + lane;
+        const long long want = row0 + t * kUmRows + r;
+        const long long qr = want < a.L_q ? want : a.L_q - 1;  // rows beyond L_q repeat the last one
         const uint4 *src = reinterpret_cast<const uint4 *>(a.q + ((size_t)(b * a.H_q + hq) * a.L_q + qr) * D_K);
 #pragma unroll
         for (int part = 0; part < D_K / 64; ++part) {
@@ -258,7 +264,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                 w[4 * i + 2] = x.z;
                 w[4 * i + 3] = x.w;
             }
-            um_st32(tm_q + part * 32 + ((uint32_t)(warp * 32) << 16), w);
+            um_st32(tmem + Lay::kColQ + t * (D_K / 2) + part * 32 + ((uint32_t)((warp & 3) * 32) << 16), w);
         }
         um_wait_st();
     }
@@ -276,55 +282,62 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
             const uint32_t keys_lo = ((sm0 + Lay::kOffKeys) >> 4) | (1u << 16);                    // leading offset unused (16 B)
             const uint32_t v_lo = ((sm0 + Lay::kOffV) >> 4) | ((uint32_t)(kUmChunk * 128 / 16) << 16);   // between 64-column blocks
-            auto score_mma = [&](int c) {                      // S[c & 1] = Q . [K^hi(c); K^lo(c)]^T: 64 + 64 columns
+            auto score_mma = [&](int t, int c) {               // S(t) = Q(t) . K^(c)^T: the hi plane, then the lo plane on top
                 const int buf = c & 1;
-                const uint32_t lo = keys_lo + buf * (Lay::kKeys >> 4), d = tm_s + buf * Lay::kColS;
+                const uint32_t lo = keys_lo + buf * (Lay::kKeys >> 4), d = tmem + t * kUmChunk, q = tmem + Lay::kColQ + t * (D_K / 2);
 #pragma unroll
-                for (int ks = 0; ks < D_K / 16; ++ks) {            // 128 operand rows: the hi and the lo plane of 64 tokens
-                    const uint32_t off = ((ks >> 2) * (2 * kUmChunk * 128) + (ks & 3) * 32) >> 4;
-                    if (ks == 0) um_mma_ts<false>(d, tm_q + ks * 8, lo + off, desc_hi, Lay::kIdescS);
-                    else um_mma_ts<true>(d, tm_q + ks * 8, lo + off, desc_hi, Lay::kIdescS);
-                }
-                um_commit(bar_s + 8 * buf);
+                for (int plane = 0; plane < 2; ++plane)
+#pragma unroll
+                    for (int ks = 0; ks < D_K / 16; ++ks) {
+                        const uint32_t off = ((ks >> 2) * (2 * kUmChunk * 128) + plane * (kUmChunk * 128) + (ks & 3) * 32) >> 4;
+                        if (plane == 0 && ks == 0) um_mma_ts<false>(d, q + ks * 8, lo + off, desc_hi, Lay::kIdescS);
+                        else um_mma_ts<true>(d, q + ks * 8, lo + off, desc_hi, Lay::kIdescS);
+                    }
+                um_commit(bar_s + 16 * t + 8 * buf);
             };
-            auto value_mma = [&](int c) {                      // O += P(c) . V(c), P read from tensor memory
+            auto value_mma = [&](int t, int c) {               // O(t) += P(t, c) . V(c), P read from the first half of S(t)
                 const int buf = c & 1;
-                const uint32_t lo = v_lo + buf * (Lay::kV >> 4), pa = tm_p + buf * (kUmChunk / 2);
+                const uint32_t lo = v_lo + buf * (Lay::kV >> 4), pa = tmem + t * kUmChunk, d = tmem + Lay::kColO + t * D_V;
 #pragma unroll
                 for (int kt = 0; kt < kUmChunk / 16; ++kt) {   // 16 tokens: 8 columns of weights, two 8-token groups of V
-                    if (kt == 0 && c == 0) um_mma_ts<false>(tm_o, pa + kt * 8, lo + kt * (2048 >> 4), desc_hi, Lay::kIdescO);
-                    else um_mma_ts<true>(tm_o, pa + kt * 8, lo + kt * (2048 >> 4), desc_hi, Lay::kIdescO);
+                    if (kt == 0 && c == 0) um_mma_ts<false>(d, pa + kt * 8, lo + kt * (2048 >> 4), desc_hi, Lay::kIdescO);
+                    else um_mma_ts<true>(d, pa + kt * 8, lo + kt * (2048 >> 4), desc_hi, Lay::kIdescO);
                 }
-                um_commit(bar_pv + 8 * buf);
+                um_commit(bar_pv + 16 * t + 8 * buf);
             };
-            // Whichever is ready goes first: the scores of chunk next_qk (its keys are staged and the value MMA
-            // that read the previous weights of that buffer has been issued) or the value MMA of chunk next_pv
-            // (its weights are stored and its V rows have landed).
-            int next_qk = 0, next_pv = 0;
+            // Per tile strictly scores(c) -> [softmax] -> value(c) -> scores(c + 1) (the weights overwrite the scores);
+            // the two tiles take turns, so the pipe has the other tile's MMAs while one tile's softmax runs.
+            int next_qk[kUmTiles] = {0, 0}, next_pv[kUmTiles] = {0, 0};
             long long polls = 0;
             UM_STAMPS(mm, 3)
-            while (next_pv < n_chunks) {
+            while (next_pv[0] < n_chunks || next_pv[1] < n_chunks) {
                 bool progress = false;
-                if (next_qk < n_chunks && next_qk - next_pv < 2 && um_bar_test(bar_k + 8 * (next_qk & 1), (next_qk >> 1) & 1)) {
-                    UM_STAMP(mm, 0)
-                    um_fence_after();
-                    score_mma(next_qk++);
-                    progress = true;
-                    UM_STAMP(mm, 1)
-                }
-                if (next_pv < next_qk && um_bar_test(bar_p + 8 * (next_pv & 1), (next_pv >> 1) & 1) &&
-                    um_bar_test(bar_v + 8 * (next_pv & 1), (next_pv >> 1) & 1)) {
-                    UM_STAMP(mm, 0)
-                    um_fence_after();
-                    value_mma(next_pv++);
-                    progress = true;
-                    UM_STAMP(mm, 2)
+#pragma unroll
+                for (int t = 0; t < kUmTiles; ++t) {
+                    const int cq = next_qk[t];
+                    if (cq < n_chunks && next_pv[t] == cq && um_bar_test(bar_k + 8 * (cq & 1), (cq >> 1) & 1)) {
+                        UM_STAMP(mm, 0)
+                        um_fence_after();
+                        score_mma(t, cq);
+                        next_qk[t] = cq + 1;
+                        progress = true;
+                        UM_STAMP(mm, 1)
+                    }
+                    const int cp = next_pv[t];
+                    if (cp < next_qk[t] && um_bar_test(bar_p + 8 * t, cp & 1) && um_bar_test(bar_v + 8 * (cp & 1), (cp >> 1) & 1)) {
+                        UM_STAMP(mm, 0)
+                        um_fence_after();
+                        value_mma(t, cp);
+                        next_pv[t] = cp + 1;
+                        progress = true;
+                        UM_STAMP(mm, 2)
+                    }
                 }
                 if (progress) polls = 0;
                 else if (++polls > kUmPolls) { dead = true; break; }
             }
 #ifdef LOOKAT_PHASE_STAMPS
-            if (UM_FIRST_CTA) printf("mma thread: idle %lld, score issue %lld, value issue %lld cycles per chunk\n", mm[0] / n_chunks, mm[1] / n_chunks, mm[2] / n_chunks);
+            if (UM_FIRST_CTA) printf("mma thread: idle %lld, score issue %lld, value issue %lld cycles per chunk (both tiles)\n", mm[0] / n_chunks, mm[1] / n_chunks, mm[2] / n_chunks);
 #endif
         }
     } else if (warp >= kUmSoftmax / 32 && warp < (kUmSoftmax + kUmProducers) / 32) {
@@ -339,7 +352,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         const int tl0 = ptid / Lay::kIds;                      // this thread's tokens of a chunk: tl0 + i * (producers / kIds)
         constexpr int kTokStep = kUmProducers / Lay::kIds;
         const int code_bytes = kUmChunk * a.m;                 // codes of one chunk, staged in shared memory a chunk ahead
-        auto fetch_codes = [&](int c) {                        // 4-byte cp.async pieces; pieces beyond the tile's tokens stay unread
+        auto fetch_codes = [&](int c) {                        // 4-byte cp.async pieces; pieces beyond the CTA's tokens stay unread
             const long long first = (long long)c * code_bytes, limit = t_end * a.m;
             for (int o = ptid * 4; o < code_bytes; o += kUmProducers * 4)
                 if (first + o + 4 <= limit)
@@ -350,22 +363,25 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         // key rows of chunk c into key buffer c & 1: one 16-byte item of the codebook image per (token, 8-dim group, plane)
         auto rebuild_keys = [&](int c) {
             const int buf = c & 1;
-            const bool whole = (long long)(c + 1) * kUmChunk <= t_end;   // every token of the chunk is visible to the tile
+            const bool whole = (long long)(c + 1) * kUmChunk <= t_end;   // every token of the chunk is visible to the CTA
             const uint8_t *cs = codes_s + buf * 1024 + my_j;
-            uint32_t code[Lay::kItems];
-            uint4 item[Lay::kItems];
 #pragma unroll
-            for (int i = 0; i < Lay::kItems; ++i) code[i] = cs[(tl0 + i * kTokStep) * a.m];
+            for (int half = 0; half < 2; ++half) {             // in two batches: all loads of a batch before its stores
+                uint32_t code[Lay::kItems / 2];
+                uint4 item[Lay::kItems / 2];
 #pragma unroll
-            for (int i = 0; i < Lay::kItems; ++i) {            // all loads before any store: they overlap
-                item[i] = make_uint4(0u, 0u, 0u, 0u);
-                if (whole || (long long)c * kUmChunk + tl0 + i * kTokStep < t_end)
-                    item[i] = *reinterpret_cast<const uint4 *>(my_src + code[i] * 128);
-            }
+                for (int i = 0; i < Lay::kItems / 2; ++i) code[i] = cs[(tl0 + (half * (Lay::kItems / 2) + i) * kTokStep) * a.m];
 #pragma unroll
-            for (int i = 0; i < Lay::kItems; ++i) {
-                const int tl = tl0 + i * kTokStep;
-                *reinterpret_cast<uint4 *>(my_dst + buf * Lay::kKeys + tl * 128 + (((my_gi & 7) ^ (tl & 7)) << 4)) = item[i];
+                for (int i = 0; i < Lay::kItems / 2; ++i) {
+                    item[i] = make_uint4(0u, 0u, 0u, 0u);
+                    if (whole || (long long)c * kUmChunk + tl0 + (half * (Lay::kItems / 2) + i) * kTokStep < t_end)
+                        item[i] = *reinterpret_cast<const uint4 *>(my_src + code[i] * 128);
+                }
+#pragma unroll
+                for (int i = 0; i < Lay::kItems / 2; ++i) {
+                    const int tl = tl0 + (half * (Lay::kItems / 2) + i) * kTokStep;
+                    *reinterpret_cast<uint4 *>(my_dst + buf * Lay::kKeys + tl * 128 + (((my_gi & 7) ^ (tl & 7)) << 4)) = item[i];
+                }
             }
             um_fence_async_smem();                             // generic-proxy writes before the MMA's reads
             um_bar_arrive(bar_k + 8 * buf);
@@ -377,10 +393,16 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");
         rebuild_keys(0);
         asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");   // everyone is done with the codes of chunk 0
-        // keys of chunk c into the buffer that the score MMA of chunk c - 2 has released; codes two chunks ahead
+        // keys of chunk c into the buffer that the score MMAs of chunk c - 2 (both tiles) have released
         UM_STAMPS(pp, 3)
         for (int c = 1; c < n_chunks; ++c) {
-            if (c >= 2 && !um_group_wait<1, kUmProducers>(ptid == 0, bar_s + 8 * (c & 1), ((c - 2) >> 1) & 1)) { dead = true; break; }
+            if (c >= 2) {
+                bool ok = true;
+#pragma unroll
+                for (int t = 0; t < kUmTiles; ++t)
+                    ok = um_group_wait<1, kUmProducers>(ptid == 0, bar_s + 16 * t + 8 * (c & 1), ((c - 2) >> 1) & 1) && ok;
+                if (!ok) { dead = true; break; }
+            }
             UM_STAMP(pp, 0)
             rebuild_keys(c);
             UM_STAMP(pp, 1)
@@ -401,8 +423,14 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         UM_STAMPS(vv, 3)
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
-            // the V buffer of chunk c - 2 is free once its value MMA is done
-            if (c >= 2 && !um_group_wait<2, kUmVLoaders>(vtid == 0, bar_pv + 8 * buf, ((c - 2) >> 1) & 1)) { dead = true; break; }
+            // the V buffer of chunk c - 2 is free once both tiles' value MMAs of that chunk are done
+            if (c >= 2) {
+                bool ok = true;
+#pragma unroll
+                for (int t = 0; t < kUmTiles; ++t)
+                    ok = um_group_wait<2, kUmVLoaders>(vtid == 0, bar_pv + 16 * t + 8 * buf, ((c - 2) >> 1) & 1) && ok;
+                if (!ok) { dead = true; break; }
+            }
             UM_STAMP(vv, 0)
             // V rows by cp.async: [nb][token][128 B], 16-byte pieces swizzled by token
             const bool whole = (long long)(c + 1) * kUmChunk <= t_end;
@@ -426,31 +454,30 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         if (UM_FIRST_CTA && vtid == 0) printf("V loaders: wait V buffer %lld, issue %lld, land %lld\n", vv[0] / n_chunks, vv[1] / n_chunks, vv[2] / n_chunks);
 #endif
     } else {
-        // =================== softmax: thread r owns query row r (tensor-memory lane r) ===================
-        const long long row = row0 + tid;
+        // =================== softmax of tile t: thread r owns query row r of the tile (tensor-memory lane r) ===================
+        const int t = warp >> 2, rq = warp & 3, r = rq * 32 + lane;
+        const long long row = row0 + t * kUmRows + r;
         const long long vis_end = a.q_pos0 + (row < a.L_q ? row : a.L_q - 1) + 1;    // tokens this row sees
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const uint32_t lane_base = (uint32_t)(rq * 32) << 16;
+        const uint32_t tm_s = tmem + t * kUmChunk + lane_base, tm_o = tmem + Lay::kColO + t * D_V + lane_base;
         float m_run = -INFINITY, l_run = 0.f;                  // reference point (base-2 exponent units) and row sum
-        UM_STAMPS(ss, 5)
+        UM_STAMPS(ss, 4)
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
             const long long tok0 = (long long)c * kUmChunk;
-            if (!__all_sync(0xffffffffu, um_bar_wait(bar_s + 8 * buf, (c >> 1) & 1))) { dead = true; break; }   // warp-uniform
+            if (!__all_sync(0xffffffffu, um_bar_wait(bar_s + 16 * t + 8 * buf, (c >> 1) & 1))) { dead = true; break; }   // warp-uniform
             um_fence_after();
             UM_STAMP(ss, 0)
-            float sc[kUmChunk];                                // raw scores: hi-plane sum + lo-plane sum
+            float sc[kUmChunk];                                // raw scores
             {
-                uint32_t h0[32], l0[32], h1[32], l1[32];
-                const uint32_t at = tm_s + buf * Lay::kColS + lane_base;
-                um_ld32(h0, at);
-                um_ld32(l0, at + kUmChunk);
-                um_ld32(h1, at + 32);
-                um_ld32(l1, at + kUmChunk + 32);
+                uint32_t s0[32], s1[32];
+                um_ld32(s0, tm_s);
+                um_ld32(s1, tm_s + 32);
                 um_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
-                    sc[i] = __uint_as_float(h0[i]) + __uint_as_float(l0[i]);
-                    sc[32 + i] = __uint_as_float(h1[i]) + __uint_as_float(l1[i]);
+                    sc[i] = __uint_as_float(s0[i]);
+                    sc[32 + i] = __uint_as_float(s1[i]);
                 }
             }
             if (SCORES && a.scores_out && row < a.L_q) {
@@ -459,7 +486,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                 for (int i = 0; i < kUmChunk; ++i)
                     if (tok0 + i < vis_end) dst[i] = sc[i];
             }
-            if (tok0 + kUmChunk > vis_end) {                   // the chunk crosses this row's causal limit
+            if (tok0 + kUmChunk > vis_end) {                   // the chunk crosses (or lies beyond) this row's causal limit
 #pragma unroll
                 for (int i = 0; i < kUmChunk; ++i)
                     if (tok0 + i >= vis_end) sc[i] = -INFINITY;
@@ -487,40 +514,36 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             }
             l_run = l_run * alpha + sum;
             UM_STAMP(ss, 1)
-            if (c >= 1) {
-                // the previous value MMA must be done before O is rescaled; the one before it has released this P buffer
-                if (!__all_sync(0xffffffffu, um_bar_wait(bar_pv + 8 * (buf ^ 1), ((c - 1) >> 1) & 1))) { dead = true; break; }
-                um_fence_after();
-                UM_STAMP(ss, 2)
-                if (__any_sync(0xffffffffu, alpha != 1.f)) {   // a reference point moved in this warp's rows: rescale them
+            // The tile's previous value MMA is complete: the commit behind s_full covers every MMA its thread issued
+            // before, and value(c - 1) was issued before scores(c).  So O may be rescaled right away.
+            if (c >= 1 && __any_sync(0xffffffffu, alpha != 1.f)) {   // a reference point moved in this warp's rows
 #pragma unroll 1
-                    for (int part = 0; part < D_V / 32; ++part) {
-                        uint32_t o[32];
-                        um_ld32(o, tm_o + part * 32 + lane_base);
-                        um_wait_ld();
+                for (int part = 0; part < D_V / 32; ++part) {
+                    uint32_t o[32];
+                    um_ld32(o, tm_o + part * 32);
+                    um_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        um_st32(tm_o + part * 32 + lane_base, o);
-                    }
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    um_st32(tm_o + part * 32, o);
                 }
             }
-            UM_STAMP(ss, 3)
-            um_st32(tm_p + buf * (kUmChunk / 2) + lane_base, pk);   // the 64 weights, two per column
+            UM_STAMP(ss, 2)
+            um_st32(tm_s, pk);                                 // the 64 weights over the first half of the scores, two per column
             um_wait_st();
             um_fence_before();
-            um_bar_arrive(bar_p + 8 * buf);
-            UM_STAMP(ss, 4)
+            um_bar_arrive(bar_p + 8 * t);
+            UM_STAMP(ss, 3)
         }
 #ifdef LOOKAT_PHASE_STAMPS
-        if (UM_FIRST_CTA && tid == 0) printf("softmax: wait scores %lld, load + exp %lld, wait value MMA %lld, rescale %lld, store %lld (%d chunks)\n", ss[0] / n_chunks, ss[1] / n_chunks, ss[2] / n_chunks, ss[3] / n_chunks, ss[4] / n_chunks, n_chunks);
+        if (UM_FIRST_CTA && (tid == 0 || tid == kUmRows)) printf("softmax of tile %d: wait scores %lld, load + exp %lld, rescale %lld, store %lld (%d chunks)\n", t, ss[0] / n_chunks, ss[1] / n_chunks, ss[2] / n_chunks, ss[3] / n_chunks, n_chunks);
 #endif
-        if (!dead && __all_sync(0xffffffffu, um_bar_wait(bar_pv + 8 * ((n_chunks - 1) & 1), ((n_chunks - 1) >> 1) & 1))) {
+        if (!dead && __all_sync(0xffffffffu, um_bar_wait(bar_pv + 16 * t + 8 * ((n_chunks - 1) & 1), ((n_chunks - 1) >> 1) & 1))) {
             um_fence_after();
             const float inv = 1.f / l_run;
 #pragma unroll 1
             for (int part = 0; part < D_V / 32; ++part) {
                 uint32_t o[32];
-                um_ld32(o, tm_o + part * 32 + lane_base);
+                um_ld32(o, tm_o + part * 32);
                 um_wait_ld();
                 if (row < a.L_q) {
                     float4 *dst = reinterpret_cast<float4 *>(a.out + ((size_t)(b * a.H_q + hq) * a.L_q + row) * D_V + part * 32);
@@ -555,7 +578,7 @@ lookat_status launch_um(Ctx *ctx, const PrefillArgs &a)
     st = check_launch(ctx, "um_codebook_image_kernel");
     if (st != LOOKAT_OK) return st;
 
-    const int n_tiles = (int)((a.L_q + kUmRows - 1) / kUmRows);
+    const int n_tiles = (int)((a.L_q + kUmTiles * kUmRows - 1) / (kUmTiles * kUmRows));   // CTAs per (row, head)
     const int smem = (int)Lay::bytes(a.K);
     dim3 grid((unsigned)n_tiles, (unsigned)a.H_q, (unsigned)a.B);
     auto launch = [&](auto kern) -> lookat_status {
@@ -578,7 +601,7 @@ bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a)
                          (a.L_max * a.m) % 4 == 0;
     // the row maxima are taken on the raw scores, which needs a positive softmax scale
     if (!shape || !aligned || a.H_q > 65535 || a.B > 65535 || !(a.scale_log2 > 0.f) || !ctx->timeout_flag) return false;
-    const size_t operands = (size_t)kUmRows * a.d_k * 2 + 2 * (size_t)kUmChunk * a.d_k * 2 + 2 * (size_t)kUmChunk * a.d_v * 2;
+    const size_t operands = 2 * (size_t)kUmChunk * a.d_k * 4 + 2 * (size_t)kUmChunk * a.d_v * 2;   // two key tiles (two planes), two V tiles
     return operands + (size_t)a.K * a.d_k * 4 + 256 + 2048 <= (size_t)ctx->max_smem_optin;
 }
 
