@@ -313,16 +313,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             while (next_pv[0] < n_chunks || next_pv[1] < n_chunks) {
                 bool progress = false;
 #pragma unroll
-                for (int t = 0; t < kUmTiles; ++t) {
-                    const int cq = next_qk[t];
-                    if (cq < n_chunks && next_pv[t] == cq && um_bar_test(bar_k + 8 * (cq & 1), (cq >> 1) & 1)) {
-                        UM_STAMP(mm, 0)
-                        um_fence_after();
-                        score_mma(t, cq);
-                        next_qk[t] = cq + 1;
-                        progress = true;
-                        UM_STAMP(mm, 1)
-                    }
+                for (int t = 0; t < kUmTiles; ++t) {           // value MMAs first: they release a tile's next scores
                     const int cp = next_pv[t];
                     if (cp < next_qk[t] && um_bar_test(bar_p + 8 * t, cp & 1) && um_bar_test(bar_v + 8 * (cp & 1), (cp >> 1) & 1)) {
                         UM_STAMP(mm, 0)
@@ -331,6 +322,15 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                         next_pv[t] = cp + 1;
                         progress = true;
                         UM_STAMP(mm, 2)
+                    }
+                    const int cq = next_qk[t];
+                    if (cq < n_chunks && next_pv[t] == cq && um_bar_test(bar_k + 8 * (cq & 1), (cq >> 1) & 1)) {
+                        UM_STAMP(mm, 0)
+                        um_fence_after();
+                        score_mma(t, cq);
+                        next_qk[t] = cq + 1;
+                        progress = true;
+                        UM_STAMP(mm, 1)
                     }
                 }
                 if (progress) polls = 0;
