@@ -257,6 +257,16 @@ enum {
 };
 lookat_status lookat_set_prefill_form(lookat_ctx *ctx, int32_t form);
 
+/*
+ * Self-test of the time-out status: launches a one-warp kernel whose only wait
+ * can never be satisfied and gives up after 4096 polls (it ends by itself in
+ * microseconds; nothing hangs), raising the context's time-out flag exactly as
+ * a prefill kernel would.  After the stream has drained, the next
+ * lookat_attend_prefill returns LOOKAT_ERR_TIMEOUT once and clears the flag.
+ * The paper has no counterpart.
+ */
+lookat_status lookat_selftest_timeout(lookat_ctx *ctx);
+
 /* Number of kernels this context has launched since it was created. */
 uint64_t lookat_kernel_launches(const lookat_ctx *ctx);
 

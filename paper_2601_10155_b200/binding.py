@@ -20,7 +20,7 @@ EXPORTS = [
     "lookat_create", "lookat_destroy", "lookat_last_error", "lookat_fit_codebooks",
     "lookat_encode_keys", "lookat_build_lut", "lookat_attend", "lookat_attend_static",
     "lookat_attend_prefill", "lookat_decode_step", "lookat_decode_step_host",
-    "lookat_kernel_launches", "lookat_set_prefill_form", "lookat_set_timing", "lookat_attend_kernel_ms",
+    "lookat_kernel_launches", "lookat_selftest_timeout", "lookat_set_prefill_form", "lookat_set_timing", "lookat_attend_kernel_ms",
 ]
 
 STATUS = {0: "LOOKAT_OK", 1: "LOOKAT_ERR_INVALID_ARG", 2: "LOOKAT_ERR_UNSUPPORTED",
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
     lib.lookat_decode_step_host.restype = ctypes.c_int
     lib.lookat_kernel_launches.argtypes = [vp]
     lib.lookat_kernel_launches.restype = ctypes.c_uint64
+    lib.lookat_selftest_timeout.argtypes = [vp]
+    lib.lookat_selftest_timeout.restype = i32
     lib.lookat_set_prefill_form.argtypes = [vp, i32]
     lib.lookat_set_prefill_form.restype = i32
     lib.lookat_set_timing.argtypes = [vp, i32]
@@ -280,6 +282,9 @@ class Lookat:
 
     def lookat_kernel_launches(self) -> int:
         return int(self._lib.lookat_kernel_launches(self._h))
+
+    def lookat_selftest_timeout(self):
+        self._check(self._lib.lookat_selftest_timeout(self._h))
 
     def lookat_set_prefill_form(self, form):
         """form: 'auto', 'tables', 'contraction' or 'contraction_mma_sync' (or the header's integer values)."""

@@ -302,6 +302,14 @@ lookat_status lookat_set_prefill_form(lookat_ctx *handle, int32_t form)
     return LOOKAT_OK;
 }
 
+lookat_status lookat_selftest_timeout(lookat_ctx *handle)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    DeviceGuard guard(ctx->device);
+    return launch_timeout_selftest(ctx);
+}
+
 void lookat_set_timing(lookat_ctx *handle, int32_t enabled)
 {
     if (!handle) return;

@@ -121,6 +121,7 @@ lookat_status launch_prefill_mma(Ctx *ctx, const PrefillArgs &a);
 // the same on tcgen05 with accumulators in tensor memory (prefill_umma.cu)
 bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a);
 lookat_status launch_prefill_umma(Ctx *ctx, const PrefillArgs &a);
+lookat_status launch_timeout_selftest(Ctx *ctx);
 
 lookat_status launch_build_lut(Ctx *ctx, const __half *q, int B, const float *codebooks, float *lut);
 

@@ -58,10 +58,10 @@ __device__ __forceinline__ void um_bar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// false after kUmPolls unsuccessful polls
-__device__ __forceinline__ bool um_bar_wait(uint32_t bar, uint32_t parity)
+// false after `polls` unsuccessful polls
+__device__ __forceinline__ bool um_bar_wait(uint32_t bar, uint32_t parity, int polls = kUmPolls)
 {
-    for (int it = 0; it < kUmPolls; ++it) {
+    for (int it = 0; it < polls; ++it) {
         uint32_t ok;
         asm volatile(
             "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
@@ -565,6 +565,18 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(Lay::kTmemCols) : "memory");
 }
 
+// A wait that nothing will ever satisfy, with a short limit: exercises the path wait-ran-out -> flag -> host status
+// without hanging anything (the bounded loop ends by itself after 4096 polls).
+__global__ void um_timeout_selftest_kernel(int *__restrict__ timeout_flag)
+{
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        um_bar_init(um_smem(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!um_bar_wait(um_smem(&bar), 0, 4096)) atomicExch(timeout_flag, 1);
+    }
+}
+
 template <int D_K, int D_V>
 lookat_status launch_um(Ctx *ctx, const PrefillArgs &a)
 {
@@ -603,6 +615,13 @@ bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a)
     if (!shape || !aligned || a.H_q > 65535 || a.B > 65535 || !(a.scale_log2 > 0.f) || !ctx->timeout_flag) return false;
     const size_t operands = 2 * (size_t)kUmChunk * a.d_k * 4 + 2 * (size_t)kUmChunk * a.d_v * 2;   // two key tiles (two planes), two V tiles
     return operands + (size_t)a.K * a.d_k * 4 + 256 + 2048 <= (size_t)ctx->max_smem_optin;
+}
+
+lookat_status launch_timeout_selftest(Ctx *ctx)
+{
+    if (!ctx->timeout_flag) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "no time-out flag on this context");
+    um_timeout_selftest_kernel<<<1, 32, 0, ctx->stream>>>(ctx->timeout_flag);
+    return check_launch(ctx, "um_timeout_selftest_kernel");
 }
 
 lookat_status launch_prefill_umma(Ctx *ctx, const PrefillArgs &a)

@@ -471,3 +471,25 @@ def test_attend_prefill_contraction_on_random_shapes(seed):
 
 def shape_of(w):
     return dict(B=w.B, H_q=w.n_q_heads, H_kv=w.n_kv_heads, d_k=w.d_k, d_v=w.d_v, m=w.m, K=w.K, L=w.L)
+
+
+def test_a_wait_that_runs_out_is_reported_once_and_the_context_stays_usable():
+    """The bounded-wait status, without hanging anything: a self-test kernel's only wait can never be satisfied and
+    gives up after 4096 polls; the next prefill call reports the time-out and clears it; the one after runs."""
+    w = synth.small_workload(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=64, m=8, K=64, L=200)
+    keys, v = synth.make_keys(w), synth.make_values(w)
+    q = synth.make_prefill_queries(w, 100, 1.0)
+    books, _ = oracle.fit_codebooks(keys[:, :, :200], w.m, w.K, iters=1, seed=3)
+    codes = oracle.encode_keys(keys, books)
+    ref = oracle.attend_prefill(q, books, codes, v, q_pos0=100)
+    lk = ctx_for(w)
+    args = (dev(q), dev(books), dev(codes), dev(v))
+    out = lk.lookat_attend_prefill(*args, q_pos0=100)
+    assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
+    lk.lookat_selftest_timeout()
+    torch.cuda.synchronize()
+    with pytest.raises(LookatError) as err:
+        lk.lookat_attend_prefill(*args, q_pos0=100)
+    assert err.value.status == 5                                   # LOOKAT_ERR_TIMEOUT
+    out = lk.lookat_attend_prefill(*args, q_pos0=100)              # reported once; the context is usable
+    assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
