@@ -285,6 +285,39 @@ def time_prefill(device_index: int, steps: int = 5, batch: int = 0, heads: int =
     return res
 
 
+def time_encode_1m(device_index: int):
+    """Bulk encoding at the size of BASELINE config 4: one KV head, 1,048,576 keys of d = 128, m = 16 (d_sub 8),
+    codebooks = the seeded start rule on the first 262,144 keys (no Lloyd iteration); then a refit of 10 iterations
+    on those 262,144 keys.  Bounds: HBM (keys in, codes out) and the tensor pipe (2 fp16 planes per centroid)."""
+    import torch
+
+    from paper_2601_10155_b200.binding import Lookat
+    w = synth.WORKLOADS["encode_1m_m16"]
+    lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K, device=device_index)
+    keys = torch.from_numpy(np.ascontiguousarray(synth.make_keys(w))).cuda()
+    sample = keys[:, :, :w.fit_keys_per_head].contiguous()
+    books0 = lk.lookat_fit_codebooks(sample, 0, seed=w.seed)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    for attempt in range(2):                               # the second pass is timed
+        ev[0].record()
+        codes = lk.lookat_encode_keys(keys, books0)
+        ev[1].record()
+        books = lk.lookat_fit_codebooks(sample, w.fit_iters, seed=w.seed)
+        ev[2].record()
+    torch.cuda.synchronize()
+    enc_ms, fit_ms = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
+    n = w.B * w.n_kv_heads * w.L
+    hbm_peak, which = measured_peak("hbm_gbs", FALLBACK_HBM_GBS)
+    tensor_peak, _ = measured_peak("bf16_tflops", 1590.0)
+    bytes_moved = n * (w.d_k * 2 + w.m)
+    flops = 2.0 * n * w.K * w.d_k * 2                      # two fp16 planes per centroid
+    del codes, books
+    return {"workload": w.name, "encode_ms": enc_ms, "keys_per_s": n / (enc_ms * 1e-3),
+            "hbm_frac": bytes_moved / (enc_ms * 1e-3) / 1e9 / hbm_peak,
+            "tensor_frac": flops / (enc_ms * 1e-3) / 1e12 / tensor_peak, "peaks": which,
+            "refit_ms": fit_ms, "refit": f"{w.fit_iters} Lloyd iterations on {w.fit_keys_per_head} keys"}
+
+
 def run_lookat(args, w):
     import torch
     import torch.distributed as dist
@@ -391,6 +424,8 @@ def run_lookat(args, w):
     step()
     torch.cuda.synchronize()
     same = bool(torch.allclose(out_host.cuda(), out, rtol=0, atol=1e-5))
+    # read ceiling of this GPU, same process and clocks: a read-only streaming pass over the V cache (>> L2)
+    read_ceiling = lk.lookat_probe_read_bandwidth(v, reps=5) if v.numel() * 2 >= (1 << 28) else None
 
     if rank == 0:
         units_per_step = w.B * w.n_q_heads * L * world
@@ -409,7 +444,9 @@ def run_lookat(args, w):
             "roofline": {"bound": "hbm", "kernel": "attend_stream_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
                          "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,
-                         "kernel_ms": attend_ms, "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS},
+                         "kernel_ms": attend_ms, "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+                         "read_ceiling_gbs": read_ceiling,
+                         "frac_of_read_ceiling": None if not read_ceiling else achieved / read_ceiling},
             "e2e": {"value": units_per_step / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": int(q_host.numel() * 2 + k_host.numel() * 2 + v_host.numel() * 2),
                     "d2h_bytes_per_step": int(out_host.numel() * 4), "ms_per_step": e2e_ms / e2e_steps,
@@ -430,6 +467,10 @@ def run_lookat(args, w):
                 line["prefill"] = time_prefill(local_rank)
             except Exception as exc:                      # the decode line stands on its own
                 line["prefill"] = {"error": str(exc)[:200]}
+            try:
+                line["encode_1m"] = time_encode_1m(local_rank)
+            except Exception as exc:
+                line["encode_1m"] = {"error": str(exc)[:200]}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()

@@ -258,6 +258,17 @@ enum {
 lookat_status lookat_set_prefill_form(lookat_ctx *ctx, int32_t form);
 
 /*
+ * Measurement aid (the paper has no counterpart): reads `bytes` of the device
+ * buffer `buf` (16-byte aligned) `reps` times with a read-only streaming kernel
+ * on the context's stream, one untimed pass first, and returns the bandwidth in
+ * GB/s (CUDA events around the timed passes; the call synchronises on them).
+ * bench.py reports it beside the attend kernel's bandwidth as the read ceiling
+ * of the GPU it ran on.
+ */
+lookat_status lookat_probe_read_bandwidth(lookat_ctx *ctx, const void *buf, uint64_t bytes, int32_t reps,
+                                          double *gb_per_s);
+
+/*
  * Self-test of the time-out status: launches a one-warp kernel whose only wait
  * can never be satisfied and gives up after 4096 polls (it ends by itself in
  * microseconds; nothing hangs), raising the context's time-out flag exactly as

@@ -20,7 +20,7 @@ EXPORTS = [
     "lookat_create", "lookat_destroy", "lookat_last_error", "lookat_fit_codebooks",
     "lookat_encode_keys", "lookat_build_lut", "lookat_attend", "lookat_attend_static",
     "lookat_attend_prefill", "lookat_decode_step", "lookat_decode_step_host",
-    "lookat_kernel_launches", "lookat_selftest_timeout", "lookat_set_prefill_form", "lookat_set_timing", "lookat_attend_kernel_ms",
+    "lookat_kernel_launches", "lookat_probe_read_bandwidth", "lookat_selftest_timeout", "lookat_set_prefill_form", "lookat_set_timing", "lookat_attend_kernel_ms",
 ]
 
 STATUS = {0: "LOOKAT_OK", 1: "LOOKAT_ERR_INVALID_ARG", 2: "LOOKAT_ERR_UNSUPPORTED",
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
     lib.lookat_decode_step_host.restype = ctypes.c_int
     lib.lookat_kernel_launches.argtypes = [vp]
     lib.lookat_kernel_launches.restype = ctypes.c_uint64
+    lib.lookat_probe_read_bandwidth.argtypes = [vp, vp, ctypes.c_uint64, i32, ctypes.POINTER(ctypes.c_double)]
+    lib.lookat_probe_read_bandwidth.restype = i32
     lib.lookat_selftest_timeout.argtypes = [vp]
     lib.lookat_selftest_timeout.restype = i32
     lib.lookat_set_prefill_form.argtypes = [vp, i32]
@@ -282,6 +284,14 @@ class Lookat:
 
     def lookat_kernel_launches(self) -> int:
         return int(self._lib.lookat_kernel_launches(self._h))
+
+    def lookat_probe_read_bandwidth(self, buf, reps=5):
+        """GB/s of a read-only streaming pass over the device tensor `buf` (measurement aid)."""
+        out = ctypes.c_double(0.0)
+        self._check(self._lib.lookat_probe_read_bandwidth(self._h, ctypes.c_void_p(buf.data_ptr()),
+                                                          ctypes.c_uint64(buf.numel() * buf.element_size()), int(reps),
+                                                          ctypes.byref(out)))
+        return out.value
 
     def lookat_selftest_timeout(self):
         self._check(self._lib.lookat_selftest_timeout(self._h))

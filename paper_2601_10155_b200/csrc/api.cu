@@ -302,6 +302,16 @@ lookat_status lookat_set_prefill_form(lookat_ctx *handle, int32_t form)
     return LOOKAT_OK;
 }
 
+lookat_status lookat_probe_read_bandwidth(lookat_ctx *handle, const void *buf, uint64_t bytes, int32_t reps, double *gb_per_s)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    if (!buf || !gb_per_s || bytes < 16 || reps < 1 || ((uintptr_t)buf & 15) != 0)
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "probe: need a 16-byte aligned device buffer of at least 16 bytes and reps >= 1");
+    DeviceGuard guard(ctx->device);
+    return probe_read_bandwidth(ctx, buf, (size_t)bytes, reps, gb_per_s);
+}
+
 lookat_status lookat_selftest_timeout(lookat_ctx *handle)
 {
     if (!handle) return LOOKAT_ERR_INVALID_ARG;

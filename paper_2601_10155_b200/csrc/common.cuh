@@ -122,6 +122,8 @@ lookat_status launch_prefill_mma(Ctx *ctx, const PrefillArgs &a);
 bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a);
 lookat_status launch_prefill_umma(Ctx *ctx, const PrefillArgs &a);
 lookat_status launch_timeout_selftest(Ctx *ctx);
+// read-only streaming probe (probe.cu): measurement aid
+lookat_status probe_read_bandwidth(Ctx *ctx, const void *buf, size_t bytes, int reps, double *gb_per_s);
 
 lookat_status launch_build_lut(Ctx *ctx, const __half *q, int B, const float *codebooks, float *lut);
 
