@@ -93,8 +93,11 @@ __device__ __noinline__ int exact_code_warp(const __half *x, const float *book, 
     return code;
 }
 
+#ifndef LOOKAT_ENC_MIN_CTAS
+#define LOOKAT_ENC_MIN_CTAS 3
+#endif
 template <int D_SUB>
-__global__ void __launch_bounds__(kMmaThreads)
+__global__ void __launch_bounds__(kMmaThreads, LOOKAT_ENC_MIN_CTAS)
 encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
 {
     using S = MmaShape<D_SUB>;

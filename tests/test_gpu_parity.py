@@ -493,3 +493,13 @@ def test_a_wait_that_runs_out_is_reported_once_and_the_context_stays_usable():
     assert err.value.status == 5                                   # LOOKAT_ERR_TIMEOUT
     out = lk.lookat_attend_prefill(*args, q_pos0=100)              # reported once; the context is usable
     assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
+
+
+def test_read_bandwidth_probe_reports_a_plausible_figure():
+    w = synth.small_workload(B=1, n_q_heads=1, n_kv_heads=1, d_k=64, d_v=64, m=8, K=16, L=64)
+    lk = ctx_for(w)
+    buf = torch.ones(1 << 28, dtype=torch.uint8, device="cuda")            # 256 MiB: larger than L2
+    gbs = lk.lookat_probe_read_bandwidth(buf, reps=3)
+    assert 1000.0 < gbs < 12000.0, gbs
+    with pytest.raises(LookatError):
+        lk.lookat_probe_read_bandwidth(buf[1:17], reps=1)                 # misaligned
