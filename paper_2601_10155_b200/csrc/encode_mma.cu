@@ -27,7 +27,6 @@ constexpr int kMmaWarps = 8;
 constexpr int kMmaThreads = kMmaWarps * 32;
 constexpr int kMmaKeysPerWarpStep = 32;
 constexpr int kMmaStepsPerCta = 4;
-constexpr int kMmaKeysPerCta = kMmaWarps * kMmaKeysPerWarpStep * kMmaStepsPerCta;   // 1024
 
 // Error of a fast score, for the winner w and for the true nearest centroid c* (both have
 // ||c|| <= R = ||x|| + dist(x, w), and |s| <= Q = max(||x||^2, dist(x, w)^2)):
@@ -96,15 +95,19 @@ __device__ __noinline__ int exact_code_warp(const __half *x, const float *book, 
 #ifndef LOOKAT_ENC_MIN_CTAS
 #define LOOKAT_ENC_MIN_CTAS 3
 #endif
-template <int D_SUB>
-__global__ void __launch_bounds__(kMmaThreads, LOOKAT_ENC_MIN_CTAS)
-encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
+// KMEANS: the assignment step of Lloyd's iteration (cluster sums, counts, distortion) on top of the codes
+template <int D_SUB, bool KMEANS>
+__global__ void __launch_bounds__(kMmaThreads, KMEANS ? 2 : LOOKAT_ENC_MIN_CTAS)
+encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K, int steps_per_cta)
 {
     using S = MmaShape<D_SUB>;
     extern __shared__ __align__(16) uint32_t sm_words[];
     const int n_cols = (K + 7) & ~7;                                   // centroid columns, whole n-tiles
     uint32_t *frag = sm_words;                                         // [kSteps][n_cols][4 t][kFragWords]
     float *cn4 = reinterpret_cast<float *>(frag + S::kSteps * n_cols * 4 * S::kFragWords);   // [n_cols/8][4 t][4]
+    // k-means mode: this CTA's share of the per-cluster sums and counts, flushed to global memory once at the end
+    unsigned long long *sums_s = reinterpret_cast<unsigned long long *>(cn4 + 2 * n_cols);   // [K][D_SUB]
+    unsigned *cnt_s = reinterpret_cast<unsigned *>(sums_s + (size_t)K * D_SUB);               // [K]
     __shared__ int s_force_exact;
     __shared__ double s_red[kMmaWarps];
 
@@ -116,6 +119,10 @@ encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
 
     // ---- planes of -2c in fragment order, and ||c||^2 as initial accumulators ----
     if (tid == 0) s_force_exact = 0;
+    if (KMEANS) {
+        for (int e = tid; e < K * D_SUB; e += kMmaThreads) sums_s[e] = 0ull;
+        for (int e = tid; e < K; e += kMmaThreads) cnt_s[e] = 0u;
+    }
     __syncthreads();
     for (int c = tid; c < n_cols; c += kMmaThreads) {
         float norm = 0.f;
@@ -158,8 +165,8 @@ encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
     const bool force_exact = s_force_exact != 0;
 
     double dsum = 0.0;
-    const long long cta_key0 = (long long)blockIdx.x * kMmaKeysPerCta;
-    for (int step = 0; step < kMmaStepsPerCta; ++step) {
+    const long long cta_key0 = (long long)blockIdx.x * steps_per_cta * (kMmaWarps * kMmaKeysPerWarpStep);
+    for (int step = 0; step < steps_per_cta; ++step) {
         const long long key0 = cta_key0 + ((long long)step * kMmaWarps + warp) * kMmaKeysPerWarpStep;
         if (key0 >= a.n) break;                            // warp-uniform
         // ---- operand tiles of 2 x 16 keys: rows g and g+8 of each, dims 2t,2t+1 (+8) per k-step ----
@@ -276,31 +283,51 @@ encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K)
                 }
             }
 
-        // ---- store: lane t = 0 of a row writes its code (and, for k-means, adds the key to its cluster) ----
-        if (t == 0) {
+        // ---- store: lane t = 0 of a row writes its code; for k-means the four lanes of a row add the dims they hold ----
 #pragma unroll
-            for (int u = 0; u < 2; ++u)
+        for (int u = 0; u < 2; ++u)
 #pragma unroll
-                for (int rr = 0; rr < 2; ++rr) {
-                    const long long key = key0 + u * 16 + g + rr * 8;
-                    if (key >= a.n) continue;
-                    const int cd = code[u][rr];
-                    a.codes[((size_t)bh * a.L_max + a.pos + key) * m + j] = (uint8_t)cd;
-                    if (a.sums) {
-                        const __half *x = rowp[u][rr];
-                        unsigned long long *s = a.sums + ((size_t)problem * K + cd) * D_SUB;
+            for (int rr = 0; rr < 2; ++rr) {
+                const long long key = key0 + u * 16 + g + rr * 8;
+                const int cd = __shfl_sync(0xffffffffu, code[u][rr], lane & ~3);     // the exact path told lane t = 0 only
+                if (key >= a.n) continue;
+                if (t == 0) a.codes[((size_t)bh * a.L_max + a.pos + key) * m + j] = (uint8_t)cd;
+                if (KMEANS) {
+                    unsigned long long *srow = sums_s + (size_t)cd * D_SUB;
 #pragma unroll
-                        for (int i = 0; i < D_SUB; ++i)
-                            atomicAdd(s + i, (unsigned long long)half_to_fixed24(x[i]));
-                        atomicAdd(a.cnt + (size_t)problem * K + cd, 1ull);
-                        if (a.distortion) dsum += dist_fp64(x, book + (size_t)cd * D_SUB, D_SUB);
+                    for (int ks = 0; ks < S::kSteps; ++ks) {
+                        const __half2 w0 = *reinterpret_cast<const __half2 *>(&xa[u][ks][rr]);
+                        atomicAdd(srow + ks * 16 + 2 * t, (unsigned long long)half_to_fixed24(__low2half(w0)));
+                        atomicAdd(srow + ks * 16 + 2 * t + 1, (unsigned long long)half_to_fixed24(__high2half(w0)));
+                        if (D_SUB >= 16) {
+                            const __half2 w1 = *reinterpret_cast<const __half2 *>(&xa[u][ks][2 + rr]);
+                            atomicAdd(srow + ks * 16 + 2 * t + 8, (unsigned long long)half_to_fixed24(__low2half(w1)));
+                            atomicAdd(srow + ks * 16 + 2 * t + 9, (unsigned long long)half_to_fixed24(__high2half(w1)));
+                        }
+                    }
+                    if (t == 0) {
+                        atomicAdd(cnt_s + cd, 1u);
+                        if (a.distortion) dsum += dist_fp64(rowp[u][rr], book + (size_t)cd * D_SUB, D_SUB);
                     }
                 }
-            if (tie_count && a.near_ties) atomicAdd(a.near_ties, (unsigned long long)tie_count);
+            }
+        if (t == 0 && tie_count && a.near_ties) atomicAdd(a.near_ties, (unsigned long long)tie_count);
+    }
+
+    if (KMEANS) {                                           // flush this CTA's share
+        __syncthreads();
+        unsigned long long *gs = a.sums + (size_t)problem * K * D_SUB;
+        for (int e = tid; e < K * D_SUB; e += kMmaThreads) {
+            const unsigned long long v = sums_s[e];
+            if (v) atomicAdd(gs + e, v);
+        }
+        for (int e = tid; e < K; e += kMmaThreads) {
+            const unsigned c = cnt_s[e];
+            if (c) atomicAdd(a.cnt + (size_t)problem * K + e, (unsigned long long)c);
         }
     }
 
-    if (a.distortion) {                                     // uniform over the grid
+    if (KMEANS && a.distortion) {                           // uniform over the grid
         for (int s = 16; s; s >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, s);
         if (lane == 0) s_red[warp] = dsum;
         __syncthreads();
@@ -317,13 +344,17 @@ lookat_status launch_mma(Ctx *ctx, const EncodeArgs &a)
 {
     const lookat_config &c = ctx->cfg;
     const int n_cols = (c.K + 7) & ~7;
-    const size_t smem = (size_t)n_cols * (MmaShape<D_SUB>::kSteps * 4 * MmaShape<D_SUB>::kFragWords + 2) * 4;
-    auto kern = encode_mma_kernel<D_SUB>;
+    // k-means mode keeps a CTA's share of the cluster sums in shared memory and gives it more keys to amortise the flush
+    const int steps = a.sums ? 4 * kMmaStepsPerCta : kMmaStepsPerCta;
+    const size_t smem = (size_t)n_cols * (MmaShape<D_SUB>::kSteps * 4 * MmaShape<D_SUB>::kFragWords + 2) * 4 +
+                        (a.sums ? (size_t)c.K * D_SUB * 8 + (size_t)c.K * 4 : 0);
+    auto kern = a.sums ? encode_mma_kernel<D_SUB, true> : encode_mma_kernel<D_SUB, false>;
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return check_launch(ctx, "encode: shared-memory opt-in");
-    dim3 grid((unsigned)((a.n + kMmaKeysPerCta - 1) / kMmaKeysPerCta), c.m, a.B * c.n_kv_heads);
-    kern<<<grid, kMmaThreads, smem, ctx->stream>>>(a, c.n_kv_heads, c.d_k, c.m, c.K);
+    const long long per_cta = (long long)steps * kMmaWarps * kMmaKeysPerWarpStep;
+    dim3 grid((unsigned)((a.n + per_cta - 1) / per_cta), c.m, a.B * c.n_kv_heads);
+    kern<<<grid, kMmaThreads, smem, ctx->stream>>>(a, c.n_kv_heads, c.d_k, c.m, c.K, steps);
     return check_launch(ctx, "encode_mma_kernel");
 }
 
