@@ -40,7 +40,7 @@ namespace lookat {
 
 namespace {
 
-constexpr int kUmRows = 128;                   // queries per CTA = rows of one MMA
+constexpr int kUmRows = 128;                   // queries per tile = rows of one MMA
 constexpr int kUmChunk = 64;                   // tokens per chunk = columns of the score MMA
 constexpr int kUmTiles = 2;                    // query tiles per CTA
 constexpr int kUmSoftmax = kUmTiles * kUmRows, kUmProducers = 128, kUmVLoaders = 64;
