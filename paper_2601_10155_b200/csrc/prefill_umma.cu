@@ -15,13 +15,16 @@
 //   warps 0-3 / 4-7  softmax of tile 0 / tile 1: thread r owns query row r of its tile = tensor-memory lane r;
 //   warps 8-11  key producers: rebuild the next chunk's key rows from the codebook image in shared memory
 //               (16-byte items placed so that gathers and stores are free of bank conflicts whatever the codes are);
-//   warps 12-13 fetch the V rows of the chunk after next with cp.async, on their own schedule;
+//   warps 12-13 fetch the V rows of the chunk after next, on their own schedule: whole chunks by TMA (tiled bulk
+//               copies with the 128-byte swizzle of the MMA operand), the last partial chunk by cp.async;
 //   warp 14     one thread issues every MMA and commits them to mbarriers.
 // Tensor memory (512 columns): per tile the scores of one chunk (64; the fp16 weights overwrite their first
 // half), O (d_v) and the query rows as the A operand of the score MMA (d_k / 2).
 // Hand-offs go through mbarriers, one per buffer where a buffer is reused, so that no waiter can fall two
 // phases behind; every wait gives up after a bounded number of polls, raises the context's timeout flag and
 // lets the CTA drain and free its tensor memory.
+#include <cuda.h>           // CUtensorMap and its enums only; the driver entry point is looked up at run time
+
 #include "common.cuh"
 
 // Tuning aid (-DLOOKAT_PHASE_STAMPS): per role, the cycles spent in each phase of the chunk loop, averaged
@@ -189,7 +192,8 @@ struct UmLayout {
 
 template <int D_K, int D_V, bool SCORES>
 __global__ void __launch_bounds__(kUmThreads, 1)
-attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int *__restrict__ timeout_flag)
+attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int *__restrict__ timeout_flag,
+                           const __grid_constant__ CUtensorMap v_map, int use_tma)
 {
     using Lay = UmLayout<D_K, D_V>;
     extern __shared__ __align__(1024) unsigned char um_raw[];
@@ -223,7 +227,7 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         if (tid == 0) {
             for (int i = 0; i < 2; ++i) {
                 um_bar_init(bar_k + 8 * i, kUmProducers);
-                um_bar_init(bar_v + 8 * i, kUmVLoaders);
+                um_bar_init(bar_v + 8 * i, 1);                 // one arrival: the thread that issued the copies
                 for (int t = 0; t < kUmTiles; ++t) {
                     um_bar_init(bar_s + 16 * t + 8 * i, 1);
                     um_bar_init(bar_pv + 16 * t + 8 * i, 1);
@@ -432,22 +436,39 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                 if (!ok) { dead = true; break; }
             }
             UM_STAMP(vv, 0)
-            // V rows by cp.async: [nb][token][128 B], 16-byte pieces swizzled by token
+            // V rows as [nb][token][128 B] with the 16-byte pieces swizzled by token.  A whole chunk comes by TMA (one
+            // tiled bulk copy per 64-column block, 128-byte swizzle, completion counted in bytes on the barrier);
+            // the last, partial chunk by cp.async with the rows the CTA does not see zeroed.
             const bool whole = (long long)(c + 1) * kUmChunk <= t_end;
+            if (whole && use_tma) {
+                if (vtid == 0) {
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_v + 8 * buf), "r"(Lay::kV) : "memory");
 #pragma unroll
-            for (int i = 0; i < kPieces; ++i) {
-                const int p = vtid + i * kUmVLoaders, tl = p / (D_V / 8), pc = p % (D_V / 8);
-                const uint32_t off = Lay::kOffV + buf * Lay::kV + (pc >> 3) * (kUmChunk * 128) + tl * 128 + (((pc & 7) ^ (tl & 7)) << 4);
-                if (whole || (long long)c * kUmChunk + tl < t_end)
-                    um_cp_async16(sm0 + off, vsrc + ((size_t)c * kUmChunk + tl) * D_V + pc * 8);
-                else
-                    *reinterpret_cast<uint4 *>(sm + off) = make_uint4(0u, 0u, 0u, 0u);
+                    for (int nb = 0; nb < Lay::kNb; ++nb)
+                        asm volatile(
+                            "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+                                sm0 + Lay::kOffV + buf * Lay::kV + nb * (kUmChunk * 128)),
+                            "l"(reinterpret_cast<uint64_t>(&v_map)), "r"(nb * 64), "r"(c * kUmChunk), "r"(b * a.H_kv + h), "r"(bar_v + 8 * buf)
+                            : "memory");
+                }
+                UM_STAMP(vv, 1)
+            } else {
+#pragma unroll
+                for (int i = 0; i < kPieces; ++i) {
+                    const int p = vtid + i * kUmVLoaders, tl = p / (D_V / 8), pc = p % (D_V / 8);
+                    const uint32_t off = Lay::kOffV + buf * Lay::kV + (pc >> 3) * (kUmChunk * 128) + tl * 128 + (((pc & 7) ^ (tl & 7)) << 4);
+                    if (whole || (long long)c * kUmChunk + tl < t_end)
+                        um_cp_async16(sm0 + off, vsrc + ((size_t)c * kUmChunk + tl) * D_V + pc * 8);
+                    else
+                        *reinterpret_cast<uint4 *>(sm + off) = make_uint4(0u, 0u, 0u, 0u);
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                UM_STAMP(vv, 1)
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                um_fence_async_smem();
+                asm volatile("bar.sync 2, %0;" ::"n"(kUmVLoaders) : "memory");   // every loader's rows have landed
+                if (vtid == 0) um_bar_arrive(bar_v + 8 * buf);
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
-            UM_STAMP(vv, 1)
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            um_fence_async_smem();
-            um_bar_arrive(bar_v + 8 * buf);
             UM_STAMP(vv, 2)
         }
 #ifdef LOOKAT_PHASE_STAMPS
@@ -590,13 +611,44 @@ lookat_status launch_um(Ctx *ctx, const PrefillArgs &a)
     st = check_launch(ctx, "um_codebook_image_kernel");
     if (st != LOOKAT_OK) return st;
 
+    // tensor map of V as [row * head][token][d_v] for tiled bulk copies of 64 tokens x 64 columns with the 128-byte
+    // swizzle the MMA operand wants; without the driver entry point the loaders use cp.async for every chunk
+    CUtensorMap v_map;
+    memset(&v_map, 0, sizeof(v_map));
+    int use_tma = 0;
+    {
+        typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                      const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+        static encode_fn encode = nullptr;
+        static bool looked = false;
+        if (!looked) {
+            void *fn = nullptr;
+            cudaDriverEntryPointQueryResult q;
+            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
+                q == cudaDriverEntryPointSuccess)
+                encode = reinterpret_cast<encode_fn>(fn);
+            else
+                cudaGetLastError();
+            looked = true;
+        }
+        if (encode) {
+            const cuuint64_t dims[3] = {(cuuint64_t)D_V, (cuuint64_t)a.L_max, (cuuint64_t)a.B * a.H_kv};
+            const cuuint64_t strides[2] = {(cuuint64_t)D_V * 2, (cuuint64_t)a.L_max * D_V * 2};
+            const cuuint32_t box[3] = {64, (cuuint32_t)kUmChunk, 1}, estr[3] = {1, 1, 1};
+            use_tma = encode(&v_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<__half *>(a.v), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+        }
+    }
+
     const int n_tiles = (int)((a.L_q + kUmTiles * kUmRows - 1) / (kUmTiles * kUmRows));   // CTAs per (row, head)
     const int smem = (int)Lay::bytes(a.K);
     dim3 grid((unsigned)n_tiles, (unsigned)a.H_q, (unsigned)a.B);
     auto launch = [&](auto kern) -> lookat_status {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return check_launch(ctx, "prefill (tcgen05 form): shared-memory opt-in");
-        kern<<<grid, kUmThreads, smem, ctx->stream>>>(a, ctx->split_books, ctx->timeout_flag);
+        kern<<<grid, kUmThreads, smem, ctx->stream>>>(a, ctx->split_books, ctx->timeout_flag, v_map, use_tma);
         return check_launch(ctx, "attend_prefill_umma_kernel");
     };
     if (a.scores_out) return launch(attend_prefill_umma_kernel<D_K, D_V, true>);
