@@ -214,7 +214,10 @@ lookat_status lookat_decode_step(lookat_ctx *ctx, const void *q, const void *k_n
  * (Algorithm 1) and copies the output back.  All on the context's stream;
  * the call returns after the output has arrived (it synchronises the stream).
  *
- *   q_host      host fp16 [B][H_q][d_k]          (pinned memory for speed)
+ *   q_host      host fp16 [B][H_q][d_k]          (pinned memory for speed: when
+ *               q_host, k_new_host and out_host are pinned, 16-byte aligned and
+ *               addressable by the device, the kernel reads and writes them in
+ *               place and only the value rows are copied)
  *   k_new_host  host fp16 [B][H_kv][d_k]
  *   v_new_host  host fp16 [B][H_kv][d_v]
  *   codebooks   device fp32 [H_kv][m][K][d_sub]

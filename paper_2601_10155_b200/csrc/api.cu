@@ -81,6 +81,17 @@ lookat_status need_ptr(Ctx *ctx, const void *p, const char *name)
         if (st__ != LOOKAT_OK) return st__;      \
     } while (0)
 
+// the device address of a pinned, mapped host buffer, or NULL if the device cannot address it
+static const void *mapped_host_pointer(const void *host)
+{
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return attr.type == cudaMemoryTypeHost ? attr.devicePointer : nullptr;
+}
+
 lookat_status encode_impl(Ctx *ctx, const void *keys, int32_t B, int64_t n, const float *codebooks,
                           uint8_t *codes, int64_t L_max, int64_t pos, unsigned long long *near_ties);
 
@@ -537,8 +548,18 @@ lookat_status lookat_decode_step_host(lookat_ctx *handle, const void *q_host, co
     LOOKAT_TRY(ensure(ctx, (void **)&ctx->step_out, &ctx->step_out_cap, out_bytes, "step staging"));
 
     cudaStream_t s = ctx->stream;
-    cudaError_t e = cudaMemcpyAsync(ctx->step_q, q_host, q_bytes, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->step_k, k_new_host, k_bytes, cudaMemcpyHostToDevice, s);
+    // Pinned host buffers that the device can address (any cudaHostAlloc / registered memory under unified
+    // addressing) are read and written by the kernel itself: the queries and new keys cross the bus while the first
+    // tiles are already streaming, the output rows are posted by the merging CTAs, and three copies leave the stream.
+    const void *q_dev = mapped_host_pointer(q_host), *k_dev = mapped_host_pointer(k_new_host);
+    float *out_dev = static_cast<float *>(const_cast<void *>(mapped_host_pointer(out_host)));
+    const bool direct = q_dev && k_dev && out_dev && ((uintptr_t)q_dev & 15) == 0 && ((uintptr_t)k_dev & 15) == 0 &&
+                        ((uintptr_t)out_dev & 15) == 0;
+    cudaError_t e = cudaSuccess;
+    if (!direct) {
+        e = cudaMemcpyAsync(ctx->step_q, q_host, q_bytes, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->step_k, k_new_host, k_bytes, cudaMemcpyHostToDevice, s);
+    }
     // value rows go straight into the cache: B*H_kv rows of d_v halves, one per (b, h), at token pos
     if (e == cudaSuccess)
         e = cudaMemcpy2DAsync(static_cast<char *>(v) + (size_t)pos * v_row, (size_t)L_max * v_row, v_new_host, v_row,
@@ -546,9 +567,9 @@ lookat_status lookat_decode_step_host(lookat_ctx *handle, const void *q_host, co
     if (e != cudaSuccess) return set_error(ctx, LOOKAT_ERR_CUDA, "host-to-device copy: %s", cudaGetErrorString(e));
 
     // append + attend over tokens 0..pos of every row, one launch where the shape allows
-    LOOKAT_TRY(attend_impl(ctx, nullptr, ctx->step_q, codebooks, codes, v, B, L_max, nullptr, pos + 1, n_splits,
-                           ctx->step_out, nullptr, ctx->step_k, codes, pos));
-    e = cudaMemcpyAsync(out_host, ctx->step_out, out_bytes, cudaMemcpyDeviceToHost, s);
+    LOOKAT_TRY(attend_impl(ctx, nullptr, direct ? q_dev : ctx->step_q, codebooks, codes, v, B, L_max, nullptr, pos + 1, n_splits,
+                           direct ? out_dev : ctx->step_out, nullptr, direct ? k_dev : ctx->step_k, codes, pos));
+    if (!direct) e = cudaMemcpyAsync(out_host, ctx->step_out, out_bytes, cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return set_error(ctx, LOOKAT_ERR_CUDA, "device-to-host copy: %s", cudaGetErrorString(e));
     return LOOKAT_OK;
