@@ -351,7 +351,10 @@ def test_decode_steps_grow_the_cache_like_a_generation_loop():
         assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
 
 
-def test_decode_step_from_host_buffers():
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_step_from_host_buffers(pinned):
+    """Pinned buffers are addressed by the kernel in place; pageable ones go through staging copies."""
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
     w = synth.small_workload(B=3, n_q_heads=8, n_kv_heads=2, d_k=64, d_v=64, m=4, K=64, L=300)
     keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.4)
     books = random_books(w, 4)
@@ -364,10 +367,10 @@ def test_decode_step_from_host_buffers():
     codes_dev = dev(codes_ref)
     codes_dev[:, :, w.L - 1] = 77                      # the step must write this row
     v_dev = dev(v_cache)
-    out_host = torch.empty((w.B, w.n_q_heads, w.d_v), dtype=torch.float32).pin_memory()
-    lk.lookat_decode_step_host(torch.from_numpy(q).pin_memory(),
-                               torch.from_numpy(np.ascontiguousarray(keys[:, :, w.L - 1])).pin_memory(),
-                               torch.from_numpy(np.ascontiguousarray(v[:, :, w.L - 1])).pin_memory(),
+    out_host = pin(torch.empty((w.B, w.n_q_heads, w.d_v), dtype=torch.float32))
+    lk.lookat_decode_step_host(pin(torch.from_numpy(q)),
+                               pin(torch.from_numpy(np.ascontiguousarray(keys[:, :, w.L - 1]))),
+                               pin(torch.from_numpy(np.ascontiguousarray(v[:, :, w.L - 1]))),
                                dev(books), codes_dev, v_dev, w.L - 1, out_host)
     assert np.array_equal(codes_dev.cpu().numpy()[:, :, :w.L], codes_ref[:, :, :w.L])
     assert np.array_equal(v_dev.cpu().numpy()[:, :, w.L - 1], v[:, :, w.L - 1])
