@@ -11,6 +11,8 @@
 //
 // A CTA works on two tiles of 128 queries against the same chunks, one behind the other: while the softmax
 // threads of one tile work, the tensor pipe runs the other tile's MMAs, and every rebuilt chunk serves 256 queries.
+// The two tiles are consecutive row tiles of one query head, or (grouped heads) the same rows of two query heads
+// that share the KV head.
 // Roles in a CTA of 15 warps (one CTA per SM; the shared memory is full):
 //   warps 0-3 / 4-7  softmax of tile 0 / tile 1: thread r owns query row r of its tile = tensor-memory lane r;
 //   warps 8-11  key producers: rebuild the next chunk's key rows from the codebook image in shared memory
@@ -193,7 +195,7 @@ struct UmLayout {
 template <int D_K, int D_V, bool SCORES>
 __global__ void __launch_bounds__(kUmThreads, 1)
 attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int *__restrict__ timeout_flag,
-                           const __grid_constant__ CUtensorMap v_map, int use_tma)
+                           const __grid_constant__ CUtensorMap v_map, int use_tma, int pair_heads)
 {
     using Lay = UmLayout<D_K, D_V>;
     extern __shared__ __align__(1024) unsigned char um_raw[];
@@ -210,14 +212,17 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
     const uint32_t bar_k = bar0, bar_v = bar0 + 16, bar_s = bar0 + 32, bar_pv = bar0 + 64, bar_p = bar0 + 96;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int n_super = (int)((a.L_q + kUmTiles * kUmRows - 1) / (kUmTiles * kUmRows));
+    // The two tiles of a CTA are two query heads of one KV head over the same 128 rows where heads come in groups
+    // (pair_heads: same keys, same causal limits), else two consecutive tiles of 128 rows of one head.
+    const int rows_per_cta = pair_heads ? kUmRows : kUmTiles * kUmRows;
+    const int n_super = (int)((a.L_q + rows_per_cta - 1) / rows_per_cta);
     const int super = n_super - 1 - (int)blockIdx.x;           // longest first
-    const int hq = blockIdx.y, b = blockIdx.z, h = hq / a.g;
+    const int hq_first = pair_heads ? 2 * (int)blockIdx.y : (int)blockIdx.y, b = blockIdx.z, h = hq_first / a.g;
     const int d_sub = D_K / a.m;
 
-    const long long row0 = (long long)super * (kUmTiles * kUmRows);
-    const long long t_end = a.q_pos0 + (row0 + kUmTiles * kUmRows < a.L_q ? row0 + kUmTiles * kUmRows : a.L_q);   // tokens the CTA sees
-    const int n_chunks = (int)((t_end + kUmChunk - 1) / kUmChunk);     // both tiles walk all of them (tile 0: up to two all masked)
+    const long long row0 = (long long)super * rows_per_cta;
+    const long long t_end = a.q_pos0 + (row0 + rows_per_cta < a.L_q ? row0 + rows_per_cta : a.L_q);   // tokens the CTA sees
+    const int n_chunks = (int)((t_end + kUmChunk - 1) / kUmChunk);     // both tiles walk all of them (row tiles: tile 0 has up to two all masked)
 
     // ---- prologue, all threads: codebook image into shared memory, barriers, tensor memory ----
     {
@@ -254,8 +259,9 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
     // ---- the query rows go to tensor memory as the A operand of the score MMA: lane r = row r, two halfs per column ----
     if (warp < kUmSoftmax / 32) {                              // one thread per row of each tile
         const int t = warp >> 2, r = (warp & 3) * 32 + lane;
-        const long long want = row0 + t * kUmRows + r;
+        const long long want = row0 + (pair_heads ? 0 : t * kUmRows) + r;
         const long long qr = want < a.L_q ? want : a.L_q - 1;  // rows beyond L_q repeat the last one
+        const int hq = hq_first + (pair_heads ? t : 0);
         const uint4 *src = reinterpret_cast<const uint4 *>(a.q + ((size_t)(b * a.H_q + hq) * a.L_q + qr) * D_K);
 #pragma unroll
         for (int part = 0; part < D_K / 64; ++part) {
@@ -477,7 +483,8 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
     } else {
         // =================== softmax of tile t: thread r owns query row r of the tile (tensor-memory lane r) ===================
         const int t = warp >> 2, rq = warp & 3, r = rq * 32 + lane;
-        const long long row = row0 + t * kUmRows + r;
+        const long long row = row0 + (pair_heads ? 0 : t * kUmRows) + r;
+        const int hq = hq_first + (pair_heads ? t : 0);
         const long long vis_end = a.q_pos0 + (row < a.L_q ? row : a.L_q - 1) + 1;    // tokens this row sees
         const uint32_t lane_base = (uint32_t)(rq * 32) << 16;
         const uint32_t tm_s = tmem + t * kUmChunk + lane_base, tm_o = tmem + Lay::kColO + t * D_V + lane_base;
@@ -642,13 +649,16 @@ lookat_status launch_um(Ctx *ctx, const PrefillArgs &a)
         }
     }
 
-    const int n_tiles = (int)((a.L_q + kUmTiles * kUmRows - 1) / (kUmTiles * kUmRows));   // CTAs per (row, head)
+    // grouped heads: a CTA takes two query heads of a KV head over 128 rows; else two row tiles of one head
+    const int pair_heads = a.g % 2 == 0 ? 1 : 0;
+    const int rows_per_cta = pair_heads ? kUmRows : kUmTiles * kUmRows;
+    const int n_tiles = (int)((a.L_q + rows_per_cta - 1) / rows_per_cta);
     const int smem = (int)Lay::bytes(a.K);
-    dim3 grid((unsigned)n_tiles, (unsigned)a.H_q, (unsigned)a.B);
+    dim3 grid((unsigned)n_tiles, (unsigned)(pair_heads ? a.H_q / 2 : a.H_q), (unsigned)a.B);
     auto launch = [&](auto kern) -> lookat_status {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return check_launch(ctx, "prefill (tcgen05 form): shared-memory opt-in");
-        kern<<<grid, kUmThreads, smem, ctx->stream>>>(a, ctx->split_books, ctx->timeout_flag, v_map, use_tma);
+        kern<<<grid, kUmThreads, smem, ctx->stream>>>(a, ctx->split_books, ctx->timeout_flag, v_map, use_tma, pair_heads);
         return check_launch(ctx, "attend_prefill_umma_kernel");
     };
     if (a.scores_out) return launch(attend_prefill_umma_kernel<D_K, D_V, true>);
