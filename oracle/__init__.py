@@ -200,3 +200,32 @@ def decode_step(q, codebooks, codes, v, seq_lens=None, scale=None):
     """Algorithm 1 as a whole: build the tables, then attend."""
     return attend(build_lut(q, codebooks), codes, v, seq_lens=seq_lens, scale=scale,
                   d_k=q.shape[-1])
+
+
+def attend_pqv(lut, codes, v_codebooks, v_codes, seq_lens=None, scale=None, d_k=None):
+    """Decode attention with product-quantised values as well -- the extension Section 5.2 leaves as future work;
+    the formulation is this build's own and has no counterpart in the paper.  The weights alpha are those of
+    Algorithm 1 (scores from the key codes); the output is o = sum_t alpha_t v^_t with v^_t the value centroids the
+    value codes name, taken per value subspace j as sum_c w[j][c] C^V_j[c], w[j][c] = sum of alpha_t over the
+    tokens whose code is c (a weight histogram).
+    lut fp64 [B][H_q][m][K], codes u8 [B][H_kv][L_max][m], v_codebooks fp32 [H_kv][m_v][K_v][d_vsub],
+    v_codes u8 [B][H_kv][L_max][m_v].  Returns out fp64 [B][H_q][m_v * d_vsub]."""
+    v_codebooks = np.ascontiguousarray(v_codebooks, dtype=np.float32)
+    v_codes = np.ascontiguousarray(v_codes, dtype=np.uint8)
+    B, H_q = lut.shape[:2]
+    H_kv, m_v, K_v, d_vsub = v_codebooks.shape
+    L_max = codes.shape[2]
+    assert v_codes.shape == (B, H_kv, L_max, m_v) and int(v_codes.max(initial=0)) < K_v
+    g = H_q // H_kv
+    dummy = np.zeros((B, H_kv, L_max, 1), dtype=np.float16)
+    _, alpha = attend(lut, codes, dummy, seq_lens=seq_lens, scale=scale, d_k=d_k, want_alpha=True)
+    out = np.zeros((B, H_q, m_v * d_vsub), dtype=np.float64)
+    for b in range(B):
+        n = L_max if seq_lens is None else int(seq_lens[b])
+        for hq in range(H_q):
+            h = hq // g
+            for j in range(m_v):
+                w = np.zeros(K_v, dtype=np.float64)
+                np.add.at(w, v_codes[b, h, :n, j], alpha[b, hq, :n])
+                out[b, hq, j * d_vsub:(j + 1) * d_vsub] = w @ v_codebooks[h, j].astype(np.float64)
+    return out

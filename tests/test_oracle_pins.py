@@ -338,3 +338,36 @@ def test_prefill_is_algorithm_1_per_query_and_exact_attention_in_the_exact_case(
         assert np.isnan(scores[:, :, i, n:]).all()
         np.testing.assert_allclose(out[:, :, i], _softmax_attention_numpy(s_ref, v[:, :, :n], d_k ** -0.5, g),
                                    rtol=1e-12, atol=1e-14)
+
+
+def test_value_pq_attention_is_attention_over_the_reconstructed_values():
+    """The weight-histogram form equals sum_t alpha_t v^_t written out with numpy, and when every value sub-vector is
+    itself a centroid (value codebooks list the values) it is Algorithm 1 on the fp16 values."""
+    rng = np.random.default_rng(5)
+    B, H_q, H_kv, L, d_k, m, K, m_v, d_vsub = 2, 4, 2, 40, 16, 4, 8, 2, 4
+    books = rng.standard_normal((H_kv, m, K, d_k // m)).astype(np.float32)
+    codes = rng.integers(0, K, (B, H_kv, L, m), dtype=np.uint8)
+    q = rng.standard_normal((B, H_q, d_k)).astype(np.float16)
+    lut = oracle.build_lut(q, books)
+    v_books = rng.standard_normal((H_kv, m_v, 16, d_vsub)).astype(np.float32)
+    v_codes = rng.integers(0, 16, (B, H_kv, L, m_v), dtype=np.uint8)
+    seq_lens = np.array([L, 23], np.int32)
+    out = oracle.attend_pqv(lut, codes, v_books, v_codes, seq_lens=seq_lens, d_k=d_k)
+    # written out: softmax of the lookup sums, times the reconstructed values
+    g = H_q // H_kv
+    for b in range(B):
+        n = int(seq_lens[b])
+        for hq in range(H_q):
+            h = hq // g
+            s = np.array([sum(lut[b, hq, j, codes[b, h, t, j]] for j in range(m)) for t in range(n)]) / np.sqrt(d_k)
+            a = np.exp(s - s.max())
+            a /= a.sum()
+            v_hat = np.concatenate([v_books[h, j][v_codes[b, h, :n, j]] for j in range(m_v)], axis=1).astype(np.float64)
+            assert np.allclose(out[b, hq], a @ v_hat, rtol=1e-12, atol=1e-12)
+    # exact case: 16 distinct fp16 value rows per (head, subspace), every token takes one of them
+    v_books16 = v_books.astype(np.float16).astype(np.float32)
+    v = np.concatenate([v_books16[:, j][np.arange(H_kv)[None, :, None], v_codes[:, :, :, j]] for j in range(m_v)],
+                       axis=3).astype(np.float16)
+    ref = oracle.attend(lut, codes, v, seq_lens=seq_lens, d_k=d_k)
+    assert np.allclose(oracle.attend_pqv(lut, codes, v_books16, v_codes, seq_lens=seq_lens, d_k=d_k), ref,
+                       rtol=1e-12, atol=1e-12)
