@@ -261,6 +261,30 @@ enum {
 lookat_status lookat_set_prefill_form(lookat_ctx *ctx, int32_t form);
 
 /*
+ * Decode attention with product-quantised VALUES as well.  The paper leaves
+ * value compression to future work (Section 5.2); the formulation is this
+ * build's own.  The weights alpha are those of Algorithm 1 (scores from the
+ * key codes, softmax(s * scale)); the output is o = sum_t alpha_t v^_t with
+ * v^_t the value centroids named by the value codes, taken per value subspace
+ * as sum_c w[j][c] C^V_j[c], w = the histogram of the weights over the codes.
+ * Per token only m + m_v bytes are read.  Value codebooks and codes come from
+ * lookat_fit_codebooks / lookat_encode_keys of a context configured with
+ * d_k = this context's d_v and m = m_v (values are encoded like keys).
+ *
+ *   lut          NULL or device fp32 [B][H_q][m][K]; with NULL the tables are
+ *                built from q (fp16 [B][H_q][d_k]) and codebooks first
+ *   codes        device uint8 [B][H_kv][L_max][m]      (aligned to m bytes)
+ *   v_codebooks  device fp32 [H_kv][m_v][K_v][d_v / m_v]
+ *   v_codes      device uint8 [B][H_kv][L_max][m_v]    (aligned to m_v bytes)
+ *   seq_lens     NULL (all L_max) or device int32 [B], each >= 1
+ *   out          device fp32 [B][H_q][d_v]
+ * m and m_v must be 2, 4, 8 or 16 (else LOOKAT_ERR_UNSUPPORTED); K_v <= 256.
+ */
+lookat_status lookat_attend_pqv(lookat_ctx *ctx, const float *lut, const void *q, const float *codebooks,
+                                const uint8_t *codes, const float *v_codebooks, const uint8_t *v_codes, int32_t m_v,
+                                int32_t K_v, int32_t B, int64_t L_max, const int32_t *seq_lens, float *out);
+
+/*
  * Measurement aid (the paper has no counterpart): reads `bytes` of the device
  * buffer `buf` (16-byte aligned) `reps` times with a read-only streaming kernel
  * on the context's stream, one untimed pass first, and returns the bandwidth in

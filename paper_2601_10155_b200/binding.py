@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "liblookat.so")
 
 EXPORTS = [
     "lookat_create", "lookat_destroy", "lookat_last_error", "lookat_fit_codebooks",
-    "lookat_encode_keys", "lookat_build_lut", "lookat_attend", "lookat_attend_static",
+    "lookat_encode_keys", "lookat_build_lut", "lookat_attend", "lookat_attend_static", "lookat_attend_pqv",
     "lookat_attend_prefill", "lookat_decode_step", "lookat_decode_step_host",
     "lookat_kernel_launches", "lookat_probe_read_bandwidth", "lookat_selftest_timeout", "lookat_set_prefill_form", "lookat_set_timing", "lookat_attend_kernel_ms",
 ]
@@ -69,6 +69,8 @@ def load_library() -> ctypes.CDLL:
     lib.lookat_attend.restype = ctypes.c_int
     lib.lookat_attend_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, vp, i32, vp, vp]
     lib.lookat_attend_static.restype = ctypes.c_int
+    lib.lookat_attend_pqv.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i64, vp, vp]
+    lib.lookat_attend_pqv.restype = ctypes.c_int
     lib.lookat_attend_prefill.argtypes = [vp, vp, vp, vp, vp, i32, i64, i64, i64, vp, vp]
     lib.lookat_attend_prefill.restype = ctypes.c_int
     lib.lookat_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, i64, i32, vp]
@@ -217,6 +219,25 @@ class Lookat:
             _dev(seq_lens, torch.int32, "seq_lens", (B,)), n_splits,
             _dev(out, torch.float32, "out", (B, c.n_q_heads, c.d_v)),
             _dev(scores_out, torch.float32, "scores_out", (B, c.n_q_heads, L_max))))
+        return out
+
+    def lookat_attend_pqv(self, codes, v_codebooks, v_codes, lut=None, q=None, codebooks=None, seq_lens=None, out=None):
+        """Decode attention with product-quantised values as well (weights from the key codes, output from the
+        weight histogram over the value codes)."""
+        c = self.cfg
+        B, H, L_max, m = codes.shape
+        _, m_v, K_v, d_vsub = v_codebooks.shape
+        if out is None:
+            out = torch.empty((B, c.n_q_heads, c.d_v), dtype=torch.float32, device=self.device)
+        self._check(self._lib.lookat_attend_pqv(
+            self._h, _dev(lut, torch.float32, "lut", (B, c.n_q_heads, c.m, c.K)),
+            _dev(q, torch.float16, "q", (B, c.n_q_heads, c.d_k)),
+            _dev(codebooks, torch.float32, "codebooks", (c.n_kv_heads, c.m, c.K, self.d_sub)),
+            _dev(codes, torch.uint8, "codes", (B, c.n_kv_heads, L_max, c.m)),
+            _dev(v_codebooks, torch.float32, "v_codebooks", (c.n_kv_heads, m_v, K_v, c.d_v // m_v)),
+            _dev(v_codes, torch.uint8, "v_codes", (B, c.n_kv_heads, L_max, m_v)), m_v, K_v, B, L_max,
+            _dev(seq_lens, torch.int32, "seq_lens", (B,)),
+            _dev(out, torch.float32, "out", (B, c.n_q_heads, c.d_v))))
         return out
 
     def lookat_attend_static(self, codes, v, lut=None, q=None, codebooks=None, seq_lens=None, n_splits=0,

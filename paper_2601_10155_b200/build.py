@@ -16,7 +16,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG, "liblookat.so")
-SOURCES = ["api.cu", "attend.cu", "attend_static.cu", "prefill.cu", "prefill_mma.cu", "prefill_umma.cu", "lut.cu", "encode.cu", "encode_mma.cu", "fit.cu", "probe.cu"]
+SOURCES = ["api.cu", "attend.cu", "attend_static.cu", "attend_pqv.cu", "prefill.cu", "prefill_mma.cu", "prefill_umma.cu", "lut.cu", "encode.cu", "encode_mma.cu", "fit.cu", "probe.cu"]
 
 
 def _nvcc() -> str:

@@ -313,6 +313,35 @@ lookat_status lookat_set_prefill_form(lookat_ctx *handle, int32_t form)
     return LOOKAT_OK;
 }
 
+lookat_status lookat_attend_pqv(lookat_ctx *handle, const float *lut, const void *q, const float *codebooks, const uint8_t *codes,
+                                const float *v_codebooks, const uint8_t *v_codes, int32_t m_v, int32_t K_v, int32_t B,
+                                int64_t L_max, const int32_t *seq_lens, float *out)
+{
+    if (!handle) return LOOKAT_ERR_INVALID_ARG;
+    Ctx *ctx = reinterpret_cast<Ctx *>(handle);
+    const lookat_config &c = ctx->cfg;
+    if (B < 1 || L_max < 1 || L_max > (1ll << 31))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "B=%d L_max=%lld out of range", B, (long long)L_max);
+    if (!lut && !(q && codebooks))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "lut is NULL and (q, codebooks) is incomplete");
+    LOOKAT_TRY(need_ptr(ctx, codes, "codes"));
+    LOOKAT_TRY(need_ptr(ctx, v_codebooks, "v_codebooks"));
+    LOOKAT_TRY(need_ptr(ctx, v_codes, "v_codes"));
+    LOOKAT_TRY(need_ptr(ctx, out, "out"));
+    if (seq_lens && (reinterpret_cast<uintptr_t>(seq_lens) & 3u))
+        return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "seq_lens is not 4-byte aligned");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return set_error(ctx, LOOKAT_ERR_CUDA, "cannot select device %d", ctx->device);
+    if (!lut) {
+        LOOKAT_TRY(need_ptr(ctx, q, "q"));
+        const size_t need = (size_t)B * c.n_q_heads * c.m * c.K * sizeof(float);
+        LOOKAT_TRY(ensure(ctx, (void **)&ctx->lut_scratch, &ctx->lut_cap, need, "table scratch"));
+        LOOKAT_TRY(launch_build_lut(ctx, static_cast<const __half *>(q), B, codebooks, ctx->lut_scratch));
+        lut = ctx->lut_scratch;
+    }
+    return attend_pqv_impl(ctx, lut, codes, v_codebooks, v_codes, m_v, K_v, B, L_max, seq_lens, out);
+}
+
 lookat_status lookat_probe_read_bandwidth(lookat_ctx *handle, const void *buf, uint64_t bytes, int32_t reps, double *gb_per_s)
 {
     if (!handle) return LOOKAT_ERR_INVALID_ARG;

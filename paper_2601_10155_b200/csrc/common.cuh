@@ -122,6 +122,9 @@ lookat_status launch_prefill_mma(Ctx *ctx, const PrefillArgs &a);
 bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a);
 lookat_status launch_prefill_umma(Ctx *ctx, const PrefillArgs &a);
 lookat_status launch_timeout_selftest(Ctx *ctx);
+// decode attention with product-quantised values as well (attend_pqv.cu)
+lookat_status attend_pqv_impl(Ctx *ctx, const float *lut, const uint8_t *codes, const float *v_books, const uint8_t *v_codes,
+                              int m_v, int K_v, int B, long long L_max, const int32_t *seq_lens, float *out);
 // read-only streaming probe (probe.cu): measurement aid
 lookat_status probe_read_bandwidth(Ctx *ctx, const void *buf, size_t bytes, int reps, double *gb_per_s);
 

@@ -506,3 +506,36 @@ def test_read_bandwidth_probe_reports_a_plausible_figure():
     assert 1000.0 < gbs < 12000.0, gbs
     with pytest.raises(LookatError):
         lk.lookat_probe_read_bandwidth(buf[1:17], reps=1)                 # misaligned
+
+
+# ------------------------------------------------------------------ product-quantised values (beyond the paper)
+@pytest.mark.parametrize("shape,m_v", [
+    (dict(B=2, n_q_heads=8, n_kv_heads=2, d_k=128, d_v=128, m=8, K=256, L=9000), 8),     # grouped heads, two chunks, ragged
+    (dict(B=3, n_q_heads=3, n_kv_heads=3, d_k=64, d_v=64, m=4, K=64, L=777), 16),        # d_vsub 4
+    (dict(B=1, n_q_heads=6, n_kv_heads=1, d_k=32, d_v=32, m=2, K=16, L=300), 2),         # 6 heads: groups of 4 + 2
+    (dict(B=2, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=128, m=16, K=200, L=100), 4),      # K < 256
+])
+@pytest.mark.parametrize("q_scale", [1.0, 0.1])
+def test_attend_with_quantised_values_matches_oracle(shape, m_v, q_scale):
+    w = synth.small_workload(**shape)
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, q_scale)
+    books, _ = oracle.fit_codebooks(keys[:, :, :min(w.L, 300)], w.m, w.K, iters=2, seed=3)
+    codes = oracle.encode_keys(keys, books)
+    K_v = 256 if w.L >= 300 else 64
+    v_books, _ = oracle.fit_codebooks(v[:, :, :min(w.L, 300)], m_v, K_v, iters=2, seed=4)     # values are encoded like keys
+    v_codes = oracle.encode_keys(v, v_books)
+    seq_lens = np.array([w.L - 5 * b for b in range(w.B)], np.int32)
+    lut = oracle.build_lut(q, books)
+    ref = oracle.attend_pqv(lut, codes, v_books, v_codes, seq_lens=seq_lens, d_k=w.d_k)
+    lk = ctx_for(w)
+    out = lk.lookat_attend_pqv(dev(codes), dev(v_books), dev(v_codes), q=dev(q), codebooks=dev(books),
+                               seq_lens=dev(seq_lens))
+    assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
+    out2 = lk.lookat_attend_pqv(dev(codes), dev(v_books), dev(v_codes), lut=dev(lut.astype(np.float32)),
+                                seq_lens=dev(seq_lens))
+    assert np.abs(out2.cpu().numpy() - ref).max() <= OUT_TOL
+    # the value codes and codebooks of the GPU's own encoder give the same codes as the oracle's (values are keys to it)
+    lv = Lookat(w.n_kv_heads, w.n_kv_heads, w.d_v, w.d_v, m_v, K_v)
+    ref_gap = oracle.encode_keys(v, v_books, want_gap=True)[1]
+    got = lv.lookat_encode_keys(dev(v), dev(v_books)).cpu().numpy()
+    check_codes(got, v_codes, ref_gap)
