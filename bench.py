@@ -318,6 +318,54 @@ def time_encode_1m(device_index: int):
             "refit_ms": fit_ms, "refit": f"{w.fit_iters} Lloyd iterations on {w.fit_keys_per_head} keys"}
 
 
+def time_pqv(lk, w, q, books, codes, v, steps: int, sm_mhz: float):
+    """Beyond the paper (its Section 5.2 names value compression as future work): the same decode attention with
+    the values product-quantised too (m_v = m subspaces, K = 256), `lookat_attend_pqv`.  Per (token, KV head) pair it
+    reads m + m_v bytes instead of m + 2 d_v; the codes of one copy fit in L2, so the step rotates through copies."""
+    import torch
+
+    from paper_2601_10155_b200.binding import Lookat
+    m_v = w.m
+    lv = Lookat(w.n_kv_heads, w.n_kv_heads, w.d_v, w.d_v, m_v, 256, device=lk.device.index)
+    n_fit = w.fit_keys_per_head or w.B * w.L
+    sample = v[:, :, :max(1, n_fit // w.B)].contiguous()
+    v_books = lv.lookat_fit_codebooks(sample, w.fit_iters, seed=w.seed + 1)       # values are encoded like keys
+    v_codes = lv.lookat_encode_keys(v, v_books)
+    bytes_per_copy = codes.numel() + v_codes.numel()
+    n_sets = max(2, int(np.ceil(3 * L2_BYTES / bytes_per_copy)))                  # every step reads from HBM
+    sets = [(codes.clone(), v_codes.clone()) for _ in range(n_sets)]
+    out = torch.empty((w.B, w.n_q_heads, w.d_v), dtype=torch.float32, device="cuda")
+    for i in range(3):
+        lk.lookat_attend_pqv(sets[i % n_sets][0], v_books, sets[i % n_sets][1], q=q, codebooks=books, out=out)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(steps):
+        lk.lookat_attend_pqv(sets[i % n_sets][0], v_books, sets[i % n_sets][1], q=q, codebooks=books, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    pairs = w.B * w.n_kv_heads * w.L
+    peak, which = measured_peak("hbm_gbs", FALLBACK_HBM_GBS)
+    achieved = pairs * (w.m + m_v) / (ms * 1e-3) / 1e9
+    smem_bytes = w.B * w.n_q_heads * w.L * (w.m * 4 + m_v * 4)
+    smem_peak = 148 * 128 * sm_mhz * 1e6 / 1e9
+    # what the compression costs in accuracy on these inputs: against the fp16-V result of the same step
+    ref = lk.lookat_attend(codes, v, q=q, codebooks=books)
+    err = float((out - ref).abs().max())
+    return {"ms_per_step": ms, "tokens_heads_per_s": w.B * w.n_q_heads * w.L / (ms * 1e-3), "m_v": m_v, "K_v": 256,
+            "launches_per_step": 2, "l2": f"{n_sets} copies of the codes in rotation",
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "note": f"(m + m_v) bytes per (token, KV head) pair; peak {which}.  The kernel is bound by its "
+                                 "table reads and histogram adds in shared memory, not by HBM: see shared_memory"},
+            # 4 bytes read and 4 bytes added per (token, query head, subspace), against 128 bytes per clock and SM
+            "shared_memory": {"bytes_per_step": smem_bytes, "achieved_gbs": smem_bytes / (ms * 1e-3) / 1e9,
+                              "peak_gbs": smem_peak, "frac": smem_bytes / (ms * 1e-3) / 1e9 / smem_peak,
+                              "note": "peak = 148 SMs x 128 B/clk x the median SM clock sampled during the timed decode steps"},
+            "max_abs_diff_to_fp16_values": err,
+            "note": "value compression is not part of the paper's method (its Section 5.2: future work)"}
+
+
 def run_lookat(args, w):
     import torch
     import torch.distributed as dist
@@ -426,6 +474,12 @@ def run_lookat(args, w):
     same = bool(torch.allclose(out_host.cuda(), out, rtol=0, atol=1e-5))
     # read ceiling of this GPU, same process and clocks: a read-only streaming pass over the V cache (>> L2)
     read_ceiling = lk.lookat_probe_read_bandwidth(v, reps=5) if v.numel() * 2 >= (1 << 28) else None
+    pqv = None
+    if world == 1 and args.prefill:                        # the extra legs run together
+        try:
+            pqv = time_pqv(lk, w, q, books, codes, v, min(args.steps, 50), sampler.summary()["sm_mhz"] or sampler.max_mhz or 1965)
+        except Exception as exc:
+            pqv = {"error": str(exc)[:200]}
 
     if rank == 0:
         units_per_step = w.B * w.n_q_heads * L * world
@@ -460,6 +514,8 @@ def run_lookat(args, w):
         }
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = time_oracle(w)
+        if pqv is not None:
+            line["pqv"] = pqv
         if world == 1 and args.prefill:
             del keys, v, codes, code_sets, v_sets
             torch.cuda.empty_cache()

@@ -514,6 +514,9 @@ def test_read_bandwidth_probe_reports_a_plausible_figure():
     (dict(B=3, n_q_heads=3, n_kv_heads=3, d_k=64, d_v=64, m=4, K=64, L=777), 16),        # d_vsub 4
     (dict(B=1, n_q_heads=6, n_kv_heads=1, d_k=32, d_v=32, m=2, K=16, L=300), 2),         # 6 heads: groups of 4 + 2
     (dict(B=2, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=128, m=16, K=200, L=100), 4),      # K < 256
+    (dict(B=1, n_q_heads=2, n_kv_heads=1, d_k=64, d_v=24, m=8, K=256, L=5000), 8),       # pairs of heads; d_vsub 3
+    (dict(B=1, n_q_heads=1, n_kv_heads=1, d_k=32, d_v=32, m=2, K=256, L=20000), 4),      # one unit over five CTAs
+    (dict(B=1, n_q_heads=4, n_kv_heads=1, d_k=64, d_v=64, m=16, K=256, L=4500), 16),     # rows not doubled, small blocks
 ])
 @pytest.mark.parametrize("q_scale", [1.0, 0.1])
 def test_attend_with_quantised_values_matches_oracle(shape, m_v, q_scale):
@@ -539,3 +542,28 @@ def test_attend_with_quantised_values_matches_oracle(shape, m_v, q_scale):
     ref_gap = oracle.encode_keys(v, v_books, want_gap=True)[1]
     got = lv.lookat_encode_keys(dev(v), dev(v_books)).cpu().numpy()
     check_codes(got, v_codes, ref_gap)
+
+
+@pytest.mark.parametrize("direction", [1, -1])
+def test_attend_with_quantised_values_rescales_its_histograms(direction):
+    """Scores that rise (fall) steadily along the sequence: with rising scores every block of tokens moves the
+    running maximum far up, so the fixed-point weight histograms are rescaled at every block; with falling scores the
+    first block fixes maximum and scale and everything later adds weights that are tiny against it.  The tables are
+    handed in directly: with m = 2, table 0 = delta * c and table 1 = 256 * delta * c, token t with codes
+    (t mod 256, t div 256) scores delta * t."""
+    L, d_v, m_v = 20000, 64, 8
+    w = synth.small_workload(B=1, n_q_heads=4, n_kv_heads=1, d_k=32, d_v=d_v, m=2, K=256, L=L)
+    v = synth.make_values(w)
+    v_books, _ = oracle.fit_codebooks(v[:, :, :400], m_v, 256, iters=2, seed=5)
+    v_codes = oracle.encode_keys(v, v_books)
+    t = np.arange(L)
+    codes = np.stack([t % 256, t // 256], axis=-1).astype(np.uint8)[None, None]
+    c = np.arange(256, dtype=np.float64)
+    lut = np.zeros((1, 4, 2, 256))
+    for h in range(4):
+        delta = direction * (h + 1) * 0.004               # over 20,000 tokens: 80 to 320, times 1/sqrt(32) in the exponent
+        lut[0, h, 0], lut[0, h, 1] = delta * c, 256 * delta * c
+    lut = lut.astype(np.float32).astype(np.float64)        # both sides start from the same fp32 tables
+    ref = oracle.attend_pqv(lut, codes, v_books, v_codes, seq_lens=np.array([L], np.int32), d_k=w.d_k)
+    out = ctx_for(w).lookat_attend_pqv(dev(codes), dev(v_books), dev(v_codes), lut=dev(lut.astype(np.float32)))
+    assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
