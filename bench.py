@@ -475,7 +475,7 @@ def run_lookat(args, w):
     # read ceiling of this GPU, same process and clocks: a read-only streaming pass over the V cache (>> L2)
     read_ceiling = lk.lookat_probe_read_bandwidth(v, reps=5) if v.numel() * 2 >= (1 << 28) else None
     pqv = None
-    if world == 1 and args.prefill:                        # the extra legs run together
+    if world == 1 and args.pqv:
         try:
             pqv = time_pqv(lk, w, q, books, codes, v, min(args.steps, 50), sampler.summary()["sm_mhz"] or sampler.max_mhz or 1965)
         except Exception as exc:
@@ -544,6 +544,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", dest="prefill", action="store_false",
                     help="skip the extra timing of the causal multi-query kernel")
+    ap.add_argument("--no-pqv", dest="pqv", action="store_false",
+                    help="skip the extra leg that times decode attention with product-quantised values")
     ap.add_argument("--only-prefill", action="store_true",
                     help="time only the causal multi-query kernel (prints its object alone)")
     ap.add_argument("--prefill-batch", type=int, default=0, help="smaller prefill case: batch rows")
