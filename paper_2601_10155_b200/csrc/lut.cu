@@ -40,10 +40,12 @@ build_lut_kernel(const __half *__restrict__ q, const float *__restrict__ codeboo
     for (int u = 0; u < 4; ++u)
         pre[u] = (live && vec && 4 * u < d_sub) ? __ldg(reinterpret_cast<const float4 *>(cen) + u) : make_float4(0.f, 0.f, 0.f, 0.f);
 
-    for (int i = threadIdx.x; i < chunks * d_k * kLutHeads; i += kLutThreads) {
-        const int h = i % kLutHeads, dim = (i / kLutHeads) % d_k, ch = i / (kLutHeads * d_k);
-        const int hg = ch * kLutHeads + h;
-        qs[i] = hg < g ? (double)__half2float(q[((size_t)b * H_q + kvh * g + hg) * d_k + dim]) : 0.0;
+    const __half *qrow = q + ((size_t)b * H_q + kvh * g) * d_k;     // the group's g query rows are contiguous
+    for (int ch = 0; ch < chunks; ++ch) {
+        for (int x = threadIdx.x; x < d_k * kLutHeads; x += kLutThreads) {
+            const int hg = ch * kLutHeads + (x & (kLutHeads - 1)), dim = x / kLutHeads;
+            qs[ch * d_k * kLutHeads + x] = hg < g ? (double)__half2float(qrow[hg * d_k + dim]) : 0.0;
+        }
     }
     __syncthreads();
     if (!live) return;
@@ -56,8 +58,10 @@ build_lut_kernel(const __half *__restrict__ q, const float *__restrict__ codeboo
             const double c[4] = {(double)c4.x, (double)c4.y, (double)c4.z, (double)c4.w};
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-#pragma unroll
-                for (int h = 0; h < kLutHeads; ++h) acc[h] = fma(qj[(i + u) * kLutHeads + h], c[u], acc[h]);
+                const double2 q01 = *reinterpret_cast<const double2 *>(qj + (i + u) * kLutHeads);
+                const double2 q23 = *reinterpret_cast<const double2 *>(qj + (i + u) * kLutHeads + 2);
+                acc[0] = fma(q01.x, c[u], acc[0]), acc[1] = fma(q01.y, c[u], acc[1]);
+                acc[2] = fma(q23.x, c[u], acc[2]), acc[3] = fma(q23.y, c[u], acc[3]);
             }
         };
         if (vec) {
