@@ -112,6 +112,56 @@ def test_full_size_properties(gqa_32k):
     assert float((o_r[0] - ref[0]).abs().max()) <= 2e-5
 
 
+def test_full_size_attention_with_quantised_values(gqa_32k):
+    """`lookat_attend_pqv` in the launch configuration bench.py times (16 rows, 32,768 tokens, m = m_v = 8): the
+    value codebooks are the oracle's k-means on 4096 values per head, the value codes the GPU encoder's (the
+    sampled rows get the oracle's codes, checked against the GPU's first), the tables come from q inside the call;
+    sampled (row, KV head) units against the oracle, plus properties that need no oracle."""
+    s = gqa_32k
+    w, lk = s["w"], s["lk"]
+    m_v = w.m
+    v_books, _ = oracle.fit_codebooks(s["v"][:1, :, :4096], m_v, 256, iters=2, seed=w.seed + 1)
+    lv = Lookat(w.n_kv_heads, w.n_kv_heads, w.d_v, w.d_v, m_v, 256)
+    v_books_d = dev(v_books)
+    v_codes_d = lv.lookat_encode_keys(s["v_d"], v_books_d)
+    rows = [(0, 0), (6, 5), (15, 7)]
+    for b, h in rows:
+        ref_codes, gap = oracle.encode_keys(s["v"][b:b + 1, h:h + 1], v_books[h:h + 1], want_gap=True)
+        got = v_codes_d[b, h].cpu().numpy()
+        assert not ((got != ref_codes[0, 0]) & ~((gap[0, 0] > 0) & (gap[0, 0] < 1e-6))).any()
+        v_codes_d[b, h] = dev(ref_codes[0, 0])
+    for q_scale in (1.0, 0.1):
+        q = synth.make_queries(w, q_scale)
+        out = lk.lookat_attend_pqv(s["codes_d"], v_books_d, v_codes_d, q=dev(q), codebooks=s["books_d"]).cpu().numpy()
+        assert np.isfinite(out).all()
+        for b, h in rows:
+            hq = slice(h * w.g, (h + 1) * w.g)
+            lut = oracle.build_lut(q[b:b + 1, hq], s["books"][h:h + 1])
+            codes = s["codes_d"][b:b + 1, h:h + 1].cpu().numpy()
+            ref = oracle.attend_pqv(lut, codes, v_books[h:h + 1], v_codes_d[b:b + 1, h:h + 1].cpu().numpy(), d_k=w.d_k)
+            assert np.abs(out[b, hq] - ref[0]).max() <= OUT_TOL
+    # bit-reproducible: the histogram adds are integer adds, whatever order they land in
+    q_d = dev(synth.make_queries(w, 0.1))
+    o1 = lk.lookat_attend_pqv(s["codes_d"], v_books_d, v_codes_d, q=q_d, codebooks=s["books_d"])
+    o2 = lk.lookat_attend_pqv(s["codes_d"], v_books_d, v_codes_d, q=q_d, codebooks=s["books_d"])
+    assert torch.equal(o1, o2)
+    # q = 0: uniform weights, the output is the mean of the dequantised values
+    o0 = lk.lookat_attend_pqv(s["codes_d"], v_books_d, v_codes_d, q=torch.zeros_like(q_d), codebooks=s["books_d"])
+    b, h = 3, 2
+    vc = v_codes_d[b, h].long()                             # [L][m_v]
+    deq = torch.cat([v_books_d[h, j][vc[:, j]] for j in range(m_v)], dim=1)      # [L][d_v]
+    assert float((o0[b, h * w.g] - deq.double().mean(dim=0).float()).abs().max()) <= 1e-4
+    # a row cut short by seq_lens equals attending over a cache of that length
+    sl = torch.full((w.B,), w.L, dtype=torch.int32, device="cuda")
+    sl[2], sl[9] = 5000, 0
+    o_r = lk.lookat_attend_pqv(s["codes_d"], v_books_d, v_codes_d, q=q_d, codebooks=s["books_d"], seq_lens=sl)
+    short = lk.lookat_attend_pqv(s["codes_d"][2:3, :, :5000].contiguous(), v_books_d, v_codes_d[2:3, :, :5000].contiguous(),
+                                 q=q_d[2:3].contiguous(), codebooks=s["books_d"])
+    assert float((o_r[2] - short[0]).abs().max()) <= 2e-5
+    assert float(o_r[9].abs().max()) == 0.0
+    assert torch.equal(o_r[0], o1[0])
+
+
 def test_encode_shape_of_the_1m_key_workload_on_a_subset():
     """d_k = 128, m = 16 (d_sub = 8), K = 256: 65,536 of the 1,048,576 keys against codebooks taken
     from the first keys by the start rule (0 Lloyd iterations), checked in full against the oracle."""
