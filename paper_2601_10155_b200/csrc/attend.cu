@@ -234,7 +234,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
     // shared memory: [tables | merge buffer (same bytes, used in turn)] [queries, fp64] [rings]
     const int merge_bytes = kWarps * 4 * (DV + 2) * 4;
     const int region0 = lut_bytes > merge_bytes ? lut_bytes : merge_bytes;
-    const int q_bytes = a.fused_lut ? (heads_max * a.d_k * 8 + 15) & ~15 : 0;
+    const int q_bytes = a.fused_lut ? 4 * a.d_k * 8 : 0;             // four heads' dims, widened (unused heads zero)
     float *lut_s = reinterpret_cast<float *>(smem_raw);
     double *q_s = reinterpret_cast<double *>(smem_raw + region0);
     unsigned char *ring = smem_raw + region0 + q_bytes + (size_t)warp * STAGES * SLOT;
@@ -439,8 +439,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         } else {
             // Section 3.5 "Precomputation Lookup Tables" for the heads of this unit:
             // lut[h][j][c] = q_h^(j) . C_j[c], fp64 accumulation, one rounding.
-            for (int i = tid; i < heads_here * a.d_k; i += kThreads)
-                q_s[i] = (double)__half2float(a.q[((size_t)b * a.H_q + hq0) * a.d_k + i]);
+            // the unit's queries, widened, head fastest: one 16-byte read serves two heads
+            for (int i = tid; i < 4 * a.d_k; i += kThreads) {
+                const int h = i & 3, dim = i >> 2;
+                q_s[i] = h < heads_here ? (double)__half2float(a.q[((size_t)b * a.H_q + hq0 + h) * a.d_k + dim]) : 0.0;
+            }
             __syncthreads();
 
             const int d_sub = a.d_k / M_SUB;
@@ -449,14 +452,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
                 const float *cen = book + (size_t)e * d_sub;
                 const int j = e / a.K;
                 const int es = j * kTableStride + (e - j * a.K);      // position in the shared-memory table
-                const double *qj = q_s + j * d_sub;
+                const double *qj = q_s + 4 * j * d_sub;
                 double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
                 auto step = [&](int i, float cf) {
                     const double cv = (double)cf;
-                    t0 = fma(qj[i], cv, t0);
-                    if (heads_here > 1) t1 = fma(qj[a.d_k + i], cv, t1);
-                    if (heads_here > 2) t2 = fma(qj[2 * a.d_k + i], cv, t2);
-                    if (heads_here > 3) t3 = fma(qj[3 * a.d_k + i], cv, t3);
+                    const double2 q01 = *reinterpret_cast<const double2 *>(qj + 4 * i);
+                    const double2 q23 = *reinterpret_cast<const double2 *>(qj + 4 * i + 2);
+                    t0 = fma(q01.x, cv, t0), t1 = fma(q01.y, cv, t1);
+                    t2 = fma(q23.x, cv, t2), t3 = fma(q23.y, cv, t3);
                 };
                 if ((d_sub & 3) == 0) {
 #pragma unroll 4
@@ -728,7 +731,7 @@ size_t stream_smem_bytes(const AttendArgs &a, int stages)
     const size_t lut_bytes = ((size_t)heads * (a.m * kTableStride + kHeadPad) * 4 + 15) & ~(size_t)15;
     const size_t merge_bytes = (size_t)kWarps * 4 * (a.d_v + 2) * 4;
     const size_t region0 = lut_bytes > merge_bytes ? lut_bytes : merge_bytes;
-    const size_t q_bytes = a.fused_lut ? ((size_t)heads * a.d_k * 8 + 15) & ~(size_t)15 : 0;
+    const size_t q_bytes = a.fused_lut ? (size_t)4 * a.d_k * 8 : 0;
     const size_t slot = (size_t)kTile * (a.d_v * 2 + 16) + (size_t)kTile * a.m;
     return region0 + q_bytes + (size_t)kWarps * stages * slot;
 }
