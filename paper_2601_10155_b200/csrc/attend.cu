@@ -210,6 +210,55 @@ __device__ __forceinline__ void phase_stamp(int k)
 #define LOOKAT_STAMP(k)
 #endif
 
+// The table entries of one unit, out of line: its registers are its own, so the next entry's centroid can be
+// requested ahead without touching the allocation of the streaming loop.
+__device__ __noinline__ void build_unit_tables(const float *book, const double *q_s, float *lut_s, int table, int K,
+                                               int d_sub, int heads_here, int head_stride, int tid)
+{
+    const bool vec16 = d_sub == 16;
+    float4 pre[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+        pre[u] = (vec16 && tid < table) ? __ldg(reinterpret_cast<const float4 *>(book + (size_t)tid * 16) + u) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int e = tid; e < table; e += kThreads) {
+        const float *cen = book + (size_t)e * d_sub;
+        const int j = e / K;
+        const int es = j * kTableStride + (e - j * K);
+        const double *qj = q_s + 4 * j * d_sub;
+        double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
+        auto step = [&](int i, float cf) {
+            const double cv = (double)cf;
+            const double2 q01 = *reinterpret_cast<const double2 *>(qj + 4 * i);
+            const double2 q23 = *reinterpret_cast<const double2 *>(qj + 4 * i + 2);
+            t0 = fma(q01.x, cv, t0), t1 = fma(q01.y, cv, t1);
+            t2 = fma(q23.x, cv, t2), t3 = fma(q23.y, cv, t3);
+        };
+        if (vec16) {
+            float4 nxt[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                nxt[u] = e + kThreads < table ? __ldg(reinterpret_cast<const float4 *>(cen + (size_t)kThreads * 16) + u) : pre[u];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                step(4 * u, pre[u].x); step(4 * u + 1, pre[u].y); step(4 * u + 2, pre[u].z); step(4 * u + 3, pre[u].w);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) pre[u] = nxt[u];
+        } else if ((d_sub & 3) == 0) {
+            for (int i = 0; i < d_sub; i += 4) {
+                const float4 c4 = __ldg(reinterpret_cast<const float4 *>(cen + i));
+                step(i, c4.x); step(i + 1, c4.y); step(i + 2, c4.z); step(i + 3, c4.w);
+            }
+        } else {
+            for (int i = 0; i < d_sub; ++i) step(i, __ldg(cen + i));
+        }
+        lut_s[es] = (float)t0;
+        if (heads_here > 1) lut_s[head_stride + es] = (float)t1;
+        if (heads_here > 2) lut_s[2 * head_stride + es] = (float)t2;
+        if (heads_here > 3) lut_s[3 * head_stride + es] = (float)t3;
+    }
+}
+
 template <int M_SUB, int DV, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a)
 {
@@ -448,33 +497,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
 
             const int d_sub = a.d_k / M_SUB;
             const float *book = a.codebooks + (size_t)kvh * table * d_sub;
-            for (int e = tid; e < table; e += kThreads) {
-                const float *cen = book + (size_t)e * d_sub;
-                const int j = e / a.K;
-                const int es = j * kTableStride + (e - j * a.K);      // position in the shared-memory table
-                const double *qj = q_s + 4 * j * d_sub;
-                double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
-                auto step = [&](int i, float cf) {
-                    const double cv = (double)cf;
-                    const double2 q01 = *reinterpret_cast<const double2 *>(qj + 4 * i);
-                    const double2 q23 = *reinterpret_cast<const double2 *>(qj + 4 * i + 2);
-                    t0 = fma(q01.x, cv, t0), t1 = fma(q01.y, cv, t1);
-                    t2 = fma(q23.x, cv, t2), t3 = fma(q23.y, cv, t3);
-                };
-                if ((d_sub & 3) == 0) {
-#pragma unroll 4
-                    for (int i = 0; i < d_sub; i += 4) {
-                        const float4 c4 = __ldg(reinterpret_cast<const float4 *>(cen + i));
-                        step(i, c4.x); step(i + 1, c4.y); step(i + 2, c4.z); step(i + 3, c4.w);
-                    }
-                } else {
-                    for (int i = 0; i < d_sub; ++i) step(i, __ldg(cen + i));
-                }
-                lut_s[es] = (float)t0;
-                if (heads_here > 1) lut_s[head_stride + es] = (float)t1;
-                if (heads_here > 2) lut_s[2 * head_stride + es] = (float)t2;
-                if (heads_here > 3) lut_s[3 * head_stride + es] = (float)t3;
-            }
+            build_unit_tables(book, q_s, lut_s, table, a.K, d_sub, heads_here, head_stride, tid);
         }
         __syncthreads();
 
