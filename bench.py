@@ -550,7 +550,7 @@ def main():
                     help="time only the causal multi-query kernel (prints its object alone)")
     ap.add_argument("--prefill-batch", type=int, default=0, help="smaller prefill case: batch rows")
     ap.add_argument("--prefill-heads", type=int, default=0, help="smaller prefill case: heads")
-    ap.add_argument("--prefill-form", default="auto", choices=["auto", "tables", "contraction", "contraction_mma_sync"],
+    ap.add_argument("--prefill-form", default="auto", choices=["auto", "tables", "contraction"],
                     help="which kernel lookat_attend_prefill uses in the prefill timing")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size (smaller cases for profiler captures)")

@@ -96,8 +96,11 @@ lookat_status lookat_fit_codebooks(lookat_ctx *ctx, const void *keys, int32_t B,
  *   near_ties  NULL, or in/out uint64[1]: incremented once per (key, subspace)
  *              whose best and second-best distance differ by a relative gap in
  *              (0, 1e-6) as evaluated in fp64.
- * Decisions are taken in fp32 and re-taken in fp64 wherever the two best
- * fp32 distances are within 1e-4 relative, so codes equal the fp64 argmin.
+ * Codes equal the fp64 argmin of the difference-form distance.  Bulk calls
+ * (d_sub 8, 16 or 32) search on the tensor cores (fp16 planes, fp32
+ * accumulation) and accept a winner only beyond a proven error margin; every
+ * other key, and every shape the tensor-core search does not cover (searched in
+ * fp32, accepted beyond a 1e-4 relative margin), is re-decided in fp64.
  * Requires pos >= 0, pos + n <= L_max.
  */
 lookat_status lookat_encode_keys(lookat_ctx *ctx, const void *keys, int32_t B, int64_t n,
@@ -153,8 +156,13 @@ lookat_status lookat_attend(lookat_ctx *ctx, const float *lut, const void *q, co
  * as does a shape whose tables cannot be built inside the kernel when lut is
  * NULL (pass ready tables then).
  *
- * The first call on a device looks up the device address of the array (no
- * allocation either); make that first call before starting a stream capture.
+ * The first call on a device looks up the device address of the array; make
+ * that first call before starting a stream capture.  The array and the kernel
+ * images take their device memory when the CUDA runtime loads the library's
+ * module on that device, which under the default lazy loading can be as late
+ * as this first call: a process that hands the whole device to its own pool
+ * must make one warm-up call (or run with CUDA_MODULE_LOADING=EAGER) BEFORE the
+ * pool takes the memory, else that first call can return LOOKAT_ERR_CUDA.
  * All calls share the array: two calls whose kernels overlap on the GPU
  * (different streams or contexts, same device) race on it and give wrong
  * results; calls on one stream are safe.  The counters are cleared at every
@@ -233,7 +241,7 @@ lookat_status lookat_decode_step_host(lookat_ctx *ctx, const void *q_host, const
 
 /*
  * Which of its two kernels lookat_attend_prefill uses.  Both compute Algorithm
- * 1 for every query; they differ in how the score of Section 3.4 is formed:
+ * 1 for every query; they differ in how the score of Section 3.5 ("Lookup and Sum") is formed:
  *   LOOKAT_PREFILL_TABLES       per-query tables built on chip, then m lookups
  *                               per (query, token) pair (any shape);
  *   LOOKAT_PREFILL_CONTRACTION  the centroids named by a chunk of codes are
@@ -241,11 +249,9 @@ lookat_status lookat_decode_step_host(lookat_ctx *ctx, const void *q_host, const
  *                               taken as q . (C_1[c_1], ..., C_m[c_m]) on the
  *                               tensor cores (d_k and d_v in {64, 128}, d_sub a
  *                               multiple of 8, both codebook planes of a head
- *                               in shared memory: K * d_k * 4 bytes);
- *                               tcgen05.mma with accumulators in tensor memory;
- *   LOOKAT_PREFILL_CONTRACTION_MMA_SYNC  the same contraction on the legacy
- *                               mma.sync path, kept as the baseline the tcgen05
- *                               kernel is measured against;
+ *                               in shared memory: K * d_k * 4 bytes; L_max * m a
+ *                               multiple of 4); tcgen05.mma with accumulators
+ *                               in tensor memory;
  *   LOOKAT_PREFILL_AUTO         (default) contraction where it applies and
  *                               L_q >= 32, tables otherwise.
  * Asking for the contraction form on a shape it does not cover makes
@@ -255,8 +261,7 @@ lookat_status lookat_decode_step_host(lookat_ctx *ctx, const void *q_host, const
 enum {
     LOOKAT_PREFILL_AUTO = 0,
     LOOKAT_PREFILL_TABLES = 1,
-    LOOKAT_PREFILL_CONTRACTION = 2,
-    LOOKAT_PREFILL_CONTRACTION_MMA_SYNC = 3
+    LOOKAT_PREFILL_CONTRACTION = 2
 };
 lookat_status lookat_set_prefill_form(lookat_ctx *ctx, int32_t form);
 
@@ -276,7 +281,7 @@ lookat_status lookat_set_prefill_form(lookat_ctx *ctx, int32_t form);
  *   codes        device uint8 [B][H_kv][L_max][m]      (aligned to m bytes)
  *   v_codebooks  device fp32 [H_kv][m_v][K_v][d_v / m_v]
  *   v_codes      device uint8 [B][H_kv][L_max][m_v]    (aligned to m_v bytes)
- *   seq_lens     NULL (all L_max) or device int32 [B], each >= 1
+ *   seq_lens     NULL (all L_max) or device int32 [B], 0..L_max; a row with 0 tokens gives zeros
  *   out          device fp32 [B][H_q][d_v]
  * m and m_v must be 2, 4, 8 or 16 (else LOOKAT_ERR_UNSUPPORTED); K_v <= 256.
  */

@@ -318,8 +318,8 @@ class Lookat:
         self._check(self._lib.lookat_selftest_timeout(self._h))
 
     def lookat_set_prefill_form(self, form):
-        """form: 'auto', 'tables', 'contraction' or 'contraction_mma_sync' (or the header's integer values)."""
-        code = {"auto": 0, "tables": 1, "contraction": 2, "contraction_mma_sync": 3}.get(form, form)
+        """form: 'auto', 'tables' or 'contraction' (or the header's integer values)."""
+        code = {"auto": 0, "tables": 1, "contraction": 2}.get(form, form)
         self._check(self._lib.lookat_set_prefill_form(self._h, int(code)))
 
     def lookat_set_timing(self, enabled: bool):

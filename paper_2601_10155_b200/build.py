@@ -16,7 +16,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG, "liblookat.so")
-SOURCES = ["api.cu", "attend.cu", "attend_static.cu", "attend_pqv.cu", "prefill.cu", "prefill_mma.cu", "prefill_umma.cu", "lut.cu", "encode.cu", "encode_mma.cu", "fit.cu", "probe.cu"]
+SOURCES = ["api.cu", "attend.cu", "attend_multi.cu", "attend_static.cu", "attend_pqv.cu", "prefill.cu", "prefill_umma.cu", "lut.cu", "encode.cu", "encode_mma.cu", "fit.cu", "probe.cu"]
 
 
 def _nvcc() -> str:
@@ -39,7 +39,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [_nvcc(), "--threads", "0", "-O3", "-std=c++20", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-shared", "-Xcompiler", "-fPIC", "-cudart", "static", "-I", INCLUDE, "-I", CSRC]
-    cmd += os.environ.get("LOOKAT_NVCC_FLAGS", "").split()      # e.g. -DNAME for tuning experiments
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]

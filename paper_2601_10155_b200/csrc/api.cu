@@ -306,8 +306,7 @@ lookat_status lookat_set_prefill_form(lookat_ctx *handle, int32_t form)
 {
     if (!handle) return LOOKAT_ERR_INVALID_ARG;
     Ctx *ctx = reinterpret_cast<Ctx *>(handle);
-    if (form != LOOKAT_PREFILL_AUTO && form != LOOKAT_PREFILL_TABLES && form != LOOKAT_PREFILL_CONTRACTION &&
-        form != LOOKAT_PREFILL_CONTRACTION_MMA_SYNC)
+    if (form != LOOKAT_PREFILL_AUTO && form != LOOKAT_PREFILL_TABLES && form != LOOKAT_PREFILL_CONTRACTION)
         return set_error(ctx, LOOKAT_ERR_INVALID_ARG, "set_prefill_form: unknown form %d", (int)form);
     ctx->prefill_form = form;
     return LOOKAT_OK;

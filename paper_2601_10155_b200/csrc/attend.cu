@@ -33,95 +33,12 @@
 #include <type_traits>
 
 #include "common.cuh"
+#include "attend_tile.cuh"
 #include "encode_warp.cuh"
 
 namespace lookat {
 
 namespace {
-
-constexpr int kWarps = 16;
-constexpr int kThreads = kWarps * 32;
-constexpr int kTile = 16;           // tokens per warp step (the MMA's k extent)
-constexpr int kHeadPad = 8;         // floats between the table sets of two heads (bank shift)
-constexpr int kTableStride = 256;   // shared-memory entries per subspace table (codes are bytes)
-constexpr float kNegBig = -1.0e30f; // running-max start: finite, so differences never give NaN
-
-__device__ __forceinline__ void cp_async16(unsigned smem_dst, const void *gmem_src)
-{
-#ifdef LOOKAT_CP_ASYNC_PLAIN
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
-#else
-    asm volatile("cp.async.cg.shared.global.L2::128B [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
-#endif
-}
-// Four 8x8 fp16 matrices, transposed on the way: lane l gives the address of one 16-byte matrix row.
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], unsigned smem_src)
-{
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(smem_src));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait()
-{
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-
-__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                          uint32_t a3, uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// Two weights as packed fp16: their roundings (part 0) or what the roundings left over (part 1).
-__device__ __forceinline__ uint32_t weight_pair(float w0, float w1, int part)
-{
-    const __half2 h = __floats2half2_rn(w0, w1);
-    const float2 f = __half22float2(h);
-    const __half2 r = __floats2half2_rn(w0 - f.x, w1 - f.y);
-    const __half2 out = part ? r : h;
-    return *reinterpret_cast<const uint32_t *>(&out);
-}
-
-template <int M_SUB>
-struct CodePair {                    // the codes of two consecutive tokens
-    uint32_t w[(2 * M_SUB + 3) / 4];
-};
-
-template <int M_SUB>
-__device__ __forceinline__ CodePair<M_SUB> read_code_pair(const unsigned char *p)
-{
-    CodePair<M_SUB> c;
-    if constexpr (M_SUB == 16) {
-        uint4 a = *reinterpret_cast<const uint4 *>(p);
-        uint4 b = *reinterpret_cast<const uint4 *>(p + 16);
-        c.w[0] = a.x; c.w[1] = a.y; c.w[2] = a.z; c.w[3] = a.w;
-        c.w[4] = b.x; c.w[5] = b.y; c.w[6] = b.z; c.w[7] = b.w;
-    } else if constexpr (M_SUB == 8) {
-        uint4 a = *reinterpret_cast<const uint4 *>(p);
-        c.w[0] = a.x; c.w[1] = a.y; c.w[2] = a.z; c.w[3] = a.w;
-    } else if constexpr (M_SUB == 4) {
-        uint2 a = *reinterpret_cast<const uint2 *>(p);
-        c.w[0] = a.x; c.w[1] = a.y;
-    } else if constexpr (M_SUB == 2) {
-        c.w[0] = *reinterpret_cast<const uint32_t *>(p);
-    } else {
-        c.w[0] = *reinterpret_cast<const uint16_t *>(p);
-    }
-    return c;
-}
-
-template <int M_SUB>
-__device__ __forceinline__ int code_at(const CodePair<M_SUB> &c, int token01, int j)
-{
-    const int byte = token01 * M_SUB + j;
-    return (int)__byte_perm(c.w[byte >> 2], 0u, 0x4440u | (unsigned)(byte & 3));
-}
 
 // Position in the flat tile sequence: tile `lt` of unit `unit`, with that unit's row facts and
 // the addresses of the tile's V rows and codes.
@@ -194,76 +111,11 @@ __device__ __noinline__ void append_encode_warp(const __half *x_sub, const float
     __syncwarp();
 }
 
-#ifdef LOOKAT_PHASE_STAMPS
-// Tuning aid, compiled only on request: per CTA, the global timer at a few points of the kernel.
-__device__ unsigned long long g_phase_stamps[1024][8];
-__device__ __forceinline__ void phase_stamp(int k)
-{
-    if (threadIdx.x == 0 && blockIdx.x < 1024) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-        g_phase_stamps[blockIdx.x][k] = t;
-    }
-}
-#define LOOKAT_STAMP(k) phase_stamp(k)
-#else
-#define LOOKAT_STAMP(k)
-#endif
-
-// The table entries of one unit, out of line: its registers are its own, so the next entry's centroid can be
-// requested ahead without touching the allocation of the streaming loop.
-__device__ __noinline__ void build_unit_tables(const float *book, const double *q_s, float *lut_s, int table, int K,
-                                               int d_sub, int heads_here, int head_stride, int tid)
-{
-    const bool vec16 = d_sub == 16;
-    float4 pre[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-        pre[u] = (vec16 && tid < table) ? __ldg(reinterpret_cast<const float4 *>(book + (size_t)tid * 16) + u) : make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int e = tid; e < table; e += kThreads) {
-        const float *cen = book + (size_t)e * d_sub;
-        const int j = e / K;
-        const int es = j * kTableStride + (e - j * K);
-        const double *qj = q_s + 4 * j * d_sub;
-        double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
-        auto step = [&](int i, float cf) {
-            const double cv = (double)cf;
-            const double2 q01 = *reinterpret_cast<const double2 *>(qj + 4 * i);
-            const double2 q23 = *reinterpret_cast<const double2 *>(qj + 4 * i + 2);
-            t0 = fma(q01.x, cv, t0), t1 = fma(q01.y, cv, t1);
-            t2 = fma(q23.x, cv, t2), t3 = fma(q23.y, cv, t3);
-        };
-        if (vec16) {
-            float4 nxt[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                nxt[u] = e + kThreads < table ? __ldg(reinterpret_cast<const float4 *>(cen + (size_t)kThreads * 16) + u) : pre[u];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                step(4 * u, pre[u].x); step(4 * u + 1, pre[u].y); step(4 * u + 2, pre[u].z); step(4 * u + 3, pre[u].w);
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) pre[u] = nxt[u];
-        } else if ((d_sub & 3) == 0) {
-            for (int i = 0; i < d_sub; i += 4) {
-                const float4 c4 = __ldg(reinterpret_cast<const float4 *>(cen + i));
-                step(i, c4.x); step(i + 1, c4.y); step(i + 2, c4.z); step(i + 3, c4.w);
-            }
-        } else {
-            for (int i = 0; i < d_sub; ++i) step(i, __ldg(cen + i));
-        }
-        lut_s[es] = (float)t0;
-        if (heads_here > 1) lut_s[head_stride + es] = (float)t1;
-        if (heads_here > 2) lut_s[2 * head_stride + es] = (float)t2;
-        if (heads_here > 3) lut_s[3 * head_stride + es] = (float)t3;
-    }
-}
 
 template <int M_SUB, int DV, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    LOOKAT_STAMP(0);
     constexpr int ROW = DV * 2 + 16;                      // a V row plus 16 bytes of padding
     constexpr int SLOT = kTile * ROW + kTile * M_SUB;     // V rows, then the tile's codes
     constexpr int V_CHUNKS = kTile * DV * 2 / 512;        // 16-byte pieces per lane and tile
@@ -470,7 +322,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         const bool head_ok = hl < heads_here;
 
         __syncthreads();                                   // the previous unit's merge is over
-        if (unit == unit_first) LOOKAT_STAMP(1);
         if (a.lut) {
             for (int h = 0; h < heads_here; ++h) {
                 const float *src = a.lut + ((size_t)b * a.H_q + hq0 + h) * table;
@@ -508,7 +359,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         float *scores_row =
             (a.scores_out && head_ok) ? a.scores_out + ((size_t)b * a.H_q + hq0 + hl) * a.L_max : nullptr;
 
-        if (unit == unit_first) LOOKAT_STAMP(2);
         const long long seg_hi = min(T_hi, (long long)(unit + 1) * a.tiles_per_unit);
         const bool full_unit = heads_here == 4 && !a.scores_out;
         while (cc.T < seg_hi) {
@@ -535,8 +385,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             cursor_advance<M_SUB, DV>(a, cc, hgroups);
         }
 
-        if (unit == unit_first) LOOKAT_STAMP(3);
-        if (unit == unit_last) LOOKAT_STAMP(4);
         // ---- this warp's result for the unit: fold the weight and remainder columns ----
 #pragma unroll
         for (int i = 0; i < DV / 16; ++i)
@@ -584,7 +432,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             }
         }
 
-        if (unit == unit_last) LOOKAT_STAMP(5);
         // ---- the CTA that completes a unit merges the unit's partials into the output ----
         long long c_lo, c_hi;
         if (a.splits_per_unit > 0) {
@@ -621,17 +468,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         }
     }
     cp_async_wait<0>();
-    LOOKAT_STAMP(6);
-#ifdef LOOKAT_PHASE_STAMPS
-    if (threadIdx.x == 0 && blockIdx.x < 1024) {
-        unsigned smid;
-        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
-        g_phase_stamps[blockIdx.x][7] = smid;
-    }
-#endif
 }
 
 // Any shape.  One CTA per (chunk, query head, batch row); 128 threads.
+constexpr int kMultiMaxTiles = 512;     // tiles per unit up to which attend_multi_kernel is used
 constexpr int kGenThreads = 128;
 constexpr int kGenBlockTokens = 1024;
 
@@ -813,14 +653,21 @@ lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_
     if (stages) {
         const int hgroups = (a.g + 3) / 4;
         const long long units = (long long)a.B * a.H_kv * hgroups;
-        const long long tpu = (a.L_max + kTile - 1) / kTile;
+        // the flat tile sequence covers the tokens that exist: where the host knows the length (no seq_lens), tiles
+        // beyond it are left out, so a cache with spare capacity still spreads over every CTA; L_max stays the row stride
+        const long long len_plan = a.seq_lens ? a.L_max : (a.uniform_len < a.L_max ? (long long)a.uniform_len : a.L_max);
+        const long long tpu = len_plan > 0 ? (len_plan + kTile - 1) / kTile : 1;
         if (units > (1ll << 30) || units * tpu > (1ll << 40))
             return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "attend: problem too large");
-        int per_sm = 0;
-        lookat_status st = dispatch_stream(a.m, a.d_v, stages, [&]<int M, int D, int S>() {
-            return stream_kernel_ready<M, D, S>(ctx, a, &per_sm);
-        });
-        if (st != LOOKAT_OK) return st;
+        // rows of up to 8192 tokens go to the kernel that keeps several units' tables resident (attend_multi.cu)
+        a.multi = (tpu <= kMultiMaxTiles && units * tpu < (1ll << 30) && multi_fits(ctx, a)) ? 1 : 0;
+        int per_sm = 1;
+        if (!a.multi) {
+            lookat_status st = dispatch_stream(a.m, a.d_v, stages, [&]<int M, int D, int S>() {
+                return stream_kernel_ready<M, D, S>(ctx, a, &per_sm);
+            });
+            if (st != LOOKAT_OK) return st;
+        }
         a.stream = 1;
         a.n_units = (int)units;
         a.tiles_per_unit = (int)tpu;
@@ -836,8 +683,26 @@ lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_
             long long ctas = (long long)per_sm * ctx->sm_count;
             if (ctas > total) ctas = total;
             a.tiles_per_cta = (total + ctas - 1) / ctas;
+            // short rows that would be cut into less than a unit per CTA: whole units instead (no partials to merge
+            // across CTAs; as many 16-tile rounds per warp, or nearly)
+            if (a.multi && tpu <= 64 && a.tiles_per_cta <= tpu) a.tiles_per_cta = tpu;
             a.splits_per_unit = 0;
             a.n_ctas = (int)((total + a.tiles_per_cta - 1) / a.tiles_per_cta);
+            // ranges that do not cross from one KV head into the next (a CTA stages one head's codebooks): each head's
+            // tiles are cut among floor(CTAs / heads) CTAs of its own, where that leaves few SMs idle
+            const long long cph = ctas / a.H_kv, tph = (long long)hgroups * a.B * tpu;
+            if (a.multi && a.H_kv > 1 && a.tiles_per_cta > tpu && cph >= 1 && cph * a.H_kv * 10 >= ctas * 9) {
+                a.tiles_per_cta = (tph + cph - 1) / cph;
+                a.ctas_per_head = (int)((tph + a.tiles_per_cta - 1) / a.tiles_per_cta);
+                a.n_ctas = a.ctas_per_head * a.H_kv;
+            }
+        }
+        if (a.multi) {
+            // the most units a CTA's range can touch
+            const long long span = a.splits_per_unit > 0 ? 1
+                                   : (a.tiles_per_cta % tpu == 0 ? a.tiles_per_cta / tpu : (a.tiles_per_cta + tpu - 2) / tpu + 1);
+            lookat_status st = plan_multi(ctx, a, (int)(span < kMaxRoundUnits ? span : kMaxRoundUnits));
+            if (st != LOOKAT_OK) return st;
         }
         const size_t slots = (size_t)a.n_ctas + (size_t)a.n_units;     // slot of (CTA c, unit u) = c + u
         *part_o_floats = slots * 4 * a.d_v;
@@ -884,7 +749,9 @@ lookat_status launch_attend(Ctx *ctx, const AttendArgs &a)
         cudaEventRecord(e0, ctx->stream);
     }
     lookat_status st;
-    if (a.stream) {
+    if (a.stream && a.multi) {
+        st = launch_multi(ctx, a);
+    } else if (a.stream) {
         st = dispatch_stream(a.m, a.d_v, stream_stages(ctx, a), [&]<int M, int D, int S>() {
             return stream_launch<M, D, S>(ctx, a);
         });
@@ -901,12 +768,6 @@ lookat_status launch_attend(Ctx *ctx, const AttendArgs &a)
     return st;
 }
 
-#ifdef LOOKAT_PHASE_STAMPS
-extern "C" int lookat_debug_phase_stamps(unsigned long long *host_out)     // [1024][8]
-{
-    return (int)cudaMemcpyFromSymbol(host_out, g_phase_stamps, sizeof(unsigned long long) * 1024 * 8);
-}
-#endif
 
 lookat_status launch_combine(Ctx *ctx, const AttendArgs &a)
 {

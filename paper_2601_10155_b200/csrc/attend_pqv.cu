@@ -41,10 +41,7 @@ namespace lookat {
 
 namespace {
 
-#ifndef LOOKAT_PQV_THREADS
-#define LOOKAT_PQV_THREADS 512
-#endif
-constexpr int kPqThreads = LOOKAT_PQV_THREADS;
+constexpr int kPqThreads = 512;
 constexpr int kPqWarps = kPqThreads / 32;
 // Coalesced code loads per lane and block: a block is 16 warps x 32 lanes x this many tokens.  Larger blocks spread
 // the per-block barriers and reductions over more tokens; the loaded codes and the weights of a block live in
@@ -52,11 +49,7 @@ constexpr int kPqWarps = kPqThreads / 32;
 template <int M_K, int M_V>
 __host__ __device__ constexpr int pqv_loads()
 {
-#ifdef LOOKAT_PQV_LOADS
-    return LOOKAT_PQV_LOADS;
-#else
     return M_K + M_V <= 16 ? 8 : 4;
-#endif
 }
 constexpr int kPqEntries = 256;                       // codes are bytes
 constexpr float kPqNegBig = -1.0e30f;

@@ -61,6 +61,13 @@ lookat_status check_launch(Ctx *ctx, const char *what);
 lookat_status ensure(Ctx *ctx, void **ptr, size_t *cap, size_t need_bytes, const char *what);
 
 // ---- launchers (each validates nothing: the API layer has done it) ----
+// Shared memory of attend_multi_kernel, byte offsets: tables of `ut` units, the warps' partials of those units, the
+// units' queries in fp64, the appended codes, the staged codebooks of one KV head (optional), the copy rings.
+struct MultiLayout {
+    int tables, partials, q, xk, newc, book, ring, total;
+    int set_floats;                 // floats per unit in `tables`
+};
+
 struct AttendArgs {
     const float *lut;          // [B][H_q][m][K], or null: built from q and codebooks
     const __half *q;           // [B][H_q][d_k]            (used when lut is null)
@@ -90,11 +97,18 @@ struct AttendArgs {
     // (batch row, KV head, group of <= 4 query heads); CTA c owns a contiguous range of it
     int stream;                // 1: streaming kernel and its partial layout
     int n_units;
-    int tiles_per_unit;        // ceil(L_max / 16)
+    int tiles_per_unit;        // ceil(len / 16), len = L_max with seq_lens, else the uniform length
     long long tiles_per_cta;
     int n_ctas;
     int splits_per_unit;       // > 0: CTA c = chunk c % splits of unit c / splits; 0: flat ranges
     float scale_log2;          // scale * log2(e)
+    // attend_multi_kernel (rows of up to a few thousand tokens): units ordered KV head first, several per round
+    int multi;                 // 1: that kernel
+    int ut;                    // units per round (tables resident together)
+    int stage_book;            // 1: a KV head's codebooks are staged in shared memory
+    int stages;                // depth of the per-warp copy rings
+    int ctas_per_head;         // > 0: every KV head's tiles are cut among this many CTAs of its own; 0: one flat cut
+    MultiLayout lay;           // its shared-memory layout
 };
 
 // Fills the decomposition fields of `a` (kernel choice, chunking) for n_splits as given to the
@@ -102,6 +116,10 @@ struct AttendArgs {
 lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_floats, size_t *part_ml_floats);
 lookat_status launch_attend(Ctx *ctx, const AttendArgs &a);
 lookat_status launch_combine(Ctx *ctx, const AttendArgs &a);
+// attend_multi.cu: shared-memory plan (units per round, staged codebooks, ring depth) and launch
+bool multi_fits(const Ctx *ctx, const AttendArgs &a);
+lookat_status plan_multi(Ctx *ctx, AttendArgs &a, int ut_wanted);
+lookat_status launch_multi(Ctx *ctx, const AttendArgs &a);
 
 struct PrefillArgs {
     const __half *q;           // [B][H_q][L_q][d_k]
@@ -115,10 +133,8 @@ struct PrefillArgs {
     float scale_log2;
 };
 lookat_status launch_prefill(Ctx *ctx, const PrefillArgs &a);
-// contraction form (prefill_mma.cu): centroids gathered per chunk, scores on the tensor cores
-bool prefill_mma_covers(const Ctx *ctx, const PrefillArgs &a);
-lookat_status launch_prefill_mma(Ctx *ctx, const PrefillArgs &a);
-// the same on tcgen05 with accumulators in tensor memory (prefill_umma.cu)
+// contraction form (prefill_umma.cu): centroids gathered per chunk, scores and value sums on tcgen05 with
+// accumulators in tensor memory
 bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a);
 lookat_status launch_prefill_umma(Ctx *ctx, const PrefillArgs &a);
 lookat_status launch_timeout_selftest(Ctx *ctx);

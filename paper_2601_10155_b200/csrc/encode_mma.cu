@@ -92,12 +92,9 @@ __device__ __noinline__ int exact_code_warp(const __half *x, const float *book, 
     return code;
 }
 
-#ifndef LOOKAT_ENC_MIN_CTAS
-#define LOOKAT_ENC_MIN_CTAS 3
-#endif
 // KMEANS: the assignment step of Lloyd's iteration (cluster sums, counts, distortion) on top of the codes
 template <int D_SUB, bool KMEANS>
-__global__ void __launch_bounds__(kMmaThreads, KMEANS ? 2 : LOOKAT_ENC_MIN_CTAS)
+__global__ void __launch_bounds__(kMmaThreads, KMEANS ? 2 : 3)
 encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K, int steps_per_cta)
 {
     using S = MmaShape<D_SUB>;
@@ -260,7 +257,9 @@ encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K, int steps_per_c
                 const float r = sqrtf(x2) + sqrtf(dw2);
                 const float err = kMmaErrR2 * r * r + kMmaErrQ * fmaxf(x2, dw2) + kMmaErrX * sqrtf(x2);
                 const bool unsure = force_exact || !(s - b > err);      // also true when anything is not a number
-                redo[u][rr] = __ballot_sync(0xffffffffu, unsure && t == 0);
+                // rows past the end were clamped to the last key: they are dropped, so they are not redone (nor counted)
+                const bool exists = key0 + u * 16 + g + rr * 8 < a.n;
+                redo[u][rr] = __ballot_sync(0xffffffffu, unsure && t == 0 && exists);
             }
         int tie_count = 0;
 #pragma unroll

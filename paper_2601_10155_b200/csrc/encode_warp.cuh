@@ -68,11 +68,51 @@ static __device__ double dist_fp64(const __half *x, const float *cen, int d_sub)
     return acc;
 }
 
+// Where the centroids of one codebook (K rows of d_sub floats) are read from.
+struct GlobalBook {                    // row-major in global memory
+    const float *p;
+    int d_sub;
+    __device__ __forceinline__ float4 load4(int c, int i) const
+    {
+        return __ldg(reinterpret_cast<const float4 *>(p + (size_t)c * d_sub + i));
+    }
+    __device__ __forceinline__ float load1(int c, int i) const { return __ldg(p + (size_t)c * d_sub + i); }
+};
+
+// Position (in 16-byte pieces) of piece `c4` of row `e` in a codebook staged in shared memory: rows stay where they
+// are, the n_c = d_sub / 4 pieces of a row are permuted so that eight consecutive rows read the same piece from
+// eight different 16-byte bank groups.  n_c must be 1, 2, 4, 8 or 16.
+__device__ __forceinline__ int staged_shift(int n_c) { return n_c >= 8 ? 0 : (n_c == 4 ? 1 : (n_c == 2 ? 2 : 3)); }
+__device__ __forceinline__ int staged_piece(int e, int c4, int n_c, int shift)
+{
+    return c4 ^ ((e >> shift) & (n_c - 1));
+}
+
+struct StagedBook {                    // a head's codebooks staged in shared memory; this codebook starts at row row0
+    const float *p;
+    int row0, d_sub, n_c, shift;
+    __device__ __forceinline__ float4 load4(int c, int i) const
+    {
+        const int e = row0 + c;
+        return *reinterpret_cast<const float4 *>(p + e * d_sub + staged_piece(e, i >> 2, n_c, shift) * 4);
+    }
+    __device__ __forceinline__ float load1(int c, int i) const
+    {
+        const int e = row0 + c;
+        return p[e * d_sub + staged_piece(e, i >> 2, n_c, shift) * 4 + (i & 3)];
+    }
+};
+
+// the key sub-vector as fp16 (global memory) or already widened to fp32 (shared memory): both exact
+__device__ __forceinline__ float key_dim(const __half *x, int i) { return __half2float(x[i]); }
+__device__ __forceinline__ float key_dim(const float *x, int i) { return x[i]; }
+
 // One (key sub-vector, codebook) search by a whole warp: lane l owns centroids l, l+32, ...
 // Every lane returns the code; *near_tie (if given) tells whether the fp64 gap of the two best
 // distances lies in (0, kNearTie).
-__device__ __forceinline__ int nearest_centroid_warp(const __half *x, const float *book, int K, int d_sub,
-                                                     int lane, bool *near_tie)
+template <class Book, class KeyT>
+__device__ __forceinline__ int nearest_centroid_warp_in(const KeyT *x, const Book &book, int K, int d_sub,
+                                                        int lane, bool *near_tie)
 {
     // lane l owns centroids l, l+32, ... (at most 8, K <= 256); dimensions in the outer loop so
     // that the lane's centroid loads of one step are independent of each other
@@ -82,13 +122,13 @@ __device__ __forceinline__ int nearest_centroid_warp(const __half *x, const floa
     if ((d_sub & 3) == 0) {
 #pragma unroll 2
         for (int i = 0; i < d_sub; i += 4) {
-            const float x0 = __half2float(x[i]), x1 = __half2float(x[i + 1]);
-            const float x2 = __half2float(x[i + 2]), x3 = __half2float(x[i + 3]);
+            const float x0 = key_dim(x, i), x1 = key_dim(x, i + 1);
+            const float x2 = key_dim(x, i + 2), x3 = key_dim(x, i + 3);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 const int c = lane + 32 * k;
                 if (c < K) {
-                    const float4 cv = __ldg(reinterpret_cast<const float4 *>(book + (size_t)c * d_sub + i));
+                    const float4 cv = book.load4(c, i);
                     float t = x0 - cv.x; d[k] = fmaf(t, t, d[k]);
                     t = x1 - cv.y; d[k] = fmaf(t, t, d[k]);
                     t = x2 - cv.z; d[k] = fmaf(t, t, d[k]);
@@ -98,12 +138,12 @@ __device__ __forceinline__ int nearest_centroid_warp(const __half *x, const floa
         }
     } else {
         for (int i = 0; i < d_sub; ++i) {
-            const float xi = __half2float(x[i]);
+            const float xi = key_dim(x, i);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 const int c = lane + 32 * k;
                 if (c < K) {
-                    const float t = xi - __ldg(book + (size_t)c * d_sub + i);
+                    const float t = xi - book.load1(c, i);
                     d[k] = fmaf(t, t, d[k]);
                 }
             }
@@ -127,12 +167,30 @@ __device__ __forceinline__ int nearest_centroid_warp(const __half *x, const floa
     int code = r.idx;
     bool tie = false;
     if (needs_fp64(r)) {
+        // the lane's (up to 8) centroids side by side: eight independent sums, each taken in dimension order
+        double dd[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) dd[k] = 0.0;
+        for (int i = 0; i < d_sub; ++i) {
+            const double xd = (double)key_dim(x, i);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int c = lane + 32 * k;
+                if (c < K) {
+                    const double t = xd - (double)book.load1(c, i);
+                    dd[k] = __dadd_rn(dd[k], __dmul_rn(t, t));      // product and sum rounded separately
+                }
+            }
+        }
         double best = INFINITY, second = INFINITY;
         int idx = 0x7fffffff;
-        for (int c = lane; c < K; c += 32) {
-            const double d = dist_fp64(x, book + (size_t)c * d_sub, d_sub);
-            if (d < best) { second = best; best = d; idx = c; }
-            else if (d < second) second = d;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int c = lane + 32 * k;
+            if (c < K) {
+                if (dd[k] < best) { second = best; best = dd[k]; idx = c; }
+                else if (dd[k] < second) second = dd[k];
+            }
         }
         for (int s = 16; s; s >>= 1) {
             const double ob = __shfl_xor_sync(0xffffffffu, best, s);
@@ -149,6 +207,12 @@ __device__ __forceinline__ int nearest_centroid_warp(const __half *x, const floa
     }
     if (near_tie) *near_tie = tie;
     return code;
+}
+
+__device__ __forceinline__ int nearest_centroid_warp(const __half *x, const float *book, int K, int d_sub,
+                                                     int lane, bool *near_tie)
+{
+    return nearest_centroid_warp_in(x, GlobalBook{book, d_sub}, K, d_sub, lane, near_tie);
 }
 
 }  // namespace lookat

@@ -372,16 +372,15 @@ lookat_status launch_pf(Ctx *ctx, const PrefillArgs &a)
 
 lookat_status launch_prefill(Ctx *ctx, const PrefillArgs &a)
 {
-    // contraction form: tcgen05 where it applies, else (or on request) the mma.sync kernel
-    const bool want_any = ctx->prefill_form == LOOKAT_PREFILL_CONTRACTION || ctx->prefill_form == LOOKAT_PREFILL_CONTRACTION_MMA_SYNC;
+    // contraction form (tcgen05) where it applies
+    const bool want = ctx->prefill_form == LOOKAT_PREFILL_CONTRACTION;
     const bool auto_pick = ctx->prefill_form == LOOKAT_PREFILL_AUTO && a.L_q >= 32;
-    if (want_any || auto_pick) {
-        if (ctx->prefill_form != LOOKAT_PREFILL_CONTRACTION_MMA_SYNC && prefill_umma_covers(ctx, a)) return launch_prefill_umma(ctx, a);
-        if (prefill_mma_covers(ctx, a)) return launch_prefill_mma(ctx, a);
-        if (want_any)
+    if (want || auto_pick) {
+        if (prefill_umma_covers(ctx, a)) return launch_prefill_umma(ctx, a);
+        if (want)
             return set_error(ctx, LOOKAT_ERR_UNSUPPORTED,
-                             "attend_prefill: the contraction form needs d_k, d_v in {64, 128}, d_sub a multiple of 8, a positive "
-                             "scale and K * d_k * 4 bytes of shared memory for the codebooks");
+                             "attend_prefill: the contraction form needs d_k, d_v in {64, 128}, d_sub a multiple of 8, L_max * m a "
+                             "multiple of 4, a positive scale and K * d_k * 4 bytes of shared memory for the codebooks");
     }
     if (a.d_v % 8 != 0 || a.d_v > 256 || ((uintptr_t)a.v & 15) != 0 || ((uintptr_t)a.codes & 3) != 0)
         return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "attend_prefill: d_v must be a multiple of 8, at most 256");

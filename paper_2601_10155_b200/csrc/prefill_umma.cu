@@ -29,18 +29,6 @@
 
 #include "common.cuh"
 
-// Tuning aid (-DLOOKAT_PHASE_STAMPS): per role, the cycles spent in each phase of the chunk loop, averaged
-// over the chunks of the first CTA and printed at its end.
-#ifdef LOOKAT_PHASE_STAMPS
-#include <cstdio>
-#define UM_STAMPS(name, n) long long name[n] = {}; long long um_tp_ = clock64();
-#define UM_STAMP(name, k) { const long long um_tn_ = clock64(); name[k] += um_tn_ - um_tp_; um_tp_ = um_tn_; }
-#define UM_FIRST_CTA (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
-#else
-#define UM_STAMPS(name, n)
-#define UM_STAMP(name, k)
-#endif
-
 namespace lookat {
 
 namespace {
@@ -319,36 +307,28 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             // the two tiles take turns, so the pipe has the other tile's MMAs while one tile's softmax runs.
             int next_qk[kUmTiles] = {0, 0}, next_pv[kUmTiles] = {0, 0};
             long long polls = 0;
-            UM_STAMPS(mm, 3)
             while (next_pv[0] < n_chunks || next_pv[1] < n_chunks) {
                 bool progress = false;
 #pragma unroll
                 for (int t = 0; t < kUmTiles; ++t) {           // value MMAs first: they release a tile's next scores
                     const int cp = next_pv[t];
                     if (cp < next_qk[t] && um_bar_test(bar_p + 8 * t, cp & 1) && um_bar_test(bar_v + 8 * (cp & 1), (cp >> 1) & 1)) {
-                        UM_STAMP(mm, 0)
                         um_fence_after();
                         value_mma(t, cp);
                         next_pv[t] = cp + 1;
                         progress = true;
-                        UM_STAMP(mm, 2)
                     }
                     const int cq = next_qk[t];
                     if (cq < n_chunks && next_pv[t] == cq && um_bar_test(bar_k + 8 * (cq & 1), (cq >> 1) & 1)) {
-                        UM_STAMP(mm, 0)
                         um_fence_after();
                         score_mma(t, cq);
                         next_qk[t] = cq + 1;
                         progress = true;
-                        UM_STAMP(mm, 1)
                     }
                 }
                 if (progress) polls = 0;
                 else if (++polls > kUmPolls) { dead = true; break; }
             }
-#ifdef LOOKAT_PHASE_STAMPS
-            if (UM_FIRST_CTA) printf("mma thread: idle %lld, score issue %lld, value issue %lld cycles per chunk (both tiles)\n", mm[0] / n_chunks, mm[1] / n_chunks, mm[2] / n_chunks);
-#endif
         }
     } else if (warp >= kUmSoftmax / 32 && warp < (kUmSoftmax + kUmProducers) / 32) {
         // =================== key producers ===================
@@ -404,7 +384,6 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         rebuild_keys(0);
         asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");   // everyone is done with the codes of chunk 0
         // keys of chunk c into the buffer that the score MMAs of chunk c - 2 (both tiles) have released
-        UM_STAMPS(pp, 3)
         for (int c = 1; c < n_chunks; ++c) {
             if (c >= 2) {
                 bool ok = true;
@@ -413,24 +392,17 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                     ok = um_group_wait<1, kUmProducers>(ptid == 0, bar_s + 16 * t + 8 * (c & 1), ((c - 2) >> 1) & 1) && ok;
                 if (!ok) { dead = true; break; }
             }
-            UM_STAMP(pp, 0)
             rebuild_keys(c);
-            UM_STAMP(pp, 1)
             if (c + 1 < n_chunks) fetch_codes(c + 1);          // into the code buffer the keys of chunk c - 1 were built from
             asm volatile("cp.async.commit_group;" ::: "memory");
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             asm volatile("bar.sync 1, %0;" ::"n"(kUmProducers) : "memory");   // those codes are visible to all key producers
-            UM_STAMP(pp, 2)
         }
-#ifdef LOOKAT_PHASE_STAMPS
-        if (UM_FIRST_CTA && ptid == 0) printf("key producers: wait key buffer %lld, rebuild %lld, codes + sync %lld\n", pp[0] / n_chunks, pp[1] / n_chunks, pp[2] / n_chunks);
-#endif
     } else if (warp >= (kUmSoftmax + kUmProducers) / 32) {
         // =================== V loaders ===================
         const int vtid = tid - kUmSoftmax - kUmProducers;
         const __half *vsrc = a.v + (size_t)(b * a.H_kv + h) * a.L_max * D_V;
         constexpr int kPieces = kUmChunk * (D_V / 8) / kUmVLoaders;
-        UM_STAMPS(vv, 3)
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
             // the V buffer of chunk c - 2 is free once both tiles' value MMAs of that chunk are done
@@ -441,7 +413,6 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                     ok = um_group_wait<2, kUmVLoaders>(vtid == 0, bar_pv + 16 * t + 8 * buf, ((c - 2) >> 1) & 1) && ok;
                 if (!ok) { dead = true; break; }
             }
-            UM_STAMP(vv, 0)
             // V rows as [nb][token][128 B] with the 16-byte pieces swizzled by token.  A whole chunk comes by TMA (one
             // tiled bulk copy per 64-column block, 128-byte swizzle, completion counted in bytes on the barrier);
             // the last, partial chunk by cp.async with the rows the CTA does not see zeroed.
@@ -457,7 +428,6 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                             "l"(reinterpret_cast<uint64_t>(&v_map)), "r"(nb * 64), "r"(c * kUmChunk), "r"(b * a.H_kv + h), "r"(bar_v + 8 * buf)
                             : "memory");
                 }
-                UM_STAMP(vv, 1)
             } else {
 #pragma unroll
                 for (int i = 0; i < kPieces; ++i) {
@@ -469,17 +439,12 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                         *reinterpret_cast<uint4 *>(sm + off) = make_uint4(0u, 0u, 0u, 0u);
                 }
                 asm volatile("cp.async.commit_group;" ::: "memory");
-                UM_STAMP(vv, 1)
                 asm volatile("cp.async.wait_group 0;" ::: "memory");
                 um_fence_async_smem();
                 asm volatile("bar.sync 2, %0;" ::"n"(kUmVLoaders) : "memory");   // every loader's rows have landed
                 if (vtid == 0) um_bar_arrive(bar_v + 8 * buf);
             }
-            UM_STAMP(vv, 2)
         }
-#ifdef LOOKAT_PHASE_STAMPS
-        if (UM_FIRST_CTA && vtid == 0) printf("V loaders: wait V buffer %lld, issue %lld, land %lld\n", vv[0] / n_chunks, vv[1] / n_chunks, vv[2] / n_chunks);
-#endif
     } else {
         // =================== softmax of tile t: thread r owns query row r of the tile (tensor-memory lane r) ===================
         const int t = warp >> 2, rq = warp & 3, r = rq * 32 + lane;
@@ -489,13 +454,11 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         const uint32_t lane_base = (uint32_t)(rq * 32) << 16;
         const uint32_t tm_s = tmem + t * kUmChunk + lane_base, tm_o = tmem + Lay::kColO + t * D_V + lane_base;
         float m_run = -INFINITY, l_run = 0.f;                  // reference point (base-2 exponent units) and row sum
-        UM_STAMPS(ss, 4)
         for (int c = 0; c < n_chunks; ++c) {
             const int buf = c & 1;
             const long long tok0 = (long long)c * kUmChunk;
             if (!__all_sync(0xffffffffu, um_bar_wait(bar_s + 16 * t + 8 * buf, (c >> 1) & 1))) { dead = true; break; }   // warp-uniform
             um_fence_after();
-            UM_STAMP(ss, 0)
             float sc[kUmChunk];                                // raw scores
             {
                 uint32_t s0[32], s1[32];
@@ -541,7 +504,6 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                 sum += b01.x + b01.y;                          // their rounding cancels in the normalised result
             }
             l_run = l_run * alpha + sum;
-            UM_STAMP(ss, 1)
             // The tile's previous value MMA is complete: the commit behind s_full covers every MMA its thread issued
             // before, and value(c - 1) was issued before scores(c).  So O may be rescaled right away.
             if (c >= 1 && __any_sync(0xffffffffu, alpha != 1.f)) {   // a reference point moved in this warp's rows
@@ -555,16 +517,11 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                     um_st32(tm_o + part * 32, o);
                 }
             }
-            UM_STAMP(ss, 2)
             um_st32(tm_s, pk);                                 // the 64 weights over the first half of the scores, two per column
             um_wait_st();
             um_fence_before();
             um_bar_arrive(bar_p + 8 * t);
-            UM_STAMP(ss, 3)
         }
-#ifdef LOOKAT_PHASE_STAMPS
-        if (UM_FIRST_CTA && (tid == 0 || tid == kUmRows)) printf("softmax of tile %d: wait scores %lld, load + exp %lld, rescale %lld, store %lld (%d chunks)\n", t, ss[0] / n_chunks, ss[1] / n_chunks, ss[2] / n_chunks, ss[3] / n_chunks, n_chunks);
-#endif
         if (!dead && __all_sync(0xffffffffu, um_bar_wait(bar_pv + 16 * t + 8 * ((n_chunks - 1) & 1), ((n_chunks - 1) >> 1) & 1))) {
             um_fence_after();
             const float inv = 1.f / l_run;

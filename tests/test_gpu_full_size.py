@@ -193,7 +193,7 @@ def prefill_4k():
     return dict(w=w, keys=keys, v=v, q=q, books=books, lk=lk, codes_d=codes_d)
 
 
-@pytest.mark.parametrize("form", ["contraction", "contraction_mma_sync", "tables"])
+@pytest.mark.parametrize("form", ["contraction", "tables"])
 def test_full_size_prefill_on_sampled_rows(prefill_4k, form):
     """The whole config-4 launch (batch 4, 32 heads, 4096 causal queries over 4096 tokens) as bench.py times it;
     sampled (row, head, query) triples against the oracle, tile and chunk edges among them; and a closed form
@@ -222,3 +222,93 @@ def test_full_size_prefill_on_sampled_rows(prefill_4k, form):
             ref = oracle.attend_prefill(s["q"][b:b + 1, h:h + 1, i:i + 1], s["books"][h:h + 1], codes_row,
                                         s["v"][b:b + 1, h:h + 1], q_pos0=i)
             assert np.abs(out[b, h, i] - ref[0, 0, 0]).max() <= OUT_TOL, (form, b, h, i)
+
+
+# ------------------------------------------------------------------ k-means at the sizes the benchmark fits
+def _fit_against_oracle(w, keys, lk, iters, head, subspaces, seed):
+    """GPU k-means on the whole problem, the oracle's on `subspaces` (consecutive, starting at 0) of KV head `head`
+    -- the start rule depends on (head, subspace) only through head * m + subspace, so head 0 keeps its starts when
+    the oracle is given just the first subspaces.  One Lloyd step must agree bit for bit (exact integer means)
+    unless the oracle flags a near tie in that assignment; the full run must be bit-identical, or -- where a near-tie
+    decision split the two runs -- end at the same distortion to 1e-4 relative."""
+    assert head == 0 and list(subspaces) == list(range(len(subspaces)))
+    d_sub, ms = w.d_sub, len(subspaces)
+    sub = np.ascontiguousarray(keys[:, :1, :, :ms * d_sub])
+    keys_d = dev(keys)
+    one_gpu = lk.lookat_fit_codebooks(keys_d, 1, seed=seed).cpu().numpy()[0, :ms]
+    books_gpu, trace_gpu = lk.lookat_fit_codebooks(keys_d, iters, seed=seed, want_distortion=True)
+    books_gpu, trace_gpu = books_gpu.cpu().numpy()[0, :ms], trace_gpu.cpu().numpy()[0, :ms]
+    start, _ = oracle.fit_codebooks(sub, ms, w.K, 0, seed=seed)
+    _, gap0 = oracle.encode_keys(sub, start, want_gap=True)
+    one, _ = oracle.fit_codebooks(sub, ms, w.K, 1, seed=seed)
+    if not ((gap0 > 0) & (gap0 < 1e-6)).any():
+        assert np.array_equal(one_gpu, one[0]), "one Lloyd step differs from the oracle"
+    ref, ref_trace = oracle.fit_codebooks(sub, ms, w.K, iters, seed=seed)
+    if np.array_equal(books_gpu, ref[0]):
+        np.testing.assert_allclose(trace_gpu, ref_trace[0], rtol=1e-11, atol=1e-300)
+    else:
+        np.testing.assert_allclose(trace_gpu[:, -1], ref_trace[0, :, -1], rtol=1e-4)
+    assert np.all(trace_gpu[:, 1:] <= trace_gpu[:, :-1] * (1 + 1e-7))
+    return sub, ref
+
+
+def test_fit_at_the_benchmark_size_on_two_subspaces():
+    """Config 3 as bench.py fits it: 8 KV heads x 8 subspaces of 16 dims, 65,536 keys per head (16 rows x 4096), 10
+    Lloyd iterations in one call; KV head 0, subspaces 0 and 1 against the oracle.  Then the near-tie counter of the bulk
+    encoder on those keys against the oracle's count."""
+    w = synth.WORKLOADS["gqa_32k_m8"]
+    keys = synth.make_keys(w, n_tokens=w.fit_keys_per_head // w.B)
+    lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K)
+    sub, ref = _fit_against_oracle(w, keys, lk, w.fit_iters, 0, (0, 1), w.seed)
+    ref_codes, gap = oracle.encode_keys(sub, ref, want_gap=True)
+    near = (gap > 0) & (gap < 1e-6)
+    l2 = Lookat(1, 1, 2 * w.d_sub, w.d_v, 2, w.K)
+    ties = torch.zeros(1, dtype=torch.int64, device="cuda")
+    codes = l2.lookat_encode_keys(dev(sub), dev(ref), near_ties=ties).cpu().numpy()
+    assert not ((codes != ref_codes) & ~near).any()
+    assert int(ties.item()) == int(near.sum())
+
+
+def test_refit_at_the_1m_key_workload_size_on_one_subspace():
+    """Config 4's refit as bench.py runs it: one head, 16 subspaces of 8 dims, 262,144 keys, 10 Lloyd iterations --
+    256 CTAs add into the sums of every problem; subspace 0 against the oracle."""
+    w = synth.WORKLOADS["encode_1m_m16"]
+    keys = synth.make_keys(w, n_tokens=w.fit_keys_per_head)
+    lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K)
+    _fit_against_oracle(w, keys, lk, w.fit_iters, 0, (0,), w.seed)
+
+
+# ------------------------------------------------------------------ the generation loop of config 2 at its size
+def test_generation_loop_at_the_gpt2_decoder_size():
+    """One attention layer of BASELINE config 2 at size: batch 32 x 12 heads, d = 64, m = 4, a cache with room for 1088
+    tokens that `lookat_decode_step` grows from 1024 to 1028 (append-encode + Algorithm 1 per step, one launch).  Per
+    step: the appended codes of every row bit-exact against the oracle's (near ties excused), and the outputs of sampled
+    (row, head) pairs against the oracle within 2e-3."""
+    w = synth.WORKLOADS["gpt2_b32_l1024_m4"]
+    L0, L_cap, steps = w.L, w.L + 64, 4
+    keys, v = synth.make_keys(w, n_tokens=L_cap), synth.make_values(w, n_tokens=L_cap)
+    books, _ = oracle.fit_codebooks(synth.make_calibration_keys(w, 4096), w.m, w.K, iters=2, seed=w.seed)
+    lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K)
+    books_d, v_d = dev(books), dev(v)
+    cache = torch.zeros((w.B, w.n_kv_heads, L_cap, w.m), dtype=torch.uint8, device="cuda")
+    lk.lookat_encode_keys(dev(keys[:, :, :L0]), books_d, codes=cache, pos=0)          # prefill encode
+    ref_cache, gap = oracle.encode_keys(keys, books, want_gap=True)                       # every key, appended ones too
+    near = (gap > 0) & (gap < 1e-6)
+    got = cache.cpu().numpy()
+    assert not ((got[:, :, :L0] != ref_cache[:, :, :L0]) & ~near[:, :, :L0].any(axis=-1, keepdims=True)).any()
+    cache[:, :, :L0] = dev(ref_cache[:, :, :L0])            # hand-off: attention below reads the oracle's codes
+    rng = np.random.default_rng(5)
+    for t in range(steps):
+        pos = L0 + t
+        q = synth.make_queries(synth.Workload(**{**w.__dict__, "seed": w.seed + 100 * t}), (1.0, 0.1, 0.5, 0.3)[t])
+        out = lk.lookat_decode_step(dev(q), dev(keys[:, :, pos]), books_d, cache, v_d, pos)
+        torch.cuda.synchronize()
+        out = out.cpu().numpy()
+        new = cache[:, :, pos].cpu().numpy()
+        assert not ((new != ref_cache[:, :, pos]) & ~near[:, :, pos]).any(), f"appended codes differ at step {t}"
+        assert float(cache[:, :, pos + 1:].max()) == 0, "a step wrote beyond its token"
+        cache[:, :, pos] = dev(ref_cache[:, :, pos])
+        for b, h in [(0, 0), (31, 11)] + [(int(rng.integers(w.B)), int(rng.integers(w.n_q_heads))) for _ in range(2)]:
+            lut = oracle.build_lut(q[b:b + 1, h:h + 1], books[h:h + 1])
+            ref = oracle.attend(lut, ref_cache[b:b + 1, h:h + 1, :pos + 1], v[b:b + 1, h:h + 1, :pos + 1], d_k=w.d_k)
+            assert np.abs(out[b, h] - ref[0, 0]).max() <= OUT_TOL, (t, b, h)
