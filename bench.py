@@ -41,6 +41,10 @@ FALLBACK_HBM_GBS = 6650.0
 # attend_stream_kernel launch, from an ncu capture of the batch-4 case of gqa_32k_m8
 # (283,105,792 bytes over 1,048,576 pairs; traffic grows in proportion to the pairs).
 ATTEND_DRAM_BYTES_PER_PAIR = {"gqa_32k_m8": 283105792 / 1048576}
+ATTEND_TRAFFIC_SOURCE = ("ncu capture of attend_stream_kernel<8,128,2> on gqa_32k_m8 at batch 4 "
+                         "(profiles/attend_stream_kernel_gqa_32k_m8_batch4_ncu.md), scaled by the pair count")
+SMALL_WORKLOADS = ["gpt2_l128_m4", "gpt2_b8_l256_m2", "gpt2_b8_l512_m2", "gpt2_b8_l1024_m2", "gpt2_b32_l1024_m4"]
+MIN_TIMED_SECONDS = 0.25
 
 
 def measured_peak(key: str, fallback: float):
@@ -161,6 +165,32 @@ def time_oracle(w, budget_s: float = 12.0):
     return {"value": units / dt, "unit": UNIT, "cores": oracle.n_threads(), "kind": "oracle",
             "sample": f"{rows} of {w.B} batch rows ({w.n_q_heads} query heads x {w.L} tokens), "
                       f"mean of {reps} steps of {dt * 1e3:.1f} ms; fp64, OpenMP over (row, head)"}
+
+
+def time_oracle_configs(budget_s: float = 2.0):
+    """The oracle's decode step (tables + attend, the newest key encoded first) on the GPT-2 shaped workloads and one
+    batch row of the long-context one, with one thread and with all of them: tokens*heads per second each."""
+    import oracle
+    out = {}
+    cases = [("gpt2_l128_m4", None), ("gpt2_b8_l1024_m2", None), ("gpt2_b32_l1024_m4", None), ("gqa_32k_m8", 1)]
+    for name, rows in cases:
+        w = synth.WORKLOADS[name]
+        sample = oracle_step_sample(w, rows or w.B)
+        units = (rows or w.B) * w.n_q_heads * w.L
+        res = {"sample": f"{rows or w.B} of {w.B} batch rows"}
+        for label, nthreads in (("threads_1", 1), ("threads_all", oracle.all_threads())):
+            oracle.set_threads(nthreads)
+            oracle_step(*sample)
+            t0 = time.perf_counter()
+            reps = 0
+            while reps < 50 and (reps == 0 or time.perf_counter() - t0 < budget_s / 2):
+                oracle_step(*sample)
+                reps += 1
+            dt = (time.perf_counter() - t0) / reps
+            res[label] = {"value": units / dt, "unit": UNIT, "cores": nthreads, "ms_per_step": dt * 1e3, "reps": reps}
+        out[name] = res
+    oracle.set_threads(oracle.all_threads())
+    return out
 
 
 def run_reference(args, w):
@@ -353,7 +383,26 @@ def time_pqv(lk, w, q, books, codes, v, steps: int, sm_mhz: float):
     # what the compression costs in accuracy on these inputs: against the fp16-V result of the same step
     ref = lk.lookat_attend(codes, v, q=q, codebooks=books)
     err = float((out - ref).abs().max())
+    # the same comparison on values a quantiser can compress (rows near a low-rank subspace, like the keys): 2 batch rows
+    structured = None
+    try:
+        rows = min(2, w.B)
+        wl = synth.Workload(**{**w.__dict__, "B": rows})
+        v_lr = torch.from_numpy(synth.make_values_lowrank(wl)).cuda()
+        books_lr = lv.lookat_fit_codebooks(v_lr[:, :, :max(1, n_fit // rows)].contiguous(), w.fit_iters, seed=w.seed + 2)
+        codes_lr = lv.lookat_encode_keys(v_lr, books_lr)
+        q2, c2 = q[:rows].contiguous(), codes[:rows].contiguous()
+        o_pq = lk.lookat_attend_pqv(c2, books_lr, codes_lr, q=q2, codebooks=books)
+        o_fp = lk.lookat_attend(c2, v_lr, q=q2, codebooks=books)
+        structured = {"values": "fp16(z A^T + 0.1 eps), rank as the keys", "batch_rows": rows,
+                      "max_abs_diff_to_fp16_values": float((o_pq - o_fp).abs().max()),
+                      "rms_of_fp16_values_output": float(o_fp.pow(2).mean().sqrt()),
+                      "relative_rms_error": float((o_pq - o_fp).pow(2).mean().sqrt() / o_fp.pow(2).mean().sqrt())}
+        del v_lr, codes_lr
+    except Exception as exc:
+        structured = {"error": str(exc)[:200]}
     return {"ms_per_step": ms, "tokens_heads_per_s": w.B * w.n_q_heads * w.L / (ms * 1e-3), "m_v": m_v, "K_v": 256,
+            "structured_values": structured,
             "launches_per_step": 2, "l2": f"{n_sets} copies of the codes in rotation",
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "note": f"(m + m_v) bytes per (token, KV head) pair; peak {which}.  The kernel is bound by its "
@@ -364,6 +413,139 @@ def time_pqv(lk, w, q, books, codes, v, steps: int, sm_mhz: float):
                               "note": "peak = 148 SMs x 128 B/clk x the median SM clock sampled during the timed decode steps"},
             "max_abs_diff_to_fp16_values": err,
             "note": "value compression is not part of the paper's method (its Section 5.2: future work)"}
+
+
+def timed_blocks(run_block, sync, min_seconds: float = MIN_TIMED_SECONDS, max_blocks: int = 400):
+    """Calls run_block() (one block of steps, enqueued on the current stream) between CUDA events until min_seconds of
+    device time have been timed; returns the blocks' durations in milliseconds."""
+    import torch
+    times = []
+    while len(times) < max_blocks and (not times or sum(times) < min_seconds * 1e3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        run_block()
+        e1.record()
+        sync()
+        times.append(e0.elapsed_time(e1))
+    return times
+
+
+def time_small_config(name: str, device_index: int):
+    """One GPT-2 shaped decode step (`lookat_decode_step`: append-encode, tables, scores, softmax, value sum, merge in
+    one launch) timed as a CUDA graph of back-to-back steps that rotate through enough copies of codes + V that every
+    step reads from HBM; beside it the same loop as plain host calls.  Codebooks: the workload's Lloyd iterations on the
+    cached keys."""
+    import torch
+
+    from paper_2601_10155_b200.binding import Lookat
+    w = synth.WORKLOADS[name]
+    side = torch.cuda.Stream(device=device_index)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    with torch.cuda.stream(side):
+        lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K, device=device_index, stream=side)
+        keys, v, q = dev(synth.make_keys(w)), dev(synth.make_values(w)), dev(synth.make_queries(w))
+        n_fit = w.fit_keys_per_head or w.B * w.L
+        books = lk.lookat_fit_codebooks(keys[:, :, :max(1, n_fit // w.B)].contiguous(), w.fit_iters, seed=w.seed)
+        codes = lk.lookat_encode_keys(keys, books)
+        n_sets = input_sets_needed(w)
+        cs = [codes.clone() for _ in range(n_sets)]
+        vs = [v.clone() for _ in range(n_sets)]
+        new_k = keys[:, :, w.L - 1].contiguous()
+        out = torch.empty((w.B, w.n_q_heads, w.d_v), dtype=torch.float32, device="cuda")
+
+        def step(i):
+            lk.lookat_decode_step(q, new_k, books, cs[i % n_sets], vs[i % n_sets], w.L - 1, out=out)
+
+        for i in range(max(3, min(n_sets, 16))):
+            step(i)
+        side.synchronize()
+        launches0 = lk.lookat_kernel_launches()
+        step(0)
+        launches_per_step = lk.lookat_kernel_launches() - launches0
+        n_in = max(n_sets, 32)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(n_in):
+                step(i)
+        graph.replay()
+        side.synchronize()
+        g_ms = timed_blocks(graph.replay, side.synchronize)
+        h_ms = timed_blocks(lambda: [step(i) for i in range(n_in)], side.synchronize, min_seconds=0.05)
+    ms = float(np.median(g_ms)) / n_in
+    alg = w.B * w.n_kv_heads * w.L * (w.m + 2 * w.d_v) + books.numel() * 4
+    peak, which = measured_peak("hbm_gbs", FALLBACK_HBM_GBS)
+    gbs = alg / (ms * 1e-3) / 1e9
+    return {"ms_per_step": ms, "us_per_step": ms * 1e3, "tokens_heads_per_s": w.B * w.n_q_heads * w.L / (ms * 1e-3),
+            "algorithmic_bytes": int(alg), "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak,
+            "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS, "peak_source": which,
+            "ms_per_step_host_calls": float(np.median(h_ms)) / n_in, "launches_per_step": int(launches_per_step),
+            "timing": f"CUDA graph of {n_in} steps, median of {len(g_ms)} replays", "l2": workload_config(w)["l2"],
+            "batch": w.B, "heads": w.n_q_heads, "seq_len": w.L, "m": w.m}
+
+
+def time_c2_replay(device_index: int, layers: int = 12, steps: int = 64):
+    """The attention of BASELINE config 2 replayed: 12 layers with their own head generators and codebooks (25 Lloyd
+    iterations on the layer's 32,768 prefill keys per head), batch 32 x 12 heads, caches with room for 1088 tokens that
+    64 decode steps grow from 1024 to 1088; every layer-step is one `lookat_decode_step` (the new key encoded on
+    append, then Algorithm 1 over the cache).  768 launches captured as one CUDA graph; 634 MB of codes + V per
+    token-step over the 12 layers, so every layer-step reads from HBM."""
+    import torch
+
+    from paper_2601_10155_b200.binding import Lookat
+    base = synth.WORKLOADS["gpt2_b32_l1024_m4"]
+    L0, cap = base.L, base.L + steps
+    side = torch.cuda.Stream(device=device_index)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    with torch.cuda.stream(side):
+        lk = Lookat(base.n_q_heads, base.n_kv_heads, base.d_k, base.d_v, base.m, base.K, device=device_index, stream=side)
+        per_layer = []
+        fit_ms = 0.0
+        for layer in range(layers):
+            w = synth.Workload(**{**base.__dict__, "layer": layer})
+            keys = dev(synth.make_keys(w, n_tokens=cap))
+            v = dev(synth.make_values(w, n_tokens=cap))
+            q = dev(synth.make_queries(w))
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            books = lk.lookat_fit_codebooks(keys[:, :, :L0].contiguous(), w.fit_iters, seed=w.seed)
+            e1.record()
+            cache = torch.zeros((w.B, w.n_kv_heads, cap, w.m), dtype=torch.uint8, device="cuda")
+            lk.lookat_encode_keys(keys[:, :, :L0].contiguous(), books, codes=cache, pos=0)
+            new_keys = keys[:, :, L0:].permute(2, 0, 1, 3).contiguous()       # [step][B][H][d_k]
+            side.synchronize()
+            fit_ms += e0.elapsed_time(e1)
+            per_layer.append((q, new_keys, books, cache, v))
+            del keys
+        out = torch.empty((base.B, base.n_q_heads, base.d_v), dtype=torch.float32, device="cuda")
+
+        def replay():
+            for t in range(steps):
+                for q, new_keys, books, cache, v in per_layer:
+                    lk.lookat_decode_step(q, new_keys[t], books, cache, v, L0 + t, out=out)
+
+        replay()                                            # also grows the context's scratch to its final size
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            replay()
+        graph.replay()
+        side.synchronize()
+        g_ms = timed_blocks(graph.replay, side.synchronize)
+        h_ms = timed_blocks(replay, side.synchronize, min_seconds=0.05)
+    total_ms = float(np.median(g_ms))
+    n = layers * steps
+    pairs = sum(base.B * base.n_kv_heads * (L0 + t + 1) for t in range(steps)) * layers
+    alg = pairs * (base.m + 2 * base.d_v) + n * per_layer[0][2].numel() * 4
+    peak, which = measured_peak("hbm_gbs", FALLBACK_HBM_GBS)
+    gbs = alg / (total_ms * 1e-3) / 1e9
+    return {"layers": layers, "steps": steps, "batch": base.B, "heads": base.n_q_heads, "seq_len": f"{L0} -> {cap}",
+            "total_ms": total_ms, "us_per_layer_step": total_ms * 1e3 / n, "ms_per_generated_token": total_ms / steps,
+            "tokens_heads_per_s": pairs * (base.n_q_heads // base.n_kv_heads) / (total_ms * 1e-3),
+            "algorithmic_bytes": int(alg), "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak,
+            "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS, "peak_source": which,
+            "total_ms_host_calls": float(np.median(h_ms)), "launches": n,
+            "timing": f"one CUDA graph of {n} launches, median of {len(g_ms)} replays",
+            "setup_fit_ms_all_layers": fit_ms}
 
 
 def run_lookat(args, w):
@@ -435,22 +617,33 @@ def run_lookat(args, w):
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
-    launches0 = lk.lookat_kernel_launches()
-    lk.lookat_set_timing(True)
+    # a block = exactly `steps` steps between two events; blocks are repeated until MIN_TIMED_SECONDS have been timed
+    # (every rank runs the same number: the count is fixed from one untimed block), the median block is reported
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler.start()
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
-    sampler.sample()
     barrier()
+    (probe_ms,) = max_over_ranks([e0.elapsed_time(e1)], "cuda")
+    n_blocks = int(min(400, max(1, np.ceil(MIN_TIMED_SECONDS * 1e3 / max(probe_ms, 1e-3)))))
+    launches0 = lk.lookat_kernel_launches()
+    lk.lookat_set_timing(min(args.steps * n_blocks, 40000))
+    block_ms = []
+    sampler.start()
+    for _ in range(n_blocks):
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        barrier()
+        block_ms.append(e0.elapsed_time(e1))
+    sampler.sample()
     sampler.stop()
-    lk.lookat_set_timing(False)
-    elapsed_ms = e0.elapsed_time(e1)
-    attend_ms = lk.lookat_attend_kernel_ms()
-    launches = lk.lookat_kernel_launches() - launches0
-    elapsed_ms, attend_ms = max_over_ranks([elapsed_ms, attend_ms], "cuda")
+    lk.lookat_set_timing(0)
+    kstats = lk.lookat_attend_kernel_stats()
+    launches = (lk.lookat_kernel_launches() - launches0) // n_blocks
+    elapsed_ms, attend_ms = max_over_ranks([float(np.median(block_ms)), kstats["median"]], "cuda")
 
     # ---- end to end: host buffers in, host buffer out, through the C-ABI call ----
     q_host = torch.from_numpy(q_np).pin_memory()
@@ -497,8 +690,11 @@ def run_lookat(args, w):
             "config": workload_config(w),
             "roofline": {"bound": "hbm", "kernel": "attend_stream_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                         "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,
-                         "kernel_ms": attend_ms, "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+                         "traffic": traffic, "traffic_source": ATTEND_TRAFFIC_SOURCE if traffic else None,
+                         "algorithmic_bytes_per_launch": alg_bytes,
+                         "kernel_ms": attend_ms, "kernel_ms_min": kstats["min"], "kernel_ms_median": kstats["median"],
+                         "kernel_ms_max": kstats["max"], "kernel_ms_mean": kstats["mean"], "kernel_launches_timed": kstats["n"],
+                         "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
                          "read_ceiling_gbs": read_ceiling,
                          "frac_of_read_ceiling": None if not read_ceiling else achieved / read_ceiling},
             "e2e": {"value": units_per_step / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT,
@@ -506,6 +702,8 @@ def run_lookat(args, w):
                     "d2h_bytes_per_step": int(out_host.numel() * 4), "ms_per_step": e2e_ms / e2e_steps,
                     "matches_device_path": same},
             "gpu_launches": int(launches),
+            "blocks": n_blocks, "block_ms_min": float(min(block_ms)), "block_ms_max": float(max(block_ms)),
+            "timing": f"median of {n_blocks} blocks of {args.steps} steps (CUDA events, barrier between blocks)",
             "clocks": sampler.summary(),
             "step_hbm_gbs": (alg_bytes + books.numel() * 4) / (ms_per_step * 1e-3) / 1e9,
             "setup": {"fit_ms": fit_ms, "bulk_encode_ms": enc_ms,
@@ -514,10 +712,14 @@ def run_lookat(args, w):
         }
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = time_oracle(w)
+            try:
+                line["cpu_baseline_configs"] = time_oracle_configs()
+            except Exception as exc:
+                line["cpu_baseline_configs"] = {"error": str(exc)[:200]}
         if pqv is not None:
             line["pqv"] = pqv
         if world == 1 and args.prefill:
-            del keys, v, codes, code_sets, v_sets
+            keys = v = codes = code_sets = v_sets = None
             torch.cuda.empty_cache()
             try:
                 line["prefill"] = time_prefill(local_rank)
@@ -527,6 +729,21 @@ def run_lookat(args, w):
                 line["encode_1m"] = time_encode_1m(local_rank)
             except Exception as exc:
                 line["encode_1m"] = {"error": str(exc)[:200]}
+        if world == 1 and args.small:
+            keys = v = codes = code_sets = v_sets = None
+            torch.cuda.empty_cache()
+            small = {}
+            for name in SMALL_WORKLOADS:
+                try:
+                    small[name] = time_small_config(name, local_rank)
+                except Exception as exc:
+                    small[name] = {"error": str(exc)[:200]}
+                torch.cuda.empty_cache()
+            line["small_configs"] = small
+            try:
+                line["c2_replay"] = time_c2_replay(local_rank)
+            except Exception as exc:
+                line["c2_replay"] = {"error": str(exc)[:200]}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
@@ -546,6 +763,8 @@ def main():
                     help="skip the extra timing of the causal multi-query kernel")
     ap.add_argument("--no-pqv", dest="pqv", action="store_false",
                     help="skip the extra leg that times decode attention with product-quantised values")
+    ap.add_argument("--no-small", dest="small", action="store_false",
+                    help="skip the GPT-2 shaped decode steps and the 12-layer x 64-step replay")
     ap.add_argument("--only-prefill", action="store_true",
                     help="time only the causal multi-query kernel (prints its object alone)")
     ap.add_argument("--prefill-batch", type=int, default=0, help="smaller prefill case: batch rows")

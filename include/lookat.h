@@ -313,13 +313,18 @@ lookat_status lookat_selftest_timeout(lookat_ctx *ctx);
 /* Number of kernels this context has launched since it was created. */
 uint64_t lookat_kernel_launches(const lookat_ctx *ctx);
 
-/* Average device time in milliseconds of the attend kernel over the launches
- * made while timing was enabled (CUDA events on the context's stream).
- * lookat_set_timing(ctx, 1) resets and starts, (ctx, 0) stops;
- * lookat_attend_kernel_ms synchronises the events and returns the mean, or
- * -1 when nothing was timed. */
-void lookat_set_timing(lookat_ctx *ctx, int32_t enabled);
+/* Device time of the attend kernel per launch (measurement aid; the paper has
+ * no counterpart): CUDA events on the context's stream around every launch
+ * made while timing is on, read only afterwards, so the timed run itself is
+ * never synchronised.  lookat_set_timing(ctx, n) with n >= 1 resets and starts
+ * with room for n launches (at least 64; later launches go untimed), n <= 0
+ * stops.  lookat_attend_kernel_stats synchronises on the recorded events and
+ * fills stats[0..3] = minimum, median, maximum and mean in milliseconds; it
+ * returns the number of launches timed (0: stats untouched).
+ * lookat_attend_kernel_ms returns that mean, or -1 when nothing was timed. */
+void lookat_set_timing(lookat_ctx *ctx, int32_t launches);
 double lookat_attend_kernel_ms(lookat_ctx *ctx);
+int32_t lookat_attend_kernel_stats(lookat_ctx *ctx, double *stats);
 
 #ifdef __cplusplus
 }

@@ -50,6 +50,16 @@ def _f16(a):
 
 def n_threads() -> int:
     """Threads the OpenMP regions of the oracle will use."""
+    return int(_load().oracle_set_num_threads(0))
+
+
+def set_threads(n: int) -> int:
+    """Use n threads from now on (n <= 0: leave as is); returns the setting in force."""
+    return int(_load().oracle_set_num_threads(int(n)))
+
+
+def all_threads() -> int:
+    """The cores this process may run on (what OpenMP uses unless told otherwise)."""
     env = os.environ.get("OMP_NUM_THREADS")
     if env:
         return int(env.split(",")[0])

@@ -23,9 +23,18 @@
  * subspace) units; every unit runs the paper's steps in order.
  */
 #include <math.h>
+#include <omp.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
+
+/* How many threads the OpenMP loops over independent units use from now on (the benchmark times the oracle with
+ * one thread and with all of them); returns the setting in force.  No arithmetic depends on it. */
+int oracle_set_num_threads(int n)
+{
+    if (n > 0) omp_set_num_threads(n);
+    return omp_get_max_threads();
+}
 
 /* fp16 bit pattern -> double, exact (IEEE binary16: 1 sign, 5 exponent, 10 fraction bits). */
 static double half_to_double(uint16_t h)

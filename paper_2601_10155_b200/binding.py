@@ -20,7 +20,7 @@ EXPORTS = [
     "lookat_create", "lookat_destroy", "lookat_last_error", "lookat_fit_codebooks",
     "lookat_encode_keys", "lookat_build_lut", "lookat_attend", "lookat_attend_static", "lookat_attend_pqv",
     "lookat_attend_prefill", "lookat_decode_step", "lookat_decode_step_host",
-    "lookat_kernel_launches", "lookat_probe_read_bandwidth", "lookat_selftest_timeout", "lookat_set_prefill_form", "lookat_set_timing", "lookat_attend_kernel_ms",
+    "lookat_kernel_launches", "lookat_probe_read_bandwidth", "lookat_selftest_timeout", "lookat_set_prefill_form", "lookat_set_timing", "lookat_attend_kernel_ms", "lookat_attend_kernel_stats",
 ]
 
 STATUS = {0: "LOOKAT_OK", 1: "LOOKAT_ERR_INVALID_ARG", 2: "LOOKAT_ERR_UNSUPPORTED",
@@ -89,6 +89,8 @@ def load_library() -> ctypes.CDLL:
     lib.lookat_set_timing.restype = None
     lib.lookat_attend_kernel_ms.argtypes = [vp]
     lib.lookat_attend_kernel_ms.restype = ctypes.c_double
+    lib.lookat_attend_kernel_stats.argtypes = [vp, ctypes.POINTER(ctypes.c_double)]
+    lib.lookat_attend_kernel_stats.restype = i32
     _lib = lib
     return lib
 
@@ -322,8 +324,15 @@ class Lookat:
         code = {"auto": 0, "tables": 1, "contraction": 2}.get(form, form)
         self._check(self._lib.lookat_set_prefill_form(self._h, int(code)))
 
-    def lookat_set_timing(self, enabled: bool):
-        self._lib.lookat_set_timing(self._h, 1 if enabled else 0)
+    def lookat_set_timing(self, launches):
+        """launches >= 1: time up to that many attend launches from now on (True = 64); 0 / False: stop."""
+        self._lib.lookat_set_timing(self._h, 64 if launches is True else int(launches))
+
+    def lookat_attend_kernel_stats(self):
+        """{'n', 'min', 'median', 'max', 'mean'} of the timed attend launches in milliseconds, or None."""
+        st = (ctypes.c_double * 4)()
+        n = int(self._lib.lookat_attend_kernel_stats(self._h, st))
+        return None if n == 0 else {"n": n, "min": st[0], "median": st[1], "max": st[2], "mean": st[3]}
 
     def lookat_attend_kernel_ms(self) -> float:
         return float(self._lib.lookat_attend_kernel_ms(self._h))

@@ -2,6 +2,7 @@
 // the kernel launchers.  Every entry point is declared in include/lookat.h.
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -262,13 +263,6 @@ lookat_status lookat_create(const lookat_config *cfg, int device, void *cuda_str
         cudaGetLastError();
         ctx->timeout_flag = nullptr;                       // the tcgen05 prefill kernel is then not used
     }
-    for (int i = 0; i < kTimingSlots; ++i) {
-        if (cudaEventCreate(&ctx->ev0[i]) != cudaSuccess || cudaEventCreate(&ctx->ev1[i]) != cudaSuccess) {
-            cudaGetLastError();
-            lookat_destroy(reinterpret_cast<lookat_ctx *>(ctx));
-            return LOOKAT_ERR_CUDA;
-        }
-    }
     *out = reinterpret_cast<lookat_ctx *>(ctx);
     return LOOKAT_OK;
 }
@@ -284,10 +278,13 @@ void lookat_destroy(lookat_ctx *handle)
     for (void *p : bufs)
         if (p) cudaFree(p);
     if (ctx->timeout_flag) cudaFreeHost(ctx->timeout_flag);
-    for (int i = 0; i < kTimingSlots; ++i) {
+    for (int i = 0; i < ctx->ev_cap; ++i) {
         if (ctx->ev0[i]) cudaEventDestroy(ctx->ev0[i]);
         if (ctx->ev1[i]) cudaEventDestroy(ctx->ev1[i]);
     }
+    free(ctx->ev0);
+    free(ctx->ev1);
+    free(ctx->times_ms);
     cudaGetLastError();
     delete ctx;
 }
@@ -359,34 +356,81 @@ lookat_status lookat_selftest_timeout(lookat_ctx *handle)
     return launch_timeout_selftest(ctx);
 }
 
-void lookat_set_timing(lookat_ctx *handle, int32_t enabled)
+// the recorded event pairs into times_ms (synchronises on them)
+static void drain_timing(Ctx *ctx)
+{
+    for (int s = 0; s < ctx->ev_count; ++s) {
+        float ms = 0.f;
+        cudaEventSynchronize(ctx->ev1[s]);
+        if (cudaEventElapsedTime(&ms, ctx->ev0[s], ctx->ev1[s]) == cudaSuccess && ctx->n_times < ctx->ev_cap)
+            ctx->times_ms[ctx->n_times++] = ms;
+    }
+    ctx->ev_count = 0;
+}
+
+void lookat_set_timing(lookat_ctx *handle, int32_t launches)
 {
     if (!handle) return;
     Ctx *ctx = reinterpret_cast<Ctx *>(handle);
-    if (enabled) {
-        ctx->timed_ms = 0.0;
-        ctx->timed_n = 0;
-        ctx->ev_next = 0;
-        memset(ctx->ev_used, 0, sizeof(ctx->ev_used));
+    if (launches <= 0) {
+        ctx->timing = 0;
+        return;
     }
-    ctx->timing = enabled ? 1 : 0;
+    const int want = launches < 64 ? 64 : launches;
+    if (want > ctx->ev_cap) {
+        DeviceGuard guard(ctx->device);
+        cudaEvent_t *e0 = static_cast<cudaEvent_t *>(realloc(ctx->ev0, sizeof(cudaEvent_t) * want));
+        if (e0) ctx->ev0 = e0;
+        cudaEvent_t *e1 = static_cast<cudaEvent_t *>(realloc(ctx->ev1, sizeof(cudaEvent_t) * want));
+        if (e1) ctx->ev1 = e1;
+        float *t = static_cast<float *>(realloc(ctx->times_ms, sizeof(float) * want));
+        if (t) ctx->times_ms = t;
+        if (e0 && e1 && t) {
+            while (ctx->ev_cap < want) {
+                ctx->ev0[ctx->ev_cap] = ctx->ev1[ctx->ev_cap] = nullptr;
+                if (cudaEventCreate(&ctx->ev0[ctx->ev_cap]) != cudaSuccess || cudaEventCreate(&ctx->ev1[ctx->ev_cap]) != cudaSuccess) {
+                    cudaGetLastError();
+                    if (ctx->ev0[ctx->ev_cap]) cudaEventDestroy(ctx->ev0[ctx->ev_cap]);
+                    break;                                 // fewer launches are timed than asked for
+                }
+                ctx->ev_cap += 1;
+            }
+        }
+    }
+    ctx->ev_count = 0;
+    ctx->n_times = 0;
+    ctx->timing = 1;
 }
 
 double lookat_attend_kernel_ms(lookat_ctx *handle)
 {
-    if (!handle) return -1.0;
+    double st[4];
+    return lookat_attend_kernel_stats(handle, st) > 0 ? st[3] : -1.0;
+}
+
+int32_t lookat_attend_kernel_stats(lookat_ctx *handle, double *stats)
+{
+    if (!handle || !stats) return 0;
     Ctx *ctx = reinterpret_cast<Ctx *>(handle);
-    for (int s = 0; s < kTimingSlots; ++s) {
-        if (!ctx->ev_used[s]) continue;
-        float ms = 0.f;
-        cudaEventSynchronize(ctx->ev1[s]);
-        if (cudaEventElapsedTime(&ms, ctx->ev0[s], ctx->ev1[s]) == cudaSuccess) {
-            ctx->timed_ms += ms;
-            ctx->timed_n += 1;
-        }
-        ctx->ev_used[s] = 0;
+    DeviceGuard guard(ctx->device);
+    drain_timing(ctx);
+    const int n = ctx->n_times;
+    if (n == 0) return 0;
+    // insertion sort of a copy would do; the array is small and owned: sort in place
+    float *t = ctx->times_ms;
+    for (int i = 1; i < n; ++i) {
+        const float v = t[i];
+        int k = i - 1;
+        while (k >= 0 && t[k] > v) { t[k + 1] = t[k]; --k; }
+        t[k + 1] = v;
     }
-    return ctx->timed_n ? ctx->timed_ms / (double)ctx->timed_n : -1.0;
+    double sum = 0.0;
+    for (int i = 0; i < n; ++i) sum += t[i];
+    stats[0] = t[0];
+    stats[1] = (n & 1) ? t[n / 2] : 0.5 * ((double)t[n / 2 - 1] + t[n / 2]);
+    stats[2] = t[n - 1];
+    stats[3] = sum / n;
+    return n;
 }
 
 lookat_status lookat_build_lut(lookat_ctx *handle, const void *q, int32_t B, const float *codebooks, float *lut)

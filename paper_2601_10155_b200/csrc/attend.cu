@@ -733,19 +733,10 @@ lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_
 lookat_status launch_attend(Ctx *ctx, const AttendArgs &a)
 {
     cudaEvent_t e0 = nullptr, e1 = nullptr;
-    if (ctx->timing) {
-        const int s = ctx->ev_next;
-        if (ctx->ev_used[s]) {
-            float ms = 0.f;
-            cudaEventSynchronize(ctx->ev1[s]);
-            if (cudaEventElapsedTime(&ms, ctx->ev0[s], ctx->ev1[s]) == cudaSuccess) {
-                ctx->timed_ms += ms;
-                ctx->timed_n += 1;
-            }
-            ctx->ev_used[s] = 0;
-        }
-        e0 = ctx->ev0[s];
-        e1 = ctx->ev1[s];
+    const bool timed = ctx->timing && ctx->ev_count < ctx->ev_cap;     // launches beyond the room asked for go untimed
+    if (timed) {
+        e0 = ctx->ev0[ctx->ev_count];
+        e1 = ctx->ev1[ctx->ev_count];
         cudaEventRecord(e0, ctx->stream);
     }
     lookat_status st;
@@ -760,10 +751,9 @@ lookat_status launch_attend(Ctx *ctx, const AttendArgs &a)
         attend_generic_kernel<<<grid, kGenThreads, 0, ctx->stream>>>(a);
         st = check_launch(ctx, "attend_generic_kernel");
     }
-    if (ctx->timing) {
+    if (timed) {
         cudaEventRecord(e1, ctx->stream);
-        ctx->ev_used[ctx->ev_next] = 1;
-        ctx->ev_next = (ctx->ev_next + 1) % kTimingSlots;
+        ctx->ev_count += 1;
     }
     return st;
 }

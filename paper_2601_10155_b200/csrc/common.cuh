@@ -10,8 +10,6 @@
 
 namespace lookat {
 
-constexpr int kTimingSlots = 64;
-
 // Context: configuration, stream, scratch owned by the library.
 struct Ctx {
     lookat_config cfg;
@@ -47,13 +45,12 @@ struct Ctx {
     float *step_out;
     size_t step_q_cap, step_k_cap, step_out_cap;   // bytes
 
-    // per-launch timing of the attend kernel
+    // per-launch timing of the attend kernel: an event pair per timed launch, read only after the timed run
     int timing;
-    cudaEvent_t ev0[kTimingSlots], ev1[kTimingSlots];
-    int ev_used[kTimingSlots];
-    int ev_next;
-    double timed_ms;
-    long timed_n;
+    cudaEvent_t *ev0, *ev1;    // [ev_cap]
+    int ev_cap, ev_count;      // pairs created / recorded since timing was switched on
+    float *times_ms;           // [ev_cap] the launches' durations, filled when the events are drained
+    int n_times;
 };
 
 lookat_status set_error(Ctx *ctx, lookat_status st, const char *fmt, ...);

@@ -343,9 +343,11 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         constexpr int kTokStep = kUmProducers / Lay::kIds;
         const int code_bytes = kUmChunk * a.m;                 // codes of one chunk, staged in shared memory a chunk ahead
         auto fetch_codes = [&](int c) {                        // 4-byte cp.async pieces; pieces beyond the CTA's tokens stay unread
+            // a piece that starts below the limit is read whole: with m < 4 it can reach past the CTA's last token, never
+            // past the row (L_max * m is a multiple of 4); tokens past the limit are zeroed when the keys are rebuilt
             const long long first = (long long)c * code_bytes, limit = t_end * a.m;
             for (int o = ptid * 4; o < code_bytes; o += kUmProducers * 4)
-                if (first + o + 4 <= limit)
+                if (first + o < limit)
                     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(um_smem(codes_s) + (c & 1) * 1024 + o),
                                  "l"(codes + first + o)
                                  : "memory");

@@ -136,6 +136,19 @@ def make_values(w: Workload, n_tokens: int | None = None) -> np.ndarray:
     return v
 
 
+def make_values_lowrank(w: Workload, n_tokens: int | None = None) -> np.ndarray:
+    """fp16 values [B][n_kv_heads][n_tokens][d_v] with the structure of the keys (rows near a rank-`rank` subspace of
+    the head, plus noise) instead of iid N(0,1): what a value quantiser can compress.  Only the quantised-values leg
+    of the benchmark uses it."""
+    L = w.L if n_tokens is None else n_tokens
+    v = np.empty((w.B, w.n_kv_heads, L, w.d_v), dtype=np.float16)
+    for h in range(w.n_kv_heads):
+        A = head_mixing_matrix(w.seed, w.layer, h + 1000, w.d_v, w.rank, w.scales)
+        rng = np.random.default_rng([w.seed, w.layer, h, 6])
+        v[:, h] = draw_rows(rng, A, w.B * L).reshape(w.B, L, w.d_v)
+    return v
+
+
 def make_queries(w: Workload, q_scale: float = 1.0) -> np.ndarray:
     """fp16 queries [B][n_q_heads][d_k]; query head hq shares the subspace of
     KV head hq // g.  q_scale < 1 flattens the softmax (the plain generator

@@ -408,6 +408,7 @@ def test_invalid_arguments_are_rejected_without_launching():
     (dict(B=1, n_q_heads=2, n_kv_heads=1, d_k=128, d_v=64, m=16, K=200, L=450), 300, 150),  # 3 query tiles, ragged, K < 256
     (dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=128, m=8, K=256, L=257), 257, 0),     # d_k 64; one row in the last tile
     (dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=64, m=16, K=256, L=90), 90, 0),       # d_sub 4: tables only
+    (dict(B=1, n_q_heads=4, n_kv_heads=1, d_k=64, d_v=128, m=2, K=16, L=300), 259, 41),     # m 2: a CTA's last token has an odd index
 ])
 @pytest.mark.parametrize("q_scale", [1.0, 0.1])
 @pytest.mark.parametrize("form", ["tables", "contraction"])
