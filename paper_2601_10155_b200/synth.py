@@ -180,3 +180,31 @@ def small_workload(name: str = "small", **kw) -> Workload:
                 L=200, m=4, K=16, rank=8, scales="loguniform", fit_iters=5)
     base.update(kw)
     return Workload(**base)
+
+
+def gpt2_weights(seed: int, n_layer: int = 12, n_head: int = 12, d_model: int = 768, vocab: int = 50257,
+                 n_pos: int = 1088, plain_init: bool = True) -> dict:
+    """Random-init GPT-2 shaped weights as fp16 arrays in a plain dict (no arithmetic of the model here).  Linear layers
+    are stored transposed, [out][in].  plain_init: GPT-2's own scheme -- N(0, 0.02), residual projections scaled by
+    1/sqrt(2 n_layer), zero biases, unit LayerNorm gains.  Otherwise gains and biases are random too, so that a dropped
+    bias or gain cannot hide in a test."""
+    rng = np.random.default_rng([seed, 77])
+    h = lambda a: a.astype(np.float16)
+    d = d_model
+    nrm = lambda *shape, s=0.02: rng.standard_normal(shape) * s
+    gain = (lambda: np.ones(d)) if plain_init else (lambda: 1.0 + 0.2 * rng.standard_normal(d))
+    bias = (lambda n: np.zeros(n)) if plain_init else (lambda n: 0.05 * rng.standard_normal(n))
+    layers = []
+    for _ in range(n_layer):
+        layers.append(dict(
+            ln1_g=h(gain()), ln1_b=h(bias(d)), w_qkv=h(nrm(3 * d, d)), b_qkv=h(bias(3 * d)),
+            w_o=h(nrm(d, d, s=0.02 / np.sqrt(2.0 * n_layer))), b_o=h(bias(d)),
+            ln2_g=h(gain()), ln2_b=h(bias(d)), w_fc=h(nrm(4 * d, d)), b_fc=h(bias(4 * d)),
+            w_pr=h(nrm(d, 4 * d, s=0.02 / np.sqrt(2.0 * n_layer))), b_pr=h(bias(d))))
+    return dict(n_layer=n_layer, n_head=n_head, d_model=d, vocab=vocab, n_pos=n_pos, wte=h(nrm(vocab, d)),
+                wpe=h(nrm(n_pos, d, s=0.01)), lnf_g=h(gain()), lnf_b=h(bias(d)), layers=layers)
+
+
+def token_ids(seed: int, B: int, T: int, vocab: int) -> np.ndarray:
+    """Uniform-random token ids int32 [B][T]."""
+    return np.random.default_rng([seed, 78]).integers(0, vocab, (B, T), dtype=np.int32)
