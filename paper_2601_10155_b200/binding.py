@@ -21,6 +21,10 @@ EXPORTS = [
     "lookat_encode_keys", "lookat_build_lut", "lookat_attend", "lookat_attend_static", "lookat_attend_pqv",
     "lookat_attend_prefill", "lookat_decode_step", "lookat_decode_step_host",
     "lookat_kernel_launches", "lookat_probe_read_bandwidth", "lookat_selftest_timeout", "lookat_set_prefill_form", "lookat_set_timing", "lookat_attend_kernel_ms", "lookat_attend_kernel_stats",
+    # include/lookat_gpt2.h
+    "lookat_gpt2_create", "lookat_gpt2_destroy", "lookat_gpt2_last_error", "lookat_gpt2_set_weights", "lookat_gpt2_prefill",
+    "lookat_gpt2_decode", "lookat_gpt2_layer_state", "lookat_gpt2_position", "lookat_gpt2_kernel_launches",
+    "lookat_linear", "lookat_linear_qkv", "lookat_layernorm", "lookat_embed", "lookat_causal_attention", "lookat_argmax",
 ]
 
 STATUS = {0: "LOOKAT_OK", 1: "LOOKAT_ERR_INVALID_ARG", 2: "LOOKAT_ERR_UNSUPPORTED",
@@ -37,6 +41,18 @@ class lookat_config(ctypes.Structure):
     _fields_ = [("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("m", ctypes.c_int32),
                 ("K", ctypes.c_int32), ("scale", ctypes.c_float)]
+
+
+class lookat_gpt2_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("n_layer", "n_head", "d_model", "vocab", "n_pos", "m", "K", "fit_iters",
+                                              "keep_prompt_keys")]
+
+
+LAYER_FIELDS = ("ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_o", "b_o", "ln2_g", "ln2_b", "w_fc", "b_fc", "w_pr", "b_pr")
+
+
+class lookat_gpt2_layer(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in LAYER_FIELDS]
 
 
 _lib = None
@@ -91,6 +107,37 @@ def load_library() -> ctypes.CDLL:
     lib.lookat_attend_kernel_ms.restype = ctypes.c_double
     lib.lookat_attend_kernel_stats.argtypes = [vp, ctypes.POINTER(ctypes.c_double)]
     lib.lookat_attend_kernel_stats.restype = i32
+    # the GPT-2 harness (include/lookat_gpt2.h)
+    lib.lookat_gpt2_create.argtypes = [ctypes.POINTER(lookat_gpt2_config), ctypes.c_int, vp, i32, i32, ctypes.POINTER(vp)]
+    lib.lookat_gpt2_create.restype = i32
+    lib.lookat_gpt2_destroy.argtypes = [vp]
+    lib.lookat_gpt2_destroy.restype = None
+    lib.lookat_gpt2_last_error.argtypes = [vp]
+    lib.lookat_gpt2_last_error.restype = ctypes.c_char_p
+    lib.lookat_gpt2_set_weights.argtypes = [vp, vp, vp, vp, vp, ctypes.POINTER(lookat_gpt2_layer)]
+    lib.lookat_gpt2_set_weights.restype = i32
+    lib.lookat_gpt2_prefill.argtypes = [vp, vp, i32, u64, vp]
+    lib.lookat_gpt2_prefill.restype = i32
+    lib.lookat_gpt2_decode.argtypes = [vp, vp, vp, vp, vp]
+    lib.lookat_gpt2_decode.restype = i32
+    lib.lookat_gpt2_layer_state.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
+    lib.lookat_gpt2_layer_state.restype = i32
+    lib.lookat_gpt2_position.argtypes = [vp]
+    lib.lookat_gpt2_position.restype = i32
+    lib.lookat_gpt2_kernel_launches.argtypes = [vp]
+    lib.lookat_gpt2_kernel_launches.restype = ctypes.c_uint64
+    lib.lookat_linear.argtypes = [vp, vp, i32, vp, vp, i64, i32, i32, i32, vp, vp, i32]
+    lib.lookat_linear.restype = i32
+    lib.lookat_linear_qkv.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, i64, i64, vp, i64, i64, vp, i64, i64]
+    lib.lookat_linear_qkv.restype = i32
+    lib.lookat_layernorm.argtypes = [vp, vp, vp, vp, i64, i32, vp]
+    lib.lookat_layernorm.restype = i32
+    lib.lookat_embed.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]
+    lib.lookat_embed.restype = i32
+    lib.lookat_causal_attention.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, vp]
+    lib.lookat_causal_attention.restype = i32
+    lib.lookat_argmax.argtypes = [vp, vp, i32, i32, vp]
+    lib.lookat_argmax.restype = i32
     _lib = lib
     return lib
 
@@ -336,6 +383,160 @@ class Lookat:
 
     def lookat_attend_kernel_ms(self) -> float:
         return float(self._lib.lookat_attend_kernel_ms(self._h))
+
+
+    # -- the GPT-2 harness's kernels one by one (include/lookat_gpt2.h) ------------
+    def lookat_linear(self, x, w_t, bias=None, gelu=False, residual=None, out=None, out_fp16=True):
+        M, K = x.shape
+        N = w_t.shape[0]
+        if out is None:
+            out = torch.empty((M, N), dtype=torch.float16 if out_fp16 else torch.float32, device=self.device)
+        if x.dtype not in (torch.float16, torch.float32):
+            raise TypeError("x must be fp16 or fp32")
+        self._check(self._lib.lookat_linear(
+            self._h, _dev(x, x.dtype, "x", (M, K)), 1 if x.dtype == torch.float32 else 0, _dev(w_t, torch.float16, "w_t", (N, K)),
+            _dev(bias, torch.float16, "bias", (N,)), M, N, K, 1 if gelu else 0, _dev(residual, torch.float32, "residual", (M, N)),
+            _dev(out, torch.float16 if out_fp16 else torch.float32, "out", (M, N)), 1 if out_fp16 else 0))
+        return out
+
+    def lookat_linear_qkv(self, x, w_t, bias, B, T, n_head, q, k, v, q_off=0, k_off=0, v_off=0):
+        d = n_head * 64
+        self._check(self._lib.lookat_linear_qkv(
+            self._h, _dev(x, torch.float16, "x", (B * T, d)), _dev(w_t, torch.float16, "w_t", (3 * d, d)),
+            _dev(bias, torch.float16, "bias", (3 * d,)), B, T, n_head,
+            _dev(q, torch.float16, "q"), q.shape[2], q_off, _dev(k, torch.float16, "k"), k.shape[2], k_off,
+            _dev(v, torch.float16, "v"), v.shape[2], v_off))
+        return q, k, v
+
+    def lookat_layernorm(self, x, gain, bias, out=None):
+        rows, d = x.shape
+        if out is None:
+            out = torch.empty((rows, d), dtype=torch.float16, device=self.device)
+        self._check(self._lib.lookat_layernorm(self._h, _dev(x, torch.float32, "x"), _dev(gain, torch.float16, "gain", (d,)),
+                                               _dev(bias, torch.float16, "bias", (d,)), rows, d, _dev(out, torch.float16, "out", (rows, d))))
+        return out
+
+    def lookat_embed(self, ids, wte, wpe, pos0=0, out=None):
+        B, T = ids.shape
+        vocab, d = wte.shape
+        if out is None:
+            out = torch.empty((B, T, d), dtype=torch.float32, device=self.device)
+        self._check(self._lib.lookat_embed(self._h, _dev(ids, torch.int32, "ids"), _dev(wte, torch.float16, "wte"),
+                                           _dev(wpe, torch.float16, "wpe"), B, T, pos0, d, vocab, _dev(out, torch.float32, "out", (B, T, d))))
+        return out
+
+    def lookat_causal_attention(self, q, k, v, out=None):
+        B, H, T, dh = q.shape
+        if out is None:
+            out = torch.empty((B, T, H * dh), dtype=torch.float16, device=self.device)
+        self._check(self._lib.lookat_causal_attention(self._h, _dev(q, torch.float16, "q", (B, H, T, 64)), _dev(k, torch.float16, "k", (B, H, T, 64)),
+                                                      _dev(v, torch.float16, "v"), B, H, T, v.shape[2], _dev(out, torch.float16, "out", (B, T, H * 64))))
+        return out
+
+    def lookat_argmax(self, logits, out=None):
+        rows, n = logits.shape
+        if out is None:
+            out = torch.empty((rows,), dtype=torch.int32, device=self.device)
+        self._check(self._lib.lookat_argmax(self._h, _dev(logits, torch.float32, "logits"), rows, n, _dev(out, torch.int32, "out", (rows,))))
+        return out
+
+
+class LookatGpt2:
+    """The GPT-2 decoder harness (include/lookat_gpt2.h): argument marshalling only.  `weights` is the dict of fp16
+    numpy arrays the seeded generator makes; they are uploaded once and kept alive here."""
+
+    def __init__(self, weights, B, capacity, m, K, fit_iters, device=0, stream=None, keep_prompt_keys=False):
+        self._lib = load_library()
+        self._h = None
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the LOOKAT library runs on the GPU only")
+        self.device = torch.device("cuda", device)
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        self.stream = stream
+        w = weights
+        self.cfg = lookat_gpt2_config(w["n_layer"], w["n_head"], w["d_model"], w["vocab"], w["n_pos"], m, K, fit_iters,
+                                      1 if keep_prompt_keys else 0)
+        self.B, self.capacity = B, capacity
+        h = ctypes.c_void_p()
+        st = self._lib.lookat_gpt2_create(ctypes.byref(self.cfg), device, ctypes.c_void_p(stream.cuda_stream), B, capacity, ctypes.byref(h))
+        if st != 0:
+            raise LookatError(st, "lookat_gpt2_create rejected the configuration or ran out of memory")
+        self._h = h
+        up = lambda a: torch.from_numpy(a).to(self.device)
+        self._keep = {k: up(w[k]) for k in ("wte", "wpe", "lnf_g", "lnf_b")}
+        self._layers = [{k: up(lw[k]) for k in LAYER_FIELDS} for lw in w["layers"]]
+        arr = (lookat_gpt2_layer * w["n_layer"])()
+        for l, lw in enumerate(self._layers):
+            for k in LAYER_FIELDS:
+                setattr(arr[l], k, lw[k].data_ptr())
+        self._check(self._lib.lookat_gpt2_set_weights(self._h, self._keep["wte"].data_ptr(), self._keep["wpe"].data_ptr(),
+                                                      self._keep["lnf_g"].data_ptr(), self._keep["lnf_b"].data_ptr(), arr))
+
+    def _check(self, st):
+        if st != 0:
+            raise LookatError(st, self._lib.lookat_gpt2_last_error(self._h).decode())
+
+    def close(self):
+        if self._h is not None:
+            self._lib.lookat_gpt2_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def lookat_gpt2_prefill(self, ids, seed=0, want_hidden=False):
+        B, T = ids.shape
+        hidden = torch.empty((B, T, self.cfg.d_model), dtype=torch.float32, device=self.device) if want_hidden else None
+        self._check(self._lib.lookat_gpt2_prefill(self._h, _dev(ids, torch.int32, "ids", (self.B, T)), T, seed,
+                                                  None if hidden is None else hidden.data_ptr()))
+        return hidden
+
+    def lookat_gpt2_decode(self, ids, want_hidden=False, want_logits=False, want_next=False, logits=None, next_ids=None):
+        hidden = torch.empty((self.B, self.cfg.d_model), dtype=torch.float32, device=self.device) if want_hidden else None
+        if want_logits and logits is None:
+            logits = torch.empty((self.B, self.cfg.vocab), dtype=torch.float32, device=self.device)
+        if want_next and next_ids is None:
+            next_ids = torch.empty((self.B,), dtype=torch.int32, device=self.device)
+        self._check(self._lib.lookat_gpt2_decode(self._h, _dev(ids, torch.int32, "ids", (self.B,)),
+                                                 None if hidden is None else hidden.data_ptr(),
+                                                 None if logits is None else logits.data_ptr(),
+                                                 None if next_ids is None else next_ids.data_ptr()))
+        return hidden, logits, next_ids
+
+    def lookat_gpt2_layer_state(self, layer, T=None):
+        """(codebooks, codes, values, prompt_keys) of a layer as torch views of the model's own device memory."""
+        ptrs = [ctypes.c_void_p() for _ in range(4)]
+        self._check(self._lib.lookat_gpt2_layer_state(self._h, layer, *[ctypes.byref(p) for p in ptrs]))
+        c = self.cfg
+
+        def view(ptr, shape, dtype):
+            if not ptr.value:
+                return None
+            self.stream.synchronize()
+            typestr = {torch.float32: "<f4", torch.float16: "<f2", torch.uint8: "|u1"}[dtype]
+            return torch.as_tensor(_RawDeviceArray(ptr.value, shape, typestr), device=self.device).clone()
+        H, cap = c.n_head, self.capacity
+        return (view(ptrs[0], (H, c.m, c.K, 64 // c.m), torch.float32), view(ptrs[1], (self.B, H, cap, c.m), torch.uint8),
+                view(ptrs[2], (self.B, H, cap, 64), torch.float16),
+                view(ptrs[3], (self.B, H, T, 64), torch.float16) if T else None)
+
+    def lookat_gpt2_position(self) -> int:
+        return int(self._lib.lookat_gpt2_position(self._h))
+
+    def lookat_gpt2_kernel_launches(self) -> int:
+        return int(self._lib.lookat_gpt2_kernel_launches(self._h))
+
+
+class _RawDeviceArray:
+    """A device array of the library seen through the CUDA array interface (no copy, no ownership)."""
+
+    def __init__(self, ptr: int, shape, typestr: str):
+        self.__cuda_array_interface__ = {"shape": tuple(int(x) for x in shape), "typestr": typestr, "data": (int(ptr), False),
+                                         "version": 2, "strides": None}
 
 
 # ---- byte accounting of the method (Section 3.4 "Compression Ratio", Section 3.1) ----

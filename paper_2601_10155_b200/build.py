@@ -16,7 +16,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG, "liblookat.so")
-SOURCES = ["api.cu", "attend.cu", "attend_multi.cu", "attend_static.cu", "attend_pqv.cu", "prefill.cu", "prefill_umma.cu", "lut.cu", "encode.cu", "encode_mma.cu", "fit.cu", "probe.cu"]
+SOURCES = ["api.cu", "attend.cu", "attend_multi.cu", "attend_static.cu", "attend_pqv.cu", "prefill.cu", "prefill_umma.cu", "lut.cu", "encode.cu", "encode_mma.cu", "fit.cu", "probe.cu", "linear_umma.cu", "gpt2_ops.cu", "gpt2.cu"]
 
 
 def _nvcc() -> str:
@@ -28,7 +28,7 @@ def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, "lookat.h")]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, f) for f in os.listdir(INCLUDE)]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

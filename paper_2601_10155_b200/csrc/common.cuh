@@ -165,6 +165,30 @@ lookat_status launch_fit_init(Ctx *ctx, const __half *keys, int B, long long n, 
                               const float *init, float *codebooks);
 lookat_status launch_fit_update(Ctx *ctx, float *codebooks);
 
+// ---- GPT-2 decoder harness around the attention (linear_umma.cu, gpt2_ops.cu, gpt2.cu) ----
+struct LinearArgs {
+    const __half *bias;        // [N] or null
+    const float *residual;     // fp32 [M][N] or null: added to the result (may be `out`)
+    void *out;                 // [M][N] fp16 or fp32 (unused in the q/k/v form)
+    int out_fp16, gelu;
+    long long M;
+    int N, K;
+    // q/k/v form: N = 3 * d_model; row = b * T + t; third `sel`, head h, dim d of a row goes to
+    // dst[sel][((b * n_head + h) * cap[sel] + off[sel] + t) * 64 + d]
+    int qkv, T, n_head;
+    __half *dst[3];
+    long long cap[3], off[3];
+    int *timeout_flag;
+};
+// out = act(x w_t^T + bias) [+ residual]; x [M][K] fp16 (fp32 accepted for M <= 32), w_t [N][K] fp16
+lookat_status launch_linear(Ctx *ctx, const void *x, int x_fp32, const __half *w_t, LinearArgs p);
+lookat_status launch_embed(Ctx *ctx, const int32_t *ids, const __half *wte, const __half *wpe, float *x, long long rows, int T,
+                           int pos0, int d, int vocab);
+lookat_status launch_layernorm(Ctx *ctx, const float *x, const __half *g, const __half *b, __half *y, long long rows, int d);
+lookat_status launch_argmax(Ctx *ctx, const float *logits, int32_t *out, int rows, int n);
+lookat_status launch_causal_attention(Ctx *ctx, const __half *q, const __half *k, const __half *v, __half *out, int B, int H, int T,
+                                      long long v_cap);
+
 // ---- small device helpers ----
 __device__ __forceinline__ float ex2_approx(float x)
 {
