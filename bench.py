@@ -548,6 +548,62 @@ def time_c2_replay(device_index: int, layers: int = 12, steps: int = 64):
             "setup_fit_ms_all_layers": fit_ms}
 
 
+def time_gpt2_decoder(device_index: int, steps: int = 64, profile_steps: int = 8):
+    """BASELINE config 2 end to end: the 12-layer GPT-2-small decoder (d_model 768, 12 heads, MLP 3072, vocab 50257,
+    random-init fp16 weights, uniform-random prompt ids), batch 32, a prompt of 1024 tokens processed with exact
+    attention, codebooks (m = 4, K = 256, 25 Lloyd iterations) fitted per layer and head on the prompt's keys, then 64
+    tokens generated greedily with the new key encoded on append and Algorithm 1 in every layer.  Every kernel is this
+    library's own.  A few more steps are then decoded with per-category events to show where a step's time goes."""
+    import torch
+
+    from paper_2601_10155_b200.binding import LookatGpt2
+    B, T0, vocab = 32, 1024, 50257
+    cap = T0 + steps + profile_steps
+    wd = synth.gpt2_weights(1002, n_pos=cap)
+    ids = torch.from_numpy(synth.token_ids(1002, B, T0 + 1, vocab)).cuda()
+    model = LookatGpt2(wd, B, cap, m=4, K=256, fit_iters=25, device=device_index)
+    prompt = ids[:, :T0].contiguous()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    model.lookat_gpt2_prefill(prompt, seed=1002)                 # first pass: scratch grows, clocks come up
+    torch.cuda.synchronize()
+    launches0 = model.lookat_gpt2_kernel_launches()
+    ev[0].record()
+    model.lookat_gpt2_prefill(prompt, seed=1002)
+    ev[1].record()
+    torch.cuda.synchronize()
+    prefill_launches = model.lookat_gpt2_kernel_launches() - launches0
+    nxt = [torch.empty((B,), dtype=torch.int32, device="cuda") for _ in range(2)]
+    cur = ids[:, T0].contiguous()
+    launches0 = model.lookat_gpt2_kernel_launches()
+    ev[2].record()
+    for t in range(steps):
+        model.lookat_gpt2_decode(cur, want_next=True, next_ids=nxt[t & 1])
+        cur = nxt[t & 1]
+    ev[3].record()
+    torch.cuda.synchronize()
+    step_launches = (model.lookat_gpt2_kernel_launches() - launches0) // steps
+    model.lookat_gpt2_set_profile(True)
+    for t in range(profile_steps):
+        model.lookat_gpt2_decode(cur, want_next=True, next_ids=nxt[t & 1])
+        cur = nxt[t & 1]
+    torch.cuda.synchronize()
+    n_prof, cats = model.lookat_gpt2_profile()
+    model.lookat_gpt2_set_profile(False)
+    total = sum(cats.values()) or 1.0
+    prefill_ms, decode_ms = ev[0].elapsed_time(ev[1]), ev[2].elapsed_time(ev[3])
+    params = sum(int(np.prod(a.shape)) for lw in wd["layers"] for a in lw.values()) + int(np.prod(wd["wte"].shape))
+    return {"model": "GPT-2 small shape, random-init fp16", "batch": B, "prompt_tokens": T0, "generated_tokens": steps,
+            "m": 4, "K": 256, "fit_iters": 25,
+            "prefill_ms": prefill_ms, "prefill_tokens_per_s": B * T0 / (prefill_ms * 1e-3), "prefill_launches": int(prefill_launches),
+            "prefill_includes": "12 x (products, exact causal attention, k-means on 32,768 keys per head, encoding)",
+            "ms_per_generated_token": decode_ms / steps, "generated_tokens_per_s": B * steps / (decode_ms * 1e-3),
+            "launches_per_token": int(step_launches),
+            "weight_bytes_per_token": int(params * 2),
+            "weights_gbs": params * 2 / (decode_ms / steps * 1e-3) / 1e9,
+            "share_of_step": {k: v / total for k, v in cats.items()},
+            "share_measured_over_steps": int(n_prof), "sampling": "greedy (argmax on the device), ids fed back without a host copy"}
+
+
 def run_lookat(args, w):
     import torch
     import torch.distributed as dist
@@ -744,6 +800,11 @@ def run_lookat(args, w):
                 line["c2_replay"] = time_c2_replay(local_rank)
             except Exception as exc:
                 line["c2_replay"] = {"error": str(exc)[:200]}
+            torch.cuda.empty_cache()
+            try:
+                line["gpt2_decoder"] = time_gpt2_decoder(local_rank)
+            except Exception as exc:
+                line["gpt2_decoder"] = {"error": str(exc)[:200]}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
@@ -765,6 +826,7 @@ def main():
                     help="skip the extra leg that times decode attention with product-quantised values")
     ap.add_argument("--no-small", dest="small", action="store_false",
                     help="skip the GPT-2 shaped decode steps and the 12-layer x 64-step replay")
+    ap.add_argument("--only-gpt2", action="store_true", help="time only the GPT-2 decoder harness (prints its object alone)")
     ap.add_argument("--only-prefill", action="store_true",
                     help="time only the causal multi-query kernel (prints its object alone)")
     ap.add_argument("--prefill-batch", type=int, default=0, help="smaller prefill case: batch rows")
@@ -777,6 +839,9 @@ def main():
     w = synth.WORKLOADS[args.workload]
     if args.batch > 0:
         w = synth.Workload(**{**w.__dict__, "B": args.batch, "name": f"{w.name}_b{args.batch}"})
+    if args.only_gpt2:
+        print(json.dumps(time_gpt2_decoder(int(os.environ.get("LOCAL_RANK", "0")))), flush=True)
+        return
     if args.only_prefill:
         print(json.dumps(time_prefill(int(os.environ.get("LOCAL_RANK", "0")), steps=max(1, min(args.steps, 5)),
                                       batch=args.prefill_batch, heads=args.prefill_heads, form=args.prefill_form)), flush=True)

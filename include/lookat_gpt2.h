@@ -71,6 +71,23 @@ lookat_status lookat_gpt2_decode(lookat_gpt2 *model, const int32_t *ids, float *
 lookat_status lookat_gpt2_layer_state(lookat_gpt2 *model, int32_t layer, const float **codebooks, const uint8_t **codes,
                                       const void **values, const void **prompt_keys);
 
+/* Where a decode step's device time goes (measurement aid): with profiling on, lookat_gpt2_decode records a CUDA event
+ * after the launches of each category; lookat_gpt2_profile synchronises on them, fills ms[LOOKAT_GPT2_CATEGORIES] with the
+ * milliseconds per category summed over the steps decoded since profiling was switched on, and returns that number
+ * of steps.  The events add launch gaps: use the shares, time whole steps without profiling. */
+enum {
+    LOOKAT_GPT2_CAT_EMBED = 0,
+    LOOKAT_GPT2_CAT_NORM = 1,       /* both LayerNorms of a block */
+    LOOKAT_GPT2_CAT_QKV = 2,        /* fused q/k/v projection */
+    LOOKAT_GPT2_CAT_ATTENTION = 3,  /* append-encode + Algorithm 1 (lookat_decode_step) */
+    LOOKAT_GPT2_CAT_OUT_PROJ = 4,
+    LOOKAT_GPT2_CAT_MLP = 5,        /* both products of the MLP, GELU fused */
+    LOOKAT_GPT2_CAT_LM_HEAD = 6,    /* final LayerNorm, tied output projection, argmax */
+    LOOKAT_GPT2_CATEGORIES = 7
+};
+void lookat_gpt2_set_profile(lookat_gpt2 *model, int32_t enabled);
+int32_t lookat_gpt2_profile(lookat_gpt2 *model, double *ms);
+
 int32_t lookat_gpt2_position(const lookat_gpt2 *model);          /* tokens in the cache */
 uint64_t lookat_gpt2_kernel_launches(const lookat_gpt2 *model);   /* kernels launched since creation */
 

@@ -24,6 +24,7 @@ EXPORTS = [
     # include/lookat_gpt2.h
     "lookat_gpt2_create", "lookat_gpt2_destroy", "lookat_gpt2_last_error", "lookat_gpt2_set_weights", "lookat_gpt2_prefill",
     "lookat_gpt2_decode", "lookat_gpt2_layer_state", "lookat_gpt2_position", "lookat_gpt2_kernel_launches",
+    "lookat_gpt2_set_profile", "lookat_gpt2_profile",
     "lookat_linear", "lookat_linear_qkv", "lookat_layernorm", "lookat_embed", "lookat_causal_attention", "lookat_argmax",
 ]
 
@@ -126,6 +127,10 @@ def load_library() -> ctypes.CDLL:
     lib.lookat_gpt2_position.restype = i32
     lib.lookat_gpt2_kernel_launches.argtypes = [vp]
     lib.lookat_gpt2_kernel_launches.restype = ctypes.c_uint64
+    lib.lookat_gpt2_set_profile.argtypes = [vp, i32]
+    lib.lookat_gpt2_set_profile.restype = None
+    lib.lookat_gpt2_profile.argtypes = [vp, ctypes.POINTER(ctypes.c_double)]
+    lib.lookat_gpt2_profile.restype = i32
     lib.lookat_linear.argtypes = [vp, vp, i32, vp, vp, i64, i32, i32, i32, vp, vp, i32]
     lib.lookat_linear.restype = i32
     lib.lookat_linear_qkv.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, i64, i64, vp, i64, i64, vp, i64, i64]
@@ -523,6 +528,16 @@ class LookatGpt2:
         return (view(ptrs[0], (H, c.m, c.K, 64 // c.m), torch.float32), view(ptrs[1], (self.B, H, cap, c.m), torch.uint8),
                 view(ptrs[2], (self.B, H, cap, 64), torch.float16),
                 view(ptrs[3], (self.B, H, T, 64), torch.float16) if T else None)
+
+    def lookat_gpt2_set_profile(self, enabled: bool):
+        self._lib.lookat_gpt2_set_profile(self._h, 1 if enabled else 0)
+
+    def lookat_gpt2_profile(self):
+        """(steps, {category: milliseconds}) of the decode steps made since profiling was switched on."""
+        names = ("embed", "layernorm", "qkv", "attention", "out_proj", "mlp", "lm_head")
+        ms = (ctypes.c_double * len(names))()
+        steps = int(self._lib.lookat_gpt2_profile(self._h, ms))
+        return steps, {n: ms[i] for i, n in enumerate(names)}
 
     def lookat_gpt2_position(self) -> int:
         return int(self._lib.lookat_gpt2_position(self._h))

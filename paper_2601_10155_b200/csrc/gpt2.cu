@@ -37,6 +37,10 @@ struct Gpt2 {
     std::vector<__half *> values;           // [B][H][capacity][64]
     std::vector<__half *> prompt_keys;      // [B][H][T][64], kept on request (tests)
     int pos;                                // tokens in the cache
+    // optional per-category device timing of a decode step (events between the launches of one step)
+    bool profile;
+    std::vector<cudaEvent_t> prof_ev;       // boundaries, in launch order
+    std::vector<int> prof_cat;              // category of the work between boundary i and i + 1
 };
 
 namespace {
@@ -72,6 +76,20 @@ bool dev_alloc(T **p, size_t n)
         }                                                                                        \
     } while (0)
 
+// when profiling: closes the category of the launches made since the previous mark
+void mark(Gpt2 *g, int category)
+{
+    if (!g->profile) return;
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) {
+        cudaGetLastError();
+        return;
+    }
+    cudaEventRecord(e, g->stream);
+    g->prof_ev.push_back(e);
+    g->prof_cat.push_back(category);
+}
+
 LinearArgs plain(const __half *bias, long long M, int N, int K, int gelu, const float *residual, void *out, int out_fp16)
 {
     LinearArgs p;
@@ -93,8 +111,10 @@ lookat_status mlp(Gpt2 *g, const lookat_gpt2_layer &w, long long rows)
     Ctx *ctx = ctx_of(g);
     const int d = g->cfg.d_model;
     G_TRY(launch_layernorm(ctx, g->x, (const __half *)w.ln2_g, (const __half *)w.ln2_b, g->a16, rows, d));
+    mark(g, LOOKAT_GPT2_CAT_NORM);
     G_TRY(launch_linear(ctx, g->a16, 0, (const __half *)w.w_fc, plain((const __half *)w.b_fc, rows, 4 * d, d, 1, nullptr, g->fc16, 1)));
     G_TRY(launch_linear(ctx, g->fc16, 0, (const __half *)w.w_pr, plain((const __half *)w.b_pr, rows, d, 4 * d, 0, g->x, g->x, 0)));
+    mark(g, LOOKAT_GPT2_CAT_MLP);
     return LOOKAT_OK;
 }
 
@@ -123,6 +143,7 @@ lookat_status lookat_gpt2_create(const lookat_gpt2_config *cfg, int device, void
     g->err[0] = 0;
     g->have_weights = false;
     g->pos = 0;
+    g->profile = false;
     lookat_config ac = {c.n_head, c.n_head, 64, 64, c.m, c.K, 0.f};
     lookat_status st = lookat_create(&ac, device, cuda_stream, &g->attn);
     if (st != LOOKAT_OK) {
@@ -175,6 +196,7 @@ void lookat_gpt2_destroy(lookat_gpt2 *handle)
     }
     cudaGetLastError();
     if (prev >= 0) cudaSetDevice(prev);
+    for (cudaEvent_t e : g->prof_ev) cudaEventDestroy(e);
     lookat_destroy(g->attn);
     delete g;
 }
@@ -274,10 +296,13 @@ lookat_status lookat_gpt2_decode(lookat_gpt2 *handle, const int32_t *ids, float 
     struct Restore { int d; ~Restore() { if (d >= 0) cudaSetDevice(d); } } restore{prev};
     const lookat_gpt2_config &c = g->cfg;
     const int d = c.d_model, H = c.n_head, B = g->B, pos = g->pos;
+    mark(g, -1);                                             // opens the step
     G_TRY(launch_embed(ctx, ids, g->wte, g->wpe, g->x, B, 1, pos, d, c.vocab));
+    mark(g, LOOKAT_GPT2_CAT_EMBED);
     for (int l = 0; l < c.n_layer; ++l) {
         const lookat_gpt2_layer &w = g->layers[l];
         G_TRY(launch_layernorm(ctx, g->x, (const __half *)w.ln1_g, (const __half *)w.ln1_b, g->a16, B, d));
+        mark(g, LOOKAT_GPT2_CAT_NORM);
         LinearArgs p = plain((const __half *)w.b_qkv, B, 3 * d, d, 0, nullptr, nullptr, 1);
         p.qkv = 1;
         p.T = 1;
@@ -286,9 +311,12 @@ lookat_status lookat_gpt2_decode(lookat_gpt2 *handle, const int32_t *ids, float 
         p.dst[1] = g->kd; p.cap[1] = 1; p.off[1] = 0;
         p.dst[2] = g->values[l]; p.cap[2] = g->capacity; p.off[2] = pos;       // the value row goes straight into the cache
         G_TRY(launch_linear(ctx, g->a16, 0, (const __half *)w.w_qkv, p));
+        mark(g, LOOKAT_GPT2_CAT_QKV);
         // append (Section 3.4 "Encoding") and Algorithm 1 over tokens 0..pos, one launch
         G_TRY(lookat_decode_step(g->attn, g->qd, g->kd, g->books[l], g->codes[l], g->values[l], B, g->capacity, pos, 0, g->attn_out));
+        mark(g, LOOKAT_GPT2_CAT_ATTENTION);
         G_TRY(launch_linear(ctx, g->attn_out, 1, (const __half *)w.w_o, plain((const __half *)w.b_o, B, d, d, 0, g->x, g->x, 0)));
+        mark(g, LOOKAT_GPT2_CAT_OUT_PROJ);
         G_TRY(mlp(g, w, B));
     }
     if (hidden_out && cudaMemcpyAsync(hidden_out, g->x, (size_t)B * d * sizeof(float), cudaMemcpyDeviceToDevice, g->stream) != cudaSuccess)
@@ -298,9 +326,38 @@ lookat_status lookat_gpt2_decode(lookat_gpt2 *handle, const int32_t *ids, float 
         G_TRY(launch_layernorm(ctx, g->x, g->lnf_g, g->lnf_b, g->a16, B, d));
         G_TRY(launch_linear(ctx, g->a16, 0, g->wte, plain(nullptr, B, c.vocab, d, 0, nullptr, lg, 0)));     // tied output projection
         if (next_ids) G_TRY(launch_argmax(ctx, lg, next_ids, B, c.vocab));
+        mark(g, LOOKAT_GPT2_CAT_LM_HEAD);
     }
     g->pos = pos + 1;
     return LOOKAT_OK;
+}
+
+void lookat_gpt2_set_profile(lookat_gpt2 *handle, int32_t enabled)
+{
+    if (!handle) return;
+    Gpt2 *g = reinterpret_cast<Gpt2 *>(handle);
+    for (cudaEvent_t e : g->prof_ev) cudaEventDestroy(e);
+    g->prof_ev.clear();
+    g->prof_cat.clear();
+    g->profile = enabled != 0;
+}
+
+int32_t lookat_gpt2_profile(lookat_gpt2 *handle, double *ms)
+{
+    if (!handle || !ms) return 0;
+    Gpt2 *g = reinterpret_cast<Gpt2 *>(handle);
+    for (int i = 0; i < LOOKAT_GPT2_CATEGORIES; ++i) ms[i] = 0.0;
+    int steps = 0;
+    for (size_t i = 1; i < g->prof_ev.size(); ++i) {
+        if (g->prof_cat[i] < 0) {                           // a step's opening mark: nothing to attribute
+            continue;
+        }
+        float t = 0.f;
+        cudaEventSynchronize(g->prof_ev[i]);
+        if (cudaEventElapsedTime(&t, g->prof_ev[i - 1], g->prof_ev[i]) == cudaSuccess) ms[g->prof_cat[i]] += t;
+    }
+    for (int c : g->prof_cat) steps += c < 0 ? 1 : 0;
+    return steps;
 }
 
 lookat_status lookat_gpt2_layer_state(lookat_gpt2 *handle, int32_t layer, const float **codebooks, const uint8_t **codes,

@@ -62,14 +62,16 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const float *__restrict_
 }
 
 // first index of the largest logit of every row
-__global__ void __launch_bounds__(256) argmax_kernel(const float *__restrict__ logits, int32_t *__restrict__ out, int n)
+constexpr int kAmThreads = 1024;
+__global__ void __launch_bounds__(kAmThreads) argmax_kernel(const float *__restrict__ logits, int32_t *__restrict__ out, int n)
 {
-    __shared__ float sv[8];
-    __shared__ int si[8];
+    __shared__ float sv[kAmThreads / 32];
+    __shared__ int si[kAmThreads / 32];
     const float *row = logits + (size_t)blockIdx.x * n;
     float best = -INFINITY;
     int idx = 0x7fffffff;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+#pragma unroll 4
+    for (int i = threadIdx.x; i < n; i += kAmThreads) {
         const float v = row[i];
         if (v > best) { best = v; idx = i; }
     }
@@ -80,10 +82,15 @@ __global__ void __launch_bounds__(256) argmax_kernel(const float *__restrict__ l
     }
     if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = best; si[threadIdx.x >> 5] = idx; }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        for (int w = 1; w < 8; ++w)
-            if (sv[w] > best || (sv[w] == best && si[w] < idx)) { best = sv[w]; idx = si[w]; }
-        out[blockIdx.x] = idx == 0x7fffffff ? 0 : idx;
+    if (threadIdx.x < 32) {
+        best = sv[threadIdx.x];
+        idx = si[threadIdx.x];
+        for (int o = 16; o; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+            if (ov > best || (ov == best && oi < idx)) { best = ov; idx = oi; }
+        }
+        if (threadIdx.x == 0) out[blockIdx.x] = idx == 0x7fffffff ? 0 : idx;
     }
 }
 
@@ -239,7 +246,7 @@ lookat_status launch_layernorm(Ctx *ctx, const float *x, const __half *g, const 
 
 lookat_status launch_argmax(Ctx *ctx, const float *logits, int32_t *out, int rows, int n)
 {
-    argmax_kernel<<<rows, 256, 0, ctx->stream>>>(logits, out, n);
+    argmax_kernel<<<rows, kAmThreads, 0, ctx->stream>>>(logits, out, n);
     return check_launch(ctx, "argmax_kernel");
 }
 

@@ -12,10 +12,11 @@
 // Every mbarrier wait is bounded; a wait that runs out raises the context's time-out flag, the CTA drains, frees its
 // tensor memory and returns.
 //
-// linear_skinny_kernel (M <= 32: one decode step of the whole batch): the product is bound by reading W once.  A CTA
-// owns 32 output columns, a warp 8 of them: it streams its 8 rows of w_t with 16-byte loads straight into
-// mma.sync.m16n8k16 B fragments (the k order inside a 32-wide block is permuted the same way for both operands, so no
-// shuffle is needed), x waits in shared memory, two 16-row tiles cover the batch.
+// linear_skinny_kernel (M <= 32: one decode step of the whole batch): the product is bound by reading W once, and at
+// these sizes by latency.  A CTA owns 16 output columns; each of its 8 warps streams 8 rows of w_t over a quarter of K
+// with 16-byte loads straight into mma.sync.m16n8k16 B fragments (the k order inside a 32-wide block is permuted the
+// same way for both operands, so no shuffle is needed); two 16-row tiles cover the batch; the quarters meet in shared
+// memory.
 #include <cuda.h>           // CUtensorMap and its enums only; the driver entry point is looked up at run time
 
 #include "common.cuh"
@@ -161,8 +162,6 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int tile_n = blockIdx.x, tile_m = blockIdx.y;
     const int num_k = (p.K + kLnBK - 1) / kLnBK;
-    // once a wait has run out anywhere in the launch, the remaining CTAs leave at once (the call reports a time-out)
-    if (__syncthreads_or(tid == 0 && p.timeout_flag && *(volatile int *)p.timeout_flag != 0)) return;
 
     if (tid == 0) {
         for (int s = 0; s < kLnStages; ++s) {
@@ -249,7 +248,11 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-constexpr int kSkThreads = 128, kSkCols = 32, kSkChunk = 512, kSkPitch = kSkChunk + 8;     // halfs per staged x row
+// One decode step's products: M <= 32 rows, bound by reading w_t once, and small enough that latency decides.  A CTA of
+// 8 warps owns 16 output columns: warp (cw, ks) takes columns n0 + 8 cw .. +7 and the ks-th quarter of K, so 4 x as many
+// warps stream the weights as there are 8-column groups; the four partial sums meet in shared memory.  x is read from
+// global memory as it is needed (it is at most 192 KB and stays in L1/L2).
+constexpr int kSkThreads = 256, kSkCols = 16, kSkSplits = 4;
 
 __device__ __forceinline__ void sk_mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
 {
@@ -259,55 +262,61 @@ __device__ __forceinline__ void sk_mma(float (&c)[4], uint32_t a0, uint32_t a1, 
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// 8 consecutive elements of x row `r` from column k as four packed half pairs (zeros for rows >= M)
+template <bool X_FP32>
+__device__ __forceinline__ uint4 sk_x8(const void *x, int r, int M, int K, int k)
+{
+    if (r >= M) return make_uint4(0u, 0u, 0u, 0u);
+    if (X_FP32) {
+        const float4 *src = reinterpret_cast<const float4 *>(static_cast<const float *>(x) + (size_t)r * K + k);
+        const float4 f0 = src[0], f1 = src[1];
+        __half2 h0 = __floats2half2_rn(f0.x, f0.y), h1 = __floats2half2_rn(f0.z, f0.w);
+        __half2 h2 = __floats2half2_rn(f1.x, f1.y), h3 = __floats2half2_rn(f1.z, f1.w);
+        return make_uint4(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1), *reinterpret_cast<uint32_t *>(&h2),
+                          *reinterpret_cast<uint32_t *>(&h3));
+    }
+    return *reinterpret_cast<const uint4 *>(static_cast<const __half *>(x) + (size_t)r * K + k);
+}
+
 template <bool X_FP32>
 __global__ void __launch_bounds__(kSkThreads) linear_skinny_kernel(const void *__restrict__ x, const __half *__restrict__ w_t, LinearArgs p)
 {
-    __shared__ __align__(16) __half xs[32 * kSkPitch];
+    __shared__ float part[kSkSplits][2][2][4][32];              // [k quarter][column warp][row tile][accumulator][lane]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const int n0 = blockIdx.x * kSkCols + warp * 8;             // this warp's 8 output columns
+    const int cw = warp & 1, ks = warp >> 1;
+    const int n0 = blockIdx.x * kSkCols + cw * 8;               // this warp's 8 output columns
     const int M = (int)p.M, K = p.K;
+    // this warp's share of K: whole 32-wide blocks
+    const int blocks = (K + 31) / 32, per = (blocks + kSkSplits - 1) / kSkSplits;
+    const int k_lo = min(K, ks * per * 32), k_hi = min(K, (ks + 1) * per * 32);
     float acc[2][4] = {};
-    // lane (g, t) streams row n0 + g of w_t, 8 halfs at k = kk + 8 t of every 32-wide block (columns beyond N read row N - 1)
+    // lane (g, t) streams row n0 + g of w_t, 8 halfs at k = kk + 8 t of every 32-wide block (columns beyond N read row N - 1).
+    // Inside such a block the MMA's k index is a relabelling of the true one: the lane with t supplies true k = 8 t .. 8 t + 7
+    // -- (8t, 8t+1 | 8t+2, 8t+3) to the first MMA, (8t+4, 8t+5 | 8t+6, 8t+7) to the second -- for both operands alike.
     const __half *wrow = w_t + (size_t)min(n0 + g, p.N - 1) * K;
-    for (int k0 = 0; k0 < K; k0 += kSkChunk) {
-        const int kc = min(kSkChunk, K - k0);                   // a multiple of 8
-        __syncthreads();
-        for (int i = tid; i < 32 * (kSkChunk / 8); i += kSkThreads) {
-            const int r = i / (kSkChunk / 8), c8 = (i - r * (kSkChunk / 8)) * 8;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (r < M && c8 < kc) {
-                if (X_FP32) {
-                    const float4 *src = reinterpret_cast<const float4 *>(static_cast<const float *>(x) + (size_t)r * K + k0 + c8);
-                    const float4 f0 = src[0], f1 = src[1];
-                    __half2 h0 = __floats2half2_rn(f0.x, f0.y), h1 = __floats2half2_rn(f0.z, f0.w);
-                    __half2 h2 = __floats2half2_rn(f1.x, f1.y), h3 = __floats2half2_rn(f1.z, f1.w);
-                    v.x = *reinterpret_cast<uint32_t *>(&h0); v.y = *reinterpret_cast<uint32_t *>(&h1);
-                    v.z = *reinterpret_cast<uint32_t *>(&h2); v.w = *reinterpret_cast<uint32_t *>(&h3);
-                } else {
-                    v = *reinterpret_cast<const uint4 *>(static_cast<const __half *>(x) + (size_t)r * K + k0 + c8);
-                }
-            }
-            *reinterpret_cast<uint4 *>(xs + r * kSkPitch + c8) = v;
-        }
-        __syncthreads();
-        // inside a 32-wide block the MMA's k index is a relabelling of the true one: the lane with t supplies true
-        // k = 8 t .. 8 t + 7 -- (8t, 8t+1 | 8t+2, 8t+3) to the first MMA, (8t+4, 8t+5 | 8t+6, 8t+7) to the second -- for
-        // both operands alike
 #pragma unroll 4
-        for (int kk = 0; kk < kc; kk += 32) {
-            uint4 wv = make_uint4(0u, 0u, 0u, 0u);
-            if (kk + 8 * t < kc) wv = __ldg(reinterpret_cast<const uint4 *>(wrow + k0 + kk + 8 * t));
+    for (int kk = k_lo; kk < k_hi; kk += 32) {
+        const int k = kk + 8 * t;
+        uint4 wv = make_uint4(0u, 0u, 0u, 0u), xa[2][2];
+        const bool in = k < K;                                  // K is a multiple of 8
+        if (in) wv = __ldg(reinterpret_cast<const uint4 *>(wrow + k));
 #pragma unroll
-            for (int mt = 0; mt < 2; ++mt) {
-                const uint2 lo = *reinterpret_cast<const uint2 *>(xs + (mt * 16 + g) * kSkPitch + kk + 8 * t);
-                const uint2 lo8 = *reinterpret_cast<const uint2 *>(xs + (mt * 16 + g + 8) * kSkPitch + kk + 8 * t);
-                const uint2 hi = *reinterpret_cast<const uint2 *>(xs + (mt * 16 + g) * kSkPitch + kk + 8 * t + 4);
-                const uint2 hi8 = *reinterpret_cast<const uint2 *>(xs + (mt * 16 + g + 8) * kSkPitch + kk + 8 * t + 4);
-                sk_mma(acc[mt], lo.x, lo8.x, lo.y, lo8.y, wv.x, wv.y);
-                sk_mma(acc[mt], hi.x, hi8.x, hi.y, hi8.y, wv.z, wv.w);
-            }
+        for (int mt = 0; mt < 2; ++mt) {
+            xa[mt][0] = in ? sk_x8<X_FP32>(x, mt * 16 + g, M, K, k) : make_uint4(0u, 0u, 0u, 0u);
+            xa[mt][1] = in ? sk_x8<X_FP32>(x, mt * 16 + g + 8, M, K, k) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            sk_mma(acc[mt], xa[mt][0].x, xa[mt][1].x, xa[mt][0].y, xa[mt][1].y, wv.x, wv.y);
+            sk_mma(acc[mt], xa[mt][0].z, xa[mt][1].z, xa[mt][0].w, xa[mt][1].w, wv.z, wv.w);
         }
     }
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) part[ks][cw][mt][i][lane] = acc[mt][i];
+    __syncthreads();
+    if (ks != 0) return;
     // accumulator (mt, i): row mt * 16 + g + 8 * (i >> 1), column n0 + 2 t + (i & 1)
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
@@ -315,7 +324,8 @@ __global__ void __launch_bounds__(kSkThreads) linear_skinny_kernel(const void *_
         for (int i = 0; i < 4; ++i) {
             const int row = mt * 16 + g + 8 * (i >> 1), col = n0 + 2 * t + (i & 1);
             if (row >= M || col >= p.N) continue;
-            float v = acc[mt][i] + (p.bias ? __half2float(p.bias[col]) : 0.f);
+            float v = part[0][cw][mt][i][lane] + part[1][cw][mt][i][lane] + part[2][cw][mt][i][lane] + part[3][cw][mt][i][lane];
+            v += p.bias ? __half2float(p.bias[col]) : 0.f;
             if (p.gelu) v = gelu_tanh(v);
             if (p.qkv) {
                 const int d_model = p.N / 3;
