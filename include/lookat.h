@@ -60,8 +60,16 @@ typedef struct {
 lookat_status lookat_create(const lookat_config *cfg, int device, void *cuda_stream, lookat_ctx **out);
 void lookat_destroy(lookat_ctx *ctx);
 
-/* Host string describing the last error this context returned ("" if none). */
+/* Host string describing the last error this context returned ("" if none).  In the debug build of the library
+ * (compiled with -DLOOKAT_DEBUG, liblookat_debug.so) the attend kernels check every code they read from a cache:
+ * a code >= K is clamped to K - 1 before it is used as an index and the finding is recorded in a status word of the
+ * context; after the caller has synchronised the stream, this call reports it once.  The normal build does not
+ * check: a code >= K there is the caller's error (the streaming kernels then read garbage inside their tables, the
+ * any-shape kernel reads past the table). */
 const char *lookat_last_error(const lookat_ctx *ctx);
+
+/* 1 in the debug build of the library, 0 otherwise. */
+int32_t lookat_is_debug_build(void);
 
 /*
  * Section 3.4, Prototype Learning: for every KV head h and subspace j, a

@@ -15,9 +15,10 @@ import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "liblookat.so")
+LIB_DEBUG_PATH = os.path.join(_PKG, "liblookat_debug.so")      # the build whose attend kernels check the codes they read
 
 EXPORTS = [
-    "lookat_create", "lookat_destroy", "lookat_last_error", "lookat_fit_codebooks",
+    "lookat_create", "lookat_destroy", "lookat_last_error", "lookat_is_debug_build", "lookat_fit_codebooks",
     "lookat_encode_keys", "lookat_build_lut", "lookat_attend", "lookat_attend_static", "lookat_attend_pqv",
     "lookat_attend_prefill", "lookat_decode_step", "lookat_decode_step_host",
     "lookat_kernel_launches", "lookat_probe_read_bandwidth", "lookat_selftest_timeout", "lookat_set_prefill_form", "lookat_set_timing", "lookat_attend_kernel_ms", "lookat_attend_kernel_stats",
@@ -56,19 +57,19 @@ class lookat_gpt2_layer(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in LAYER_FIELDS]
 
 
-_lib = None
+_libs = {}
 
 
-def load_library() -> ctypes.CDLL:
-    """Loads liblookat.so (built by paper_2601_10155_b200.build); raises if absent."""
-    global _lib
-    if _lib is not None:
-        return _lib
-    if not os.path.exists(LIB_PATH):
+def load_library(debug: bool = False) -> ctypes.CDLL:
+    """Loads liblookat.so (built by paper_2601_10155_b200.build), or its debug build; raises if absent."""
+    if debug in _libs:
+        return _libs[debug]
+    path = LIB_DEBUG_PATH if debug else LIB_PATH
+    if not os.path.exists(path):
         raise FileNotFoundError(
-            f"{LIB_PATH} is missing: run `python -m paper_2601_10155_b200.build` (needs nvcc). "
+            f"{path} is missing: run `python -m paper_2601_10155_b200.build{' --debug' if debug else ''}` (needs nvcc). "
             "There is no fallback path.")
-    lib = ctypes.CDLL(LIB_PATH)
+    lib = ctypes.CDLL(path)
     vp, i32, i64, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint64
     lib.lookat_create.argtypes = [ctypes.POINTER(lookat_config), ctypes.c_int, vp, ctypes.POINTER(vp)]
     lib.lookat_create.restype = ctypes.c_int
@@ -143,7 +144,9 @@ def load_library() -> ctypes.CDLL:
     lib.lookat_causal_attention.restype = i32
     lib.lookat_argmax.argtypes = [vp, vp, i32, i32, vp]
     lib.lookat_argmax.restype = i32
-    _lib = lib
+    lib.lookat_is_debug_build.argtypes = []
+    lib.lookat_is_debug_build.restype = i32
+    _libs[debug] = lib
     return lib
 
 
@@ -175,8 +178,8 @@ class Lookat:
     Method names and argument order are those of the C entry points.
     """
 
-    def __init__(self, n_q_heads, n_kv_heads, d_k, d_v, m, K=256, scale=0.0, device=0, stream=None):
-        self._lib = load_library()
+    def __init__(self, n_q_heads, n_kv_heads, d_k, d_v, m, K=256, scale=0.0, device=0, stream=None, debug=False):
+        self._lib = load_library(debug)
         self._h = None
         if not torch.cuda.is_available():
             raise RuntimeError("no CUDA device: the LOOKAT library runs on the GPU only")
@@ -205,6 +208,9 @@ class Lookat:
     def _check(self, st):
         if st != 0:
             raise LookatError(st, self._lib.lookat_last_error(self._h).decode())
+
+    def lookat_last_error(self) -> str:
+        return self._lib.lookat_last_error(self._h).decode()
 
     def close(self):
         if self._h is not None:

@@ -148,6 +148,7 @@ lookat_status attend_impl(Ctx *ctx, const float *lut, const void *q, const float
     a.K = c.K;
     a.L_max = L_max;
     a.scale_log2 = ctx->scale * 1.4426950408889634f;
+    a.status = ctx->status_word;
     size_t po = 0, pml = 0;
     LOOKAT_TRY(plan_attend(ctx, a, n_splits, &po, &pml));
     if (new_keys) {
@@ -263,6 +264,12 @@ lookat_status lookat_create(const lookat_config *cfg, int device, void *cuda_str
         cudaGetLastError();
         ctx->timeout_flag = nullptr;                       // the tcgen05 prefill kernel is then not used
     }
+    if (cudaHostAlloc((void **)&ctx->status_word, sizeof(int), cudaHostAllocMapped) == cudaSuccess) {
+        *ctx->status_word = 0;
+    } else {
+        cudaGetLastError();
+        ctx->status_word = nullptr;                        // the debug build's checks then clamp without a record
+    }
     *out = reinterpret_cast<lookat_ctx *>(ctx);
     return LOOKAT_OK;
 }
@@ -278,6 +285,7 @@ void lookat_destroy(lookat_ctx *handle)
     for (void *p : bufs)
         if (p) cudaFree(p);
     if (ctx->timeout_flag) cudaFreeHost(ctx->timeout_flag);
+    if (ctx->status_word) cudaFreeHost(ctx->status_word);
     for (int i = 0; i < ctx->ev_cap; ++i) {
         if (ctx->ev0[i]) cudaEventDestroy(ctx->ev0[i]);
         if (ctx->ev1[i]) cudaEventDestroy(ctx->ev1[i]);
@@ -291,7 +299,24 @@ void lookat_destroy(lookat_ctx *handle)
 
 const char *lookat_last_error(const lookat_ctx *handle)
 {
-    return handle ? reinterpret_cast<const Ctx *>(handle)->err : "context is NULL";
+    if (!handle) return "context is NULL";
+    Ctx *ctx = const_cast<Ctx *>(reinterpret_cast<const Ctx *>(handle));
+    // asynchronous findings of the debug build's device-side checks (meaningful once the caller has synchronised)
+    if (ctx->status_word && (*(volatile int *)ctx->status_word & kStatusBadCode)) {
+        *(volatile int *)ctx->status_word = 0;
+        snprintf(ctx->err, sizeof(ctx->err),
+                 "debug check: a code >= K was found in a code cache and clamped to K - 1; results computed from it are not valid");
+    }
+    return ctx->err;
+}
+
+int32_t lookat_is_debug_build(void)
+{
+#ifdef LOOKAT_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
 }
 
 uint64_t lookat_kernel_launches(const lookat_ctx *handle)

@@ -211,8 +211,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         if (FULL || head_ok) {
 #pragma unroll
             for (int j = 0; j < M_SUB; ++j) {
-                s0 += my_table[j * kTableStride + code_at<M_SUB>(cp, 0, j)];
-                s1 += my_table[j * kTableStride + code_at<M_SUB>(cp, 1, j)];
+                s0 += my_table[j * kTableStride + LOOKAT_CHECKED_CODE(code_at<M_SUB>(cp, 0, j), a.K, a.status)];
+                s1 += my_table[j * kTableStride + LOOKAT_CHECKED_CODE(code_at<M_SUB>(cp, 1, j), a.K, a.status)];
             }
         }
         float x0 = s0 * a.scale_log2, x1 = s1 * a.scale_log2;
@@ -505,7 +505,7 @@ __global__ void __launch_bounds__(kGenThreads) attend_generic_kernel(AttendArgs 
         for (int t = tid; t < cnt; t += kGenThreads) {
             const uint8_t *cd = codes + (blk + t) * a.m;
             float s = 0.f;
-            for (int j = 0; j < a.m; ++j) s += __ldg(lut + j * a.K + cd[j]);
+            for (int j = 0; j < a.m; ++j) s += __ldg(lut + j * a.K + LOOKAT_CHECKED_CODE((int)cd[j], a.K, a.status));
             if (scores_row) scores_row[blk + t] = s;
             const float x = s * a.scale_log2;
             xs[t] = x;

@@ -700,8 +700,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_multi_kernel(const __grid_
                     if (fast || head_ok) {
 #pragma unroll
                         for (int j = 0; j < M_SUB; ++j) {
-                            s0 += my_table[j * kTableStride + code_at<M_SUB>(cp, 0, j)];
-                            s1 += my_table[j * kTableStride + code_at<M_SUB>(cp, 1, j)];
+                            s0 += my_table[j * kTableStride + LOOKAT_CHECKED_CODE(code_at<M_SUB>(cp, 0, j), a.K, a.status)];
+                            s1 += my_table[j * kTableStride + LOOKAT_CHECKED_CODE(code_at<M_SUB>(cp, 1, j), a.K, a.status)];
                         }
                     }
                     float x0 = s0 * a.scale_log2, x1 = s1 * a.scale_log2;

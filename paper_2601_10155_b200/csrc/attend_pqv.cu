@@ -69,6 +69,7 @@ struct PqvArgs {
     int B, H_q, H_kv, g, K, K_v, d_vsub, d_v;
     int vec4;                // the value codebooks can be read four dims at a time
     float scale_log2;
+    int *status;             // the context's status word (debug build)
 };
 
 // the m code bytes of one token as 32-bit words (m = 2: the low half of one word)
@@ -77,6 +78,22 @@ struct CodeWords {
     static constexpr int NW = M >= 4 ? M / 4 : 1;
     uint32_t w[NW];
 };
+
+// debug build: every code byte against its limit (clamped and recorded); nothing in the normal build
+template <int M>
+__device__ __forceinline__ void check_code_words(CodeWords<M> &c, int K, int *status)
+{
+#ifdef LOOKAT_DEBUG
+    constexpr int BYTES = M >= 4 ? M : (M == 2 ? 4 : 4);        // m = 2 keeps its two bytes twice in one word
+#pragma unroll
+    for (int byte = 0; byte < BYTES; ++byte) {
+        const unsigned sh = (unsigned)(byte & 3) * 8u;
+        const int code = (int)((c.w[byte >> 2] >> sh) & 0xffu);
+        const int ok = checked_code(code, K, status);
+        c.w[byte >> 2] = (c.w[byte >> 2] & ~(0xffu << sh)) | ((uint32_t)ok << sh);
+    }
+#endif
+}
 
 template <int M>
 __device__ __forceinline__ CodeWords<M> load_code_words(const uint8_t *row)
@@ -272,8 +289,10 @@ __global__ void __launch_bounds__(kPqThreads, pqv_min_ctas<M_K, M_V, HG>()) atte
         auto load_k = [&](int n_tok) {
 #pragma unroll
             for (int i = 0; i < kPqLoads; ++i) {
-                if (i * 32 + lane < n_tok) kc[i] = load_code_words<M_K>(kptr + (size_t)i * 32 * M_K);
-                else {
+                if (i * 32 + lane < n_tok) {
+                    kc[i] = load_code_words<M_K>(kptr + (size_t)i * 32 * M_K);
+                    check_code_words<M_K>(kc[i], a.K, a.status);
+                } else {
 #pragma unroll
                     for (int w = 0; w < CodeWords<M_K>::NW; ++w) kc[i].w[w] = 0u;
                 }
@@ -283,8 +302,10 @@ __global__ void __launch_bounds__(kPqThreads, pqv_min_ctas<M_K, M_V, HG>()) atte
         auto load_v = [&](int n_tok) {
 #pragma unroll
             for (int i = 0; i < kPqLoads; ++i) {
-                if (i * 32 + lane < n_tok) vc[i] = load_code_words<M_V>(vptr + (size_t)i * 32 * M_V);
-                else {
+                if (i * 32 + lane < n_tok) {
+                    vc[i] = load_code_words<M_V>(vptr + (size_t)i * 32 * M_V);
+                    check_code_words<M_V>(vc[i], a.K_v, a.status);
+                } else {
 #pragma unroll
                     for (int w = 0; w < CodeWords<M_V>::NW; ++w) vc[i].w[w] = 0u;
                 }
@@ -722,6 +743,7 @@ lookat_status attend_pqv_impl(Ctx *ctx, const float *lut, const uint8_t *codes, 
     a.d_v = c.d_v;
     a.d_vsub = c.d_v / m_v;
     a.scale_log2 = ctx->scale * 1.4426950408889634f;
+    a.status = ctx->status_word;
     a.vec4 = (a.d_vsub % 4 == 0 && ((uintptr_t)v_books & 15u) == 0 && a.d_v / 4 <= kPqThreads) ? 1 : 0;
     switch (c.m) {
         case 2: return launch_pqv_mv<2>(ctx, a, m_v);

@@ -124,6 +124,7 @@ extern "C" lookat_status lookat_attend_static(lookat_ctx *handle, const float *l
     a.K = c.K;
     a.L_max = L_max;
     a.scale_log2 = ctx->scale * 1.4426950408889634f;
+    a.status = ctx->status_word;
     size_t po = 0, pml = 0;
     st = plan_attend(ctx, a, n_splits, &po, &pml);
     if (st != LOOKAT_OK) return st;

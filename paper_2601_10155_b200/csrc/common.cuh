@@ -19,6 +19,7 @@ struct Ctx {
     int max_smem_optin;
     int prefill_form;          // LOOKAT_PREFILL_*
     int *timeout_flag;         // pinned, device-visible: set by a kernel whose bounded barrier wait ran out
+    int *status_word;          // pinned, device-visible: LOOKAT_STATUS_* bits set by the debug build's checks
     float scale;           // resolved softmax scale
     char err[512];
     uint64_t launches;
@@ -99,6 +100,7 @@ struct AttendArgs {
     int n_ctas;
     int splits_per_unit;       // > 0: CTA c = chunk c % splits of unit c / splits; 0: flat ranges
     float scale_log2;          // scale * log2(e)
+    int *status;               // the context's status word (written by the debug build only)
     // attend_multi_kernel (rows of up to a few thousand tokens): units ordered KV head first, several per round
     int multi;                 // 1: that kernel
     int ut;                    // units per round (tables resident together)
@@ -188,6 +190,25 @@ lookat_status launch_layernorm(Ctx *ctx, const float *x, const __half *g, const 
 lookat_status launch_argmax(Ctx *ctx, const float *logits, int32_t *out, int rows, int n);
 lookat_status launch_causal_attention(Ctx *ctx, const __half *q, const __half *k, const __half *v, __half *out, int B, int H, int T,
                                       long long v_cap);
+
+// ---- the debug build's check of cache contents (-DLOOKAT_DEBUG): a code >= K is clamped to K - 1 before it is used as an
+//      index, and a bit of the context's status word records it; lookat_last_error reports the word.  In the normal
+//      build a code >= K is the caller's error and is used as it is (the streaming kernels' tables hold 256 entries per
+//      subspace, so they read garbage but stay in bounds; the generic kernel reads past its table). ----
+constexpr int kStatusBadCode = 1;
+#ifdef LOOKAT_DEBUG
+__device__ __forceinline__ int checked_code(int code, int K, int *status)
+{
+    if (code >= K) {
+        if (status) atomicOr(status, kStatusBadCode);
+        return K - 1;
+    }
+    return code;
+}
+#define LOOKAT_CHECKED_CODE(code, K, status) ::lookat::checked_code((code), (K), (status))
+#else
+#define LOOKAT_CHECKED_CODE(code, K, status) (code)
+#endif
 
 // ---- small device helpers ----
 __device__ __forceinline__ float ex2_approx(float x)
