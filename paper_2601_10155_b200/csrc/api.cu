@@ -302,10 +302,14 @@ const char *lookat_last_error(const lookat_ctx *handle)
     if (!handle) return "context is NULL";
     Ctx *ctx = const_cast<Ctx *>(reinterpret_cast<const Ctx *>(handle));
     // asynchronous findings of the debug build's device-side checks (meaningful once the caller has synchronised)
-    if (ctx->status_word && (*(volatile int *)ctx->status_word & kStatusBadCode)) {
+    if (ctx->status_word && *(volatile int *)ctx->status_word) {
+        const int word = *(volatile int *)ctx->status_word;
         *(volatile int *)ctx->status_word = 0;
-        snprintf(ctx->err, sizeof(ctx->err),
-                 "debug check: a code >= K was found in a code cache and clamped to K - 1; results computed from it are not valid");
+        if (word & kStatusCopyTimeout)
+            snprintf(ctx->err, sizeof(ctx->err), "attend: a bounded wait for a bulk copy ran out; the output of that call is not valid");
+        else
+            snprintf(ctx->err, sizeof(ctx->err),
+                     "debug check: a code >= K was found in a code cache and clamped to K - 1; results computed from it are not valid");
     }
     return ctx->err;
 }

@@ -100,7 +100,8 @@ struct AttendArgs {
     int n_ctas;
     int splits_per_unit;       // > 0: CTA c = chunk c % splits of unit c / splits; 0: flat ranges
     float scale_log2;          // scale * log2(e)
-    int *status;               // the context's status word (written by the debug build only)
+    int *status;               // the context's status word (the debug build's checks; a bulk copy that never completed)
+    int bulk;                  // attend_stream_kernel: tiles by cp.async.bulk + mbarrier (else 16-byte cp.async)
     // attend_multi_kernel (rows of up to a few thousand tokens): units ordered KV head first, several per round
     int multi;                 // 1: that kernel
     int ut;                    // units per round (tables resident together)
@@ -183,6 +184,11 @@ struct LinearArgs {
     int *timeout_flag;
 };
 // out = act(x w_t^T + bias) [+ residual]; x [M][K] fp16 (fp32 accepted for M <= 32), w_t [N][K] fp16
+// tensor maps for tiled bulk copies (linear_umma.cu): `map` points at a CUtensorMap; [rows][inner] fp16 row-major, boxes of
+// box_rows x box_inner elements, 128-byte swizzle, zeros outside.  False if the driver entry point is missing or refuses.
+bool tile_maps_available();
+bool make_tile_map_f16(void *map, const void *base, unsigned long long inner, unsigned long long rows, unsigned box_inner,
+                       unsigned box_rows);
 lookat_status launch_linear(Ctx *ctx, const void *x, int x_fp32, const __half *w_t, LinearArgs p);
 lookat_status launch_embed(Ctx *ctx, const int32_t *ids, const __half *wte, const __half *wpe, float *x, long long rows, int T,
                            int pos0, int d, int vocab);
@@ -196,6 +202,7 @@ lookat_status launch_causal_attention(Ctx *ctx, const __half *q, const __half *k
 //      build a code >= K is the caller's error and is used as it is (the streaming kernels' tables hold 256 entries per
 //      subspace, so they read garbage but stay in bounds; the generic kernel reads past its table). ----
 constexpr int kStatusBadCode = 1;
+constexpr int kStatusCopyTimeout = 2;       // a bounded wait for a bulk copy ran out (any build)
 #ifdef LOOKAT_DEBUG
 __device__ __forceinline__ int checked_code(int code, int K, int *status)
 {

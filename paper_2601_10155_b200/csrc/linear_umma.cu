@@ -375,6 +375,21 @@ bool make_operand_map(CUtensorMap *map, const void *base, long long rows, int K)
 
 }  // namespace
 
+bool tile_maps_available() { return tensor_map_encoder() != nullptr; }
+
+bool make_tile_map_f16(void *map, const void *base, unsigned long long inner, unsigned long long rows, unsigned box_inner,
+                       unsigned box_rows)
+{
+    tensor_map_encode_fn encode = tensor_map_encoder();
+    if (!encode) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)inner * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows}, estr[2] = {1, 1};
+    return encode(static_cast<CUtensorMap *>(map), CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 lookat_status launch_linear(Ctx *ctx, const void *x, int x_fp32, const __half *w_t, LinearArgs p)
 {
     p.timeout_flag = ctx->timeout_flag;
