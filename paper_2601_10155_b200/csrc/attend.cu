@@ -157,7 +157,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
     constexpr int VT = (DV / 64) * 2048;                   // V bytes of a tile
     const unsigned ring0_s = (unsigned)__cvta_generic_to_shared(smem_raw + region0 + q_bytes);
     const unsigned vring_s = ((ring0_s + 1023u) & ~1023u) + (unsigned)(warp * STAGES * VT);
-    unsigned char *const vring = smem_raw + region0 + q_bytes + (vring_s - ring0_s);
     const unsigned cring_off = (unsigned)(kWarps * STAGES * VT + warp * STAGES * kTile * M_SUB) - (unsigned)(warp * STAGES * VT);
     const unsigned bar_s = ((ring0_s + 1023u) & ~1023u) + (unsigned)(kWarps * STAGES * (VT + kTile * M_SUB) + warp * STAGES * 8);
     if (BULK) {
@@ -220,6 +219,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
                 if (nv > 0) {
                     // ragged end of a row: plain copies into the same layout; rows at or beyond seq_len are never read from
                     // memory, zeros stand in
+                    unsigned char *const vring = smem_raw + region0 + q_bytes + (vring_s - ring0_s);
                     unsigned char *vdst = vring + slot * VT, *cdst = vring + cring_off + slot * (kTile * M_SUB);
 #pragma unroll
                     for (int it = 0; it < V_CHUNKS; ++it) {
@@ -440,11 +440,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             if (BULK) {
                 // the tile's bytes have landed when the slot's barrier completes the phase (bounded: a copy that never
                 // completes is reported through the status word and the tile is taken as it is)
-                unsigned ok = 0;
-                for (int it = 0; it < (1 << 22) && !ok; ++it)
-                    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                unsigned ok = 0;                           // each try may park the warp for up to ~2 us instead of spinning
+                for (int it = 0; it < (1 << 17) && !ok; ++it)
+                    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
                                  : "=r"(ok)
-                                 : "r"(bar_s + 8 * slot), "r"(ring_parity)
+                                 : "r"(bar_s + 8 * slot), "r"(ring_parity), "r"(2000u)
                                  : "memory");
                 if (!ok && a.status) atomicOr(a.status, kStatusCopyTimeout);
             } else {
@@ -457,7 +457,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             CodePair<M_SUB> cp;
             if (nv > 0) {                                  // tile -> registers, so the slot can be refilled
                 if (BULK) {
-                    cp = read_code_pair<M_SUB>(vring + cring_off + slot * (kTile * M_SUB) + ts_off * M_SUB);
+                    cp = read_code_pair_s<M_SUB>(vring_s + cring_off + slot * (kTile * M_SUB) + ts_off * M_SUB);
                     // row r of box nb at nb * 2048 + r * 128, its 16-byte piece c at (c ^ (r & 7)) * 16; MMA i wants pieces
                     // 2 i and 2 i + 1 of the 256-byte row: box i / 4, piece 2 (i % 4) + hi
 #pragma unroll

@@ -112,6 +112,28 @@ __device__ __forceinline__ CodePair<M_SUB> read_code_pair(const unsigned char *p
     return c;
 }
 
+// the same from a shared-memory address (32-bit), so that no generic pointer to the slot has to stay live
+template <int M_SUB>
+__device__ __forceinline__ CodePair<M_SUB> read_code_pair_s(unsigned p)
+{
+    CodePair<M_SUB> c;
+    if constexpr (M_SUB == 16) {
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(c.w[0]), "=r"(c.w[1]), "=r"(c.w[2]), "=r"(c.w[3]) : "r"(p));
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(c.w[4]), "=r"(c.w[5]), "=r"(c.w[6]), "=r"(c.w[7]) : "r"(p + 16));
+    } else if constexpr (M_SUB == 8) {
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(c.w[0]), "=r"(c.w[1]), "=r"(c.w[2]), "=r"(c.w[3]) : "r"(p));
+    } else if constexpr (M_SUB == 4) {
+        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(c.w[0]), "=r"(c.w[1]) : "r"(p));
+    } else if constexpr (M_SUB == 2) {
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(c.w[0]) : "r"(p));
+    } else {
+        unsigned short v;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(p));
+        c.w[0] = v;
+    }
+    return c;
+}
+
 template <int M_SUB>
 __device__ __forceinline__ int code_at(const CodePair<M_SUB> &c, int token01, int j)
 {
