@@ -49,60 +49,61 @@ namespace lookat {
 
 namespace {
 
-// Position in the flat tile sequence: tile `lt` of unit `unit`, with that unit's row facts and
-// the addresses of the tile's V rows and codes.
+// Position in the flat tile sequence: tile `lt` of unit `unit`, with that unit's row facts and the tile's first row of
+// the caches.  Kept small (the streaming loop holds two of them in registers): the position is counted from the start of
+// the CTA's range, addresses are formed from the row where a copy is issued.
+template <class Row>     // int where the caches have fewer than 2^31 rows (the plan sends only those to the bulk copies)
 struct TileCursor {
-    long long T;         // flat index
+    int t;               // flat index minus the first tile of the CTA's range
     int unit, lt;
     int len;             // tokens in the unit's batch row (0 beyond the last unit)
-    const unsigned char *vptr, *cptr;
+    Row row0;            // (batch row * H_kv + KV head) * L_max + 16 lt
 };
 
-template <int M_SUB, int DV>
-__device__ __forceinline__ void cursor_enter_unit(const AttendArgs &a, TileCursor &c, int hgroups)
+template <class Row>
+__device__ __forceinline__ void cursor_enter_unit(const AttendArgs &a, TileCursor<Row> &c, int hgroups)
 {
     if (c.unit < a.n_units) {
         const int kv_row = c.unit / hgroups;             // (batch row, KV head) of the unit
         const int b = kv_row / a.H_kv;
         c.len = (int)min((long long)(a.seq_lens ? a.seq_lens[b] : a.uniform_len), a.L_max);
-        const size_t row0 = (size_t)kv_row * a.L_max + (size_t)c.lt * kTile;
-        c.vptr = reinterpret_cast<const unsigned char *>(a.v) + row0 * (DV * 2);
-        c.cptr = a.codes + row0 * M_SUB;
+        c.row0 = (Row)((long long)kv_row * a.L_max + (long long)c.lt * kTile);
     } else {
         c.len = 0;
     }
 }
 
-template <int M_SUB, int DV>
-__device__ __forceinline__ TileCursor cursor_at(const AttendArgs &a, long long T, int hgroups)
+template <class Row>
+__device__ __forceinline__ TileCursor<Row> cursor_at(const AttendArgs &a, long long T_lo, int t, int hgroups)
 {
-    TileCursor c;
-    c.T = T;
+    TileCursor<Row> c;
+    const long long T = T_lo + t;
+    c.t = t;
     c.unit = (int)(T / a.tiles_per_unit);
     c.lt = (int)(T - (long long)c.unit * a.tiles_per_unit);
-    c.vptr = c.cptr = nullptr;
-    cursor_enter_unit<M_SUB, DV>(a, c, hgroups);
+    c.row0 = 0;
+    cursor_enter_unit(a, c, hgroups);
     return c;
 }
 
-template <int M_SUB, int DV>
-__device__ __forceinline__ void cursor_advance(const AttendArgs &a, TileCursor &c, int hgroups)
+template <class Row>
+__device__ __forceinline__ void cursor_advance(const AttendArgs &a, TileCursor<Row> &c, int hgroups)
 {
-    c.T += kWarps;
+    c.t += kWarps;
     c.lt += kWarps;
-    c.vptr += kWarps * kTile * DV * 2;
-    c.cptr += kWarps * kTile * M_SUB;
+    c.row0 += kWarps * kTile;
     if (c.lt >= a.tiles_per_unit) {
         do {
             c.lt -= a.tiles_per_unit;
             c.unit += 1;
         } while (c.lt >= a.tiles_per_unit);
-        cursor_enter_unit<M_SUB, DV>(a, c, hgroups);
+        cursor_enter_unit(a, c, hgroups);
     }
 }
 
 // Tokens of the cursor's tile that exist (0..16).
-__device__ __forceinline__ int cursor_valid(const TileCursor &c)
+template <class Row>
+__device__ __forceinline__ int cursor_valid(const TileCursor<Row> &c)
 {
     const int left = c.len - c.lt * kTile;
     return left >= kTile ? kTile : (left > 0 ? left : 0);
@@ -168,6 +169,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         __syncwarp();
     }
 
+    // the streamed bytes are used once: marked to leave L2 first, so that what the CTAs read again and again (codebooks,
+    // queries, partials) stays
+    unsigned long long stream_policy = 0;
+    if (BULK) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
+
     const float *my_table = lut_s + hl * head_stride;
 
     // a lane copies the 16-byte piece (lane*16 + it*512) of a tile's V bytes, it = 0..V_CHUNKS-1
@@ -192,9 +198,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         T_hi = min((long long)a.n_units * a.tiles_per_unit, T_lo + a.tiles_per_cta);
     }
 
+    const int t_hi = (int)(T_hi - T_lo);                  // a CTA's range is far below 2^31 tiles
+
     // ---- producer: the cursor's tile into ring slot `slot` (always closes one copy group) ----
-    auto issue = [&](const TileCursor &pc, int slot) {
-        const int nv = pc.T < T_hi ? cursor_valid(pc) : 0;
+    using Cursor = TileCursor<std::conditional_t<BULK, int, long long>>;
+    auto issue = [&](const Cursor &pc, int slot) {
+        const int nv = pc.t < t_hi ? cursor_valid(pc) : 0;
+        const unsigned char *const pc_vptr = reinterpret_cast<const unsigned char *>(a.v) + (size_t)pc.row0 * (DV * 2);
+        const unsigned char *const pc_cptr = a.codes + (size_t)pc.row0 * M_SUB;
         if (BULK) {
             const unsigned bar = bar_s + 8 * slot;
             const unsigned vdst_s = vring_s + slot * VT;
@@ -202,17 +213,17 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
                 if (lane == 0) {
                     // one arrival that also announces the tile's bytes, then the copies
                     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "n"(VT + kTile * M_SUB) : "memory");
-                    const int row0 = (int)((pc.vptr - reinterpret_cast<const unsigned char *>(a.v)) / (DV * 2));
+                    const int row0 = (int)pc.row0;
 #pragma unroll
                     for (int nb = 0; nb < DV / 64; ++nb)
                         asm volatile(
-                            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+                            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(
                                 vdst_s + nb * 2048),
-                            "l"(reinterpret_cast<uint64_t>(&v_map)), "r"(nb * 64), "r"(row0), "r"(bar)
+                            "l"(reinterpret_cast<uint64_t>(&v_map)), "r"(nb * 64), "r"(row0), "r"(bar), "l"(stream_policy)
                             : "memory");
-                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
                                      vring_s + cring_off + slot * (kTile * M_SUB)),
-                                 "l"(pc.cptr), "n"(kTile * M_SUB), "r"(bar)
+                                 "l"(pc_cptr), "n"(kTile * M_SUB), "r"(bar), "l"(stream_policy)
                                  : "memory");
                 }
             } else {
@@ -225,12 +236,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
                     for (int it = 0; it < V_CHUNKS; ++it) {
                         const int o = lane * 16 + it * 512, r = o / (DV * 2), ci = (o % (DV * 2)) >> 4;
                         uint4 val = make_uint4(0, 0, 0, 0);
-                        if (r < nv) val = *reinterpret_cast<const uint4 *>(pc.vptr + o);
+                        if (r < nv) val = *reinterpret_cast<const uint4 *>(pc_vptr + o);
                         *reinterpret_cast<uint4 *>(vdst + (ci >> 3) * 2048 + r * 128 + (((ci & 7) ^ (r & 7)) << 4)) = val;
                     }
                     if (lane < kTile) {
 #pragma unroll
-                        for (int j = 0; j < M_SUB; ++j) cdst[lane * M_SUB + j] = lane < nv ? pc.cptr[lane * M_SUB + j] : 0;
+                        for (int j = 0; j < M_SUB; ++j) cdst[lane * M_SUB + j] = lane < nv ? pc_cptr[lane * M_SUB + j] : 0;
                     }
                     __syncwarp();
                 }
@@ -239,8 +250,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             return;
         }
         if (nv > 0) {
-            const unsigned char *vsrc = pc.vptr;
-            const unsigned char *csrc = pc.cptr;
+            const unsigned char *vsrc = pc_vptr;
+            const unsigned char *csrc = pc_cptr;
             unsigned char *dst = ring + slot * SLOT;
             const unsigned dst_s = ring_s + slot * SLOT;
             if (nv == kTile) {
@@ -371,12 +382,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
     }
 
     // ---- prologue: fill the ring with this warp's first STAGES tiles ----
-    TileCursor cc = cursor_at<M_SUB, DV>(a, T_lo + warp, hgroups);   // tile this warp consumes next
-    TileCursor pc = cc;                                              // tile it copies next
+    Cursor cc = cursor_at<decltype(Cursor::row0)>(a, T_lo, warp, hgroups);   // tile this warp consumes next
+    Cursor pc = cc;                                                  // tile it copies next
 #pragma unroll
     for (int s = 0; s < STAGES; ++s) {
         issue(pc, s);
-        cursor_advance<M_SUB, DV>(a, pc, hgroups);
+        cursor_advance(a, pc, hgroups);
     }
     if (a.new_keys && !append_first) append_new_keys();
     int slot = 0;                                          // ring slot of the consumer's tile
@@ -423,7 +434,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
 
             const int d_sub = a.d_k / M_SUB;
             const float *book = a.codebooks + (size_t)kvh * table * d_sub;
-            build_unit_tables(book, q_s, lut_s, table, a.K, d_sub, heads_here, head_stride, tid);
+            build_unit_tables<false>(book, q_s, lut_s, table, a.K, d_sub, heads_here, head_stride, tid, nullptr, nullptr);
         }
         __syncthreads();
 
@@ -434,9 +445,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         float *scores_row =
             (a.scores_out && head_ok) ? a.scores_out + ((size_t)b * a.H_q + hq0 + hl) * a.L_max : nullptr;
 
-        const long long seg_hi = min(T_hi, (long long)(unit + 1) * a.tiles_per_unit);
+        const int seg_hi = (int)(min(T_hi, (long long)(unit + 1) * a.tiles_per_unit) - T_lo);
         const bool full_unit = heads_here == 4 && !a.scores_out;
-        while (cc.T < seg_hi) {
+        while (cc.t < seg_hi) {
             if (BULK) {
                 // the tile's bytes have landed when the slot's barrier completes the phase (bounded: a copy that never
                 // completes is reported through the status word and the tile is taken as it is)
@@ -472,14 +483,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
             }
             __syncwarp();                                  // all lanes have read the slot
             issue(pc, slot);
-            cursor_advance<M_SUB, DV>(a, pc, hgroups);
+            cursor_advance(a, pc, hgroups);
             if (nv == kTile && full_unit)
                 process_tile(std::true_type{}, 0, kTile, vf, cp, true, nullptr);
             else if (nv > 0)
                 process_tile(std::false_type{}, cc.lt * kTile, nv, vf, cp, head_ok, scores_row);
             slot = slot + 1 == STAGES ? 0 : slot + 1;
             if (slot == 0) ring_parity ^= 1u;
-            cursor_advance<M_SUB, DV>(a, cc, hgroups);
+            cursor_advance(a, cc, hgroups);
         }
 
         // ---- this warp's result for the unit: fold the weight and remainder columns ----

@@ -264,50 +264,8 @@ __device__ __forceinline__ void append_round_staged(const RoundFacts &f, const f
         const int ul = task / f.m, j = task - ul * f.m;
         if (!((mine >> ul) & 1u)) continue;
         const float *dj = dist + (size_t)ul * f.set_floats + j * f.K;
-        float d[8];
-        Best r;
-        r.best = INFINITY; r.second = INFINITY; r.idx = 0x7fffffff;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int c = lane + 32 * k;
-            d[k] = c < f.K ? dj[c] : INFINITY;
-            if (c < f.K) consider(r, d[k], c);
-        }
-        for (int s = 16; s; s >>= 1) {
-            const float ob = __shfl_xor_sync(0xffffffffu, r.best, s);
-            const float os = __shfl_xor_sync(0xffffffffu, r.second, s);
-            const int oi = __shfl_xor_sync(0xffffffffu, r.idx, s);
-            const bool other_wins = ob < r.best || (ob == r.best && oi < r.idx);
-            const float loser = other_wins ? r.best : ob;
-            r.second = fminf(fminf(r.second, os), loser);
-            if (other_wins) { r.best = ob; r.idx = oi; }
-        }
-        int code = r.idx;
-        if (needs_fp64(r)) {                               // warp-uniform
-            const float *x = xk + ul * f.d_k + j * f.d_sub;
-            const StagedBook book{book_s, j * f.K, f.d_sub, n_c, sh};
-            const float limit = r.best * (1.f + 2.f * kBand);
-            double best = INFINITY;
-            int idx = 0x7fffffff;
-#pragma unroll 1
-            for (int k = 0; k < 8; ++k) {
-                const int c = lane + 32 * k;
-                if (c < f.K && d[k] <= limit) {
-                    double dd = 0.0;
-                    for (int i = 0; i < f.d_sub; ++i) {
-                        const double t = (double)x[i] - (double)book.load1(c, i);
-                        dd = __dadd_rn(dd, __dmul_rn(t, t));      // product and sum rounded separately
-                    }
-                    if (dd < best) { best = dd; idx = c; }
-                }
-            }
-            for (int s = 16; s; s >>= 1) {
-                const double ob = __shfl_xor_sync(0xffffffffu, best, s);
-                const int oi = __shfl_xor_sync(0xffffffffu, idx, s);
-                if (ob < best || (ob == best && oi < idx)) { best = ob; idx = oi; }
-            }
-            code = idx;
-        }
+        const int code = code_from_distances(dj, xk + ul * f.d_k + j * f.d_sub, StagedBook{book_s, j * f.K, f.d_sub, n_c, sh}, f.K,
+                                             f.d_sub, lane);
         if (lane == 0) {
             cache[(((size_t)ru->b[ul] * f.H_kv + kvh) * L_max + new_pos) * f.m + j] = (uint8_t)code;
             newc[ul * 16 + j] = (unsigned char)code;
@@ -385,8 +343,8 @@ __device__ __noinline__ void round_tables(const AttendArgs &a, unsigned char *sm
     } else {
         for (int ul = 0; ul < nr; ++ul) {
             const int heads_here = min(4, f.g - ru->hgrp[ul] * 4);
-            build_unit_tables(books_g + (size_t)kvh * f.table * f.d_sub, q_s + (size_t)ul * f.d_k * 4,
-                              lut_s + (size_t)ul * f.set_floats, f.table, f.K, f.d_sub, heads_here, f.head_stride, tid);
+            build_unit_tables<false>(books_g + (size_t)kvh * f.table * f.d_sub, q_s + (size_t)ul * f.d_k * 4,
+                              lut_s + (size_t)ul * f.set_floats, f.table, f.K, f.d_sub, heads_here, f.head_stride, tid, nullptr, nullptr);
         }
     }
 }

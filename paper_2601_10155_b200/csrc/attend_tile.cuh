@@ -142,9 +142,12 @@ __device__ __forceinline__ int code_at(const CodePair<M_SUB> &c, int token01, in
 }
 
 // The table entries of one unit, out of line: its registers are its own, so the next entry's centroid can be
-// requested ahead without touching the allocation of the streaming loop.
+// requested ahead without touching the allocation of the streaming loop.  With xk (a key of d_k floats in shared
+// memory) the fp32 squared distance of every centroid to its sub-vector of the key goes to dist[j * kTableStride + c],
+// formed as the warp search of encode_warp.cuh forms it: the append's search rides on the centroids read here.
+template <bool DIST>
 __device__ __noinline__ void build_unit_tables(const float *book, const double *q_s, float *lut_s, int table, int K,
-                                               int d_sub, int heads_here, int head_stride, int tid)
+                                               int d_sub, int heads_here, int head_stride, int tid, const float *xk, float *dist)
 {
     const bool vec16 = d_sub == 16;
     float4 pre[4];
@@ -157,7 +160,13 @@ __device__ __noinline__ void build_unit_tables(const float *book, const double *
         const int es = j * kTableStride + (e - j * K);
         const double *qj = q_s + 4 * j * d_sub;
         double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
+        float dacc = 0.f;
+        const float *xj = DIST ? xk + j * d_sub : nullptr;
         auto step = [&](int i, float cf) {
+            if constexpr (DIST) {
+                const float t = xj[i] - cf;
+                dacc = fmaf(t, t, dacc);
+            }
             const double cv = (double)cf;
             const double2 q01 = *reinterpret_cast<const double2 *>(qj + 4 * i);
             const double2 q23 = *reinterpret_cast<const double2 *>(qj + 4 * i + 2);
@@ -187,6 +196,7 @@ __device__ __noinline__ void build_unit_tables(const float *book, const double *
         if (heads_here > 1) lut_s[head_stride + es] = (float)t1;
         if (heads_here > 2) lut_s[2 * head_stride + es] = (float)t2;
         if (heads_here > 3) lut_s[3 * head_stride + es] = (float)t3;
+        if constexpr (DIST) dist[es] = dacc;
     }
 }
 

@@ -103,6 +103,58 @@ struct StagedBook {                    // a head's codebooks staged in shared me
     }
 };
 
+// The code of one key sub-vector from the fp32 squared distances dj[0..K) of all centroids, formed as in the warp search
+// below (difference form, fmaf in dimension order), by one warp: the two smallest decide; where they are within kBand the
+// centroids within twice the band of the smallest are decided again in fp64 -- no other centroid can be the fp64 minimum,
+// the fp32 error being below (d_sub + 2) 2^-24 relative -- lowest index first.  Every lane returns the code.
+template <class Book>
+__device__ __forceinline__ int code_from_distances(const float *dj, const float *x, const Book &book, int K, int d_sub, int lane)
+{
+    float d[8];
+    Best r;
+    r.best = INFINITY; r.second = INFINITY; r.idx = 0x7fffffff;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int c = lane + 32 * k;
+        d[k] = c < K ? dj[c] : INFINITY;
+        if (c < K) consider(r, d[k], c);
+    }
+    for (int s = 16; s; s >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, r.best, s);
+        const float os = __shfl_xor_sync(0xffffffffu, r.second, s);
+        const int oi = __shfl_xor_sync(0xffffffffu, r.idx, s);
+        const bool other_wins = ob < r.best || (ob == r.best && oi < r.idx);
+        const float loser = other_wins ? r.best : ob;
+        r.second = fminf(fminf(r.second, os), loser);
+        if (other_wins) { r.best = ob; r.idx = oi; }
+    }
+    int code = r.idx;
+    if (needs_fp64(r)) {                               // warp-uniform
+        const float limit = r.best * (1.f + 2.f * kBand);
+        double best = INFINITY;
+        int idx = 0x7fffffff;
+#pragma unroll 1
+        for (int k = 0; k < 8; ++k) {
+            const int c = lane + 32 * k;
+            if (c < K && d[k] <= limit) {
+                double dd = 0.0;
+                for (int i = 0; i < d_sub; ++i) {
+                    const double t = (double)x[i] - (double)book.load1(c, i);
+                    dd = __dadd_rn(dd, __dmul_rn(t, t));      // product and sum rounded separately
+                }
+                if (dd < best) { best = dd; idx = c; }
+            }
+        }
+        for (int s = 16; s; s >>= 1) {
+            const double ob = __shfl_xor_sync(0xffffffffu, best, s);
+            const int oi = __shfl_xor_sync(0xffffffffu, idx, s);
+            if (ob < best || (ob == best && oi < idx)) { best = ob; idx = oi; }
+        }
+        code = idx;
+    }
+    return code;
+}
+
 // the key sub-vector as fp16 (global memory) or already widened to fp32 (shared memory): both exact
 __device__ __forceinline__ float key_dim(const __half *x, int i) { return __half2float(x[i]); }
 __device__ __forceinline__ float key_dim(const float *x, int i) { return x[i]; }
