@@ -101,6 +101,22 @@ __device__ __forceinline__ void cursor_advance(const AttendArgs &a, TileCursor<R
     }
 }
 
+// The cursor `ahead` tiles further on.  The copies run a fixed distance ahead of the tile a warp works on, so their
+// position is derived from that tile's instead of being carried along; only next to a unit's end is it looked up anew.
+template <class Row>
+__device__ __forceinline__ TileCursor<Row> cursor_ahead(const AttendArgs &a, const TileCursor<Row> &c, long long T_lo, int ahead,
+                                                        int hgroups)
+{
+    if (c.lt + ahead < a.tiles_per_unit && c.unit < a.n_units) {
+        TileCursor<Row> p = c;
+        p.t += ahead;
+        p.lt += ahead;
+        p.row0 += (Row)(ahead * kTile);
+        return p;
+    }
+    return cursor_at<Row>(a, T_lo, c.t + ahead, hgroups);
+}
+
 // Tokens of the cursor's tile that exist (0..16).
 template <class Row>
 __device__ __forceinline__ int cursor_valid(const TileCursor<Row> &c)
@@ -171,8 +187,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
 
     // the streamed bytes are used once: marked to leave L2 first, so that what the CTAs read again and again (codebooks,
     // queries, partials) stays
-    unsigned long long stream_policy = 0;
-    if (BULK) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
+    // (the value createpolicy.fractional.L2::evict_first yields for the whole line, as CUTLASS's cache-hint constants
+    // have it; as a constant it occupies no registers between copies)
+    constexpr unsigned long long stream_policy = 0x12F0000000000000ull;
 
     const float *my_table = lut_s + hl * head_stride;
 
@@ -383,12 +400,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
 
     // ---- prologue: fill the ring with this warp's first STAGES tiles ----
     Cursor cc = cursor_at<decltype(Cursor::row0)>(a, T_lo, warp, hgroups);   // tile this warp consumes next
-    Cursor pc = cc;                                                  // tile it copies next
 #pragma unroll
-    for (int s = 0; s < STAGES; ++s) {
-        issue(pc, s);
-        cursor_advance(a, pc, hgroups);
-    }
+    for (int s = 0; s < STAGES; ++s) issue(cursor_ahead(a, cc, T_lo, s * kWarps, hgroups), s);
     if (a.new_keys && !append_first) append_new_keys();
     int slot = 0;                                          // ring slot of the consumer's tile
     unsigned ring_parity = 0;                              // BULK: phase of the slots' barriers the consumer waits for
@@ -442,8 +455,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
         for (int i = 0; i < DV / 16; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
         m_run = kNegBig;
         l_run = 0.f;
-        float *scores_row =
-            (a.scores_out && head_ok) ? a.scores_out + ((size_t)b * a.H_q + hq0 + hl) * a.L_max : nullptr;
 
         const int seg_hi = (int)(min(T_hi, (long long)(unit + 1) * a.tiles_per_unit) - T_lo);
         const bool full_unit = heads_here == 4 && !a.scores_out;
@@ -482,12 +493,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_stream_kernel(AttendArgs a
                 }
             }
             __syncwarp();                                  // all lanes have read the slot
-            issue(pc, slot);
-            cursor_advance(a, pc, hgroups);
+            issue(cursor_ahead(a, cc, T_lo, STAGES * kWarps, hgroups), slot);   // the tile STAGES of this warp's tiles ahead
             if (nv == kTile && full_unit)
                 process_tile(std::true_type{}, 0, kTile, vf, cp, true, nullptr);
             else if (nv > 0)
-                process_tile(std::false_type{}, cc.lt * kTile, nv, vf, cp, head_ok, scores_row);
+                process_tile(std::false_type{}, cc.lt * kTile, nv, vf, cp, head_ok,
+                             (a.scores_out && head_ok) ? a.scores_out + ((size_t)b * a.H_q + hq0 + hl) * a.L_max : nullptr);
             slot = slot + 1 == STAGES ? 0 : slot + 1;
             if (slot == 0) ring_parity ^= 1u;
             cursor_advance(a, cc, hgroups);
