@@ -39,8 +39,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per (token, KV head) pair of one
 # attend_stream_kernel launch, from an ncu capture of the batch-4 case of gqa_32k_m8
-# (279,958,784 + 6,347,008 bytes over 1,048,576 pairs; traffic grows in proportion to the pairs).
-ATTEND_DRAM_BYTES_PER_PAIR = {"gqa_32k_m8": 286305792 / 1048576}
+# (278,003,200 + 4,173,056 bytes over 1,048,576 pairs; traffic grows in proportion to the pairs).
+ATTEND_DRAM_BYTES_PER_PAIR = {"gqa_32k_m8": 282176256 / 1048576}
 ATTEND_TRAFFIC_SOURCE = ("ncu capture of attend_stream_kernel<8,128,2,true> (bulk-copy ring) on gqa_32k_m8 at batch 4 "
                          "(profiles/attend_stream_kernel_gqa_32k_m8_batch4_ncu.md), scaled by the pair count")
 SMALL_WORKLOADS = ["gpt2_l128_m4", "gpt2_b8_l256_m2", "gpt2_b8_l512_m2", "gpt2_b8_l1024_m2", "gpt2_b32_l1024_m4"]
