@@ -255,8 +255,8 @@ lookat_status lookat_decode_step_host(lookat_ctx *ctx, const void *q_host, const
  *   LOOKAT_PREFILL_CONTRACTION  the centroids named by a chunk of codes are
  *                               gathered once per 256 queries and the scores
  *                               taken as q . (C_1[c_1], ..., C_m[c_m]) on the
- *                               tensor cores (d_k and d_v in {64, 128}, d_sub a
- *                               multiple of 8, both codebook planes of a head
+ *                               tensor cores (d_k and d_v in {64, 128}, d_sub 4
+ *                               or a multiple of 8, both codebook planes of a head
  *                               in shared memory: K * d_k * 4 bytes; L_max * m a
  *                               multiple of 4); tcgen05.mma with accumulators
  *                               in tensor memory;

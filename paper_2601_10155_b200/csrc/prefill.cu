@@ -379,7 +379,7 @@ lookat_status launch_prefill(Ctx *ctx, const PrefillArgs &a)
         if (prefill_umma_covers(ctx, a)) return launch_prefill_umma(ctx, a);
         if (want)
             return set_error(ctx, LOOKAT_ERR_UNSUPPORTED,
-                             "attend_prefill: the contraction form needs d_k, d_v in {64, 128}, d_sub a multiple of 8, L_max * m a "
+                             "attend_prefill: the contraction form needs d_k, d_v in {64, 128}, d_sub 4 or a multiple of 8, L_max * m a "
                              "multiple of 4, a positive scale and K * d_k * 4 bytes of shared memory for the codebooks");
     }
     if (a.d_v % 8 != 0 || a.d_v > 256 || ((uintptr_t)a.v & 15) != 0 || ((uintptr_t)a.codes & 3) != 0)

@@ -336,7 +336,8 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
         const uint8_t *codes = a.codes + (size_t)(b * a.H_kv + h) * a.L_max * a.m;
         // item p = ptid + i * producers of a chunk: token p / kIds, id = p % kIds = plane * (D_K/8) + gi (fixed per thread)
         const int my_id = ptid % Lay::kIds, my_plane = my_id / (D_K / 8), my_gi = my_id % (D_K / 8);
-        const int my_j = (my_gi * 8) / d_sub;
+        const int my_j = (my_gi * 8) / d_sub;                  // the (first) subspace of this thread's 8-dim group
+        const bool pair = d_sub == 4;                          // ... which holds two sub-vectors when they have 4 dims
         const unsigned char *my_src = book + (uint32_t)my_plane * (book_bytes / 2) + (uint32_t)(my_gi >> 3) * a.K * 128 + ((my_gi & 7) << 4);
         unsigned char *my_dst = sm + Lay::kOffKeys + (my_gi >> 3) * (2 * kUmChunk * 128) + my_plane * (kUmChunk * 128);   // + buf * kKeys
         const int tl0 = ptid / Lay::kIds;                      // this thread's tokens of a chunk: tl0 + i * (producers / kIds)
@@ -359,15 +360,28 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             const uint8_t *cs = codes_s + buf * 1024 + my_j;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {             // in two batches: all loads of a batch before its stores
-                uint32_t code[Lay::kItems / 2];
+                uint32_t code[Lay::kItems / 2], code_b[Lay::kItems / 2];
                 uint4 item[Lay::kItems / 2];
 #pragma unroll
-                for (int i = 0; i < Lay::kItems / 2; ++i) code[i] = cs[(tl0 + (half * (Lay::kItems / 2) + i) * kTokStep) * a.m];
+                for (int i = 0; i < Lay::kItems / 2; ++i) {
+                    const uint8_t *ct = cs + (tl0 + (half * (Lay::kItems / 2) + i) * kTokStep) * a.m;
+                    code[i] = ct[0];
+                    code_b[i] = pair ? ct[1] : 0u;
+                }
 #pragma unroll
                 for (int i = 0; i < Lay::kItems / 2; ++i) {
                     item[i] = make_uint4(0u, 0u, 0u, 0u);
-                    if (whole || (long long)c * kUmChunk + tl0 + (half * (Lay::kItems / 2) + i) * kTokStep < t_end)
-                        item[i] = *reinterpret_cast<const uint4 *>(my_src + code[i] * 128);
+                    if (whole || (long long)c * kUmChunk + tl0 + (half * (Lay::kItems / 2) + i) * kTokStep < t_end) {
+                        if (!pair) {
+                            item[i] = *reinterpret_cast<const uint4 *>(my_src + code[i] * 128);
+                        } else {
+                            // sub-vectors of 4 dims: the group's first half from the centroid of subspace 2 gi, its second
+                            // half from the centroid of subspace 2 gi + 1 (the image holds both at the same place of their rows)
+                            const uint2 lo = *reinterpret_cast<const uint2 *>(my_src + code[i] * 128);
+                            const uint2 hi = *reinterpret_cast<const uint2 *>(my_src + code_b[i] * 128 + 8);
+                            item[i] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+                        }
+                    }
                 }
 #pragma unroll
                 for (int i = 0; i < Lay::kItems / 2; ++i) {
@@ -629,7 +643,8 @@ lookat_status launch_um(Ctx *ctx, const PrefillArgs &a)
 bool prefill_umma_covers(const Ctx *ctx, const PrefillArgs &a)
 {
     const int d_sub = a.d_k / a.m;
-    const bool shape = (a.d_k == 64 || a.d_k == 128) && (a.d_v == 64 || a.d_v == 128) && d_sub % 8 == 0;
+    // (m <= 16: the codes of a chunk are staged in 1 KB of shared memory)
+    const bool shape = (a.d_k == 64 || a.d_k == 128) && (a.d_v == 64 || a.d_v == 128) && (d_sub % 8 == 0 || d_sub == 4) && a.m <= 16;
     const bool aligned = ((uintptr_t)a.q & 15) == 0 && ((uintptr_t)a.v & 15) == 0 && ((uintptr_t)a.codes & 3) == 0 &&
                          (a.L_max * a.m) % 4 == 0;
     // the row maxima are taken on the raw scores, which needs a positive softmax scale

@@ -407,7 +407,9 @@ def test_invalid_arguments_are_rejected_without_launching():
     (dict(B=1, n_q_heads=3, n_kv_heads=3, d_k=24, d_v=16, m=8, K=7, L=65), 65, 0),          # d_sub 3, small K
     (dict(B=1, n_q_heads=2, n_kv_heads=1, d_k=128, d_v=64, m=16, K=200, L=450), 300, 150),  # 3 query tiles, ragged, K < 256
     (dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=128, m=8, K=256, L=257), 257, 0),     # d_k 64; one row in the last tile
-    (dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=64, m=16, K=256, L=90), 90, 0),       # d_sub 4: tables only
+    (dict(B=1, n_q_heads=2, n_kv_heads=2, d_k=64, d_v=64, m=16, K=256, L=90), 90, 0),       # d_sub 4: two centroids per 8-dim group
+    (dict(B=2, n_q_heads=4, n_kv_heads=2, d_k=64, d_v=128, m=16, K=100, L=333), 200, 133),  # d_sub 4, grouped heads, ragged, K < 256
+    (dict(B=1, n_q_heads=2, n_kv_heads=1, d_k=128, d_v=64, m=32, K=16, L=80), 80, 0),        # 32 subspaces: tables only
     (dict(B=1, n_q_heads=4, n_kv_heads=1, d_k=64, d_v=128, m=2, K=16, L=300), 259, 41),     # m 2: a CTA's last token has an odd index
 ])
 @pytest.mark.parametrize("q_scale", [1.0, 0.1])
@@ -421,7 +423,7 @@ def test_attend_prefill_matches_oracle(shape, L_q, q_pos0, q_scale, form):
     lk = ctx_for(w)
     lk.lookat_set_prefill_form(form)
     scores = torch.full((w.B, w.n_q_heads, L_q, w.L), float("nan"), device="cuda")
-    covered = w.d_k in (64, 128) and w.d_v in (64, 128) and w.d_sub % 8 == 0
+    covered = w.d_k in (64, 128) and w.d_v in (64, 128) and (w.d_sub % 8 == 0 or w.d_sub == 4) and w.m <= 16
     if form != "tables" and not covered:
         with pytest.raises(LookatError):
             lk.lookat_attend_prefill(dev(q), dev(books), dev(codes), dev(v), q_pos0=q_pos0, scores_out=scores)
@@ -440,8 +442,9 @@ def test_attend_prefill_matches_oracle(shape, L_q, q_pos0, q_scale, form):
     # the last query of a whole prompt is a decode step over the same cache
     if q_pos0 + L_q == w.L:
         dec = lk.lookat_attend(dev(codes), dev(v), q=dev(np.ascontiguousarray(q[:, :, -1])), codebooks=dev(books))
-        # the contraction form rounds each weight to fp16 once (relative 2^-12) where decode keeps two planes
-        assert float((dec - out[:, :, -1]).abs().max()) <= (2e-5 if form == "tables" else 3e-4)
+        # the contraction form rounds each weight to fp16 once (relative 2^-12 = 2.4e-4, values up to ~4) where decode
+        # keeps two planes; both sit inside OUT_TOL of the oracle, and well inside it of each other
+        assert float((dec - out[:, :, -1]).abs().max()) <= (2e-5 if form == "tables" else 6e-4)
 
 
 @pytest.mark.parametrize("seed", range(8))
@@ -451,7 +454,8 @@ def test_attend_prefill_contraction_on_random_shapes(seed):
     (the second call reuses the context's scratch)."""
     rng = np.random.default_rng(9000 + seed)
     d_k, d_v = int(rng.choice([64, 128])), int(rng.choice([64, 128]))
-    d_sub = int(rng.choice([8, 16, 32]))
+    d_sub = int(rng.choice([4, 8, 16, 32]))
+    d_sub = max(d_sub, d_k // 16)                         # at most 16 subspaces
     H_kv = int(rng.choice([1, 2, 3]))
     g = int(rng.choice([1, 2, 4]))
     K = int(rng.choice([16, 64, 200, 256]))
