@@ -163,33 +163,62 @@ encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K, int steps_per_c
 
     double dsum = 0.0;
     const long long cta_key0 = (long long)blockIdx.x * steps_per_cta * (kMmaWarps * kMmaKeysPerWarpStep);
-    for (int step = 0; step < steps_per_cta; ++step) {
-        const long long key0 = cta_key0 + ((long long)step * kMmaWarps + warp) * kMmaKeysPerWarpStep;
-        if (key0 >= a.n) break;                            // warp-uniform
-        // ---- operand tiles of 2 x 16 keys: rows g and g+8 of each, dims 2t,2t+1 (+8) per k-step ----
-        uint32_t xa[2][S::kSteps][4];
-        float xnorm[2][2];
-        const __half *rowp[2][2];
+    // operand words of the 2 x 16 keys of a step: rows g and g+8 of each tile, dims 2t,2t+1 (+8) per k-step
+    auto fetch_keys = [&](long long key0, uint32_t (&dst)[2][S::kSteps][4]) {
 #pragma unroll
         for (int u = 0; u < 2; ++u)
 #pragma unroll
             for (int rr = 0; rr < 2; ++rr) {
                 long long key = key0 + u * 16 + g + rr * 8;
                 if (key >= a.n) key = a.n - 1;              // clamped rows are computed and dropped
+                const __half *row = a.keys + ((size_t)bh * a.n + key) * d_k + j * D_SUB;
+#pragma unroll
+                for (int ks = 0; ks < S::kSteps; ++ks) {
+                    const uint32_t w0 = *reinterpret_cast<const uint32_t *>(row + ks * 16 + 2 * t);
+                    // d_sub 8: the second half of the k-step meets the remainder plane, so it repeats x
+                    uint32_t w1 = w0;
+                    if (D_SUB >= 16) w1 = *reinterpret_cast<const uint32_t *>(row + ks * 16 + 2 * t + 8);
+                    dst[u][ks][rr] = w0;                    // a0 (row g) / a1 (row g+8)
+                    dst[u][ks][2 + rr] = w1;                // a2 / a3
+                }
+            }
+    };
+    uint32_t xa_next[2][S::kSteps][4];
+    {
+        const long long first = cta_key0 + (long long)warp * kMmaKeysPerWarpStep;
+        if (first < a.n) fetch_keys(first, xa_next);
+    }
+    for (int step = 0; step < steps_per_cta; ++step) {
+        const long long key0 = cta_key0 + ((long long)step * kMmaWarps + warp) * kMmaKeysPerWarpStep;
+        if (key0 >= a.n) break;                            // warp-uniform
+        // ---- this step's keys arrived while the previous step searched; the next step's are requested now ----
+        uint32_t xa[2][S::kSteps][4];
+        float xnorm[2][2];
+        const __half *rowp[2][2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+#pragma unroll
+            for (int ks = 0; ks < S::kSteps; ++ks)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) xa[u][ks][i] = xa_next[u][ks][i];
+        {
+            const long long next0 = key0 + (long long)kMmaWarps * kMmaKeysPerWarpStep;
+            if (step + 1 < steps_per_cta && next0 < a.n) fetch_keys(next0, xa_next);
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                long long key = key0 + u * 16 + g + rr * 8;
+                if (key >= a.n) key = a.n - 1;
                 rowp[u][rr] = a.keys + ((size_t)bh * a.n + key) * d_k + j * D_SUB;
                 float nn = 0.f;
 #pragma unroll
                 for (int ks = 0; ks < S::kSteps; ++ks) {
-                    const uint32_t w0 = *reinterpret_cast<const uint32_t *>(rowp[u][rr] + ks * 16 + 2 * t);
-                    // d_sub 8: the second half of the k-step meets the remainder plane, so it repeats x
-                    uint32_t w1 = w0;
-                    if (D_SUB >= 16) w1 = *reinterpret_cast<const uint32_t *>(rowp[u][rr] + ks * 16 + 2 * t + 8);
-                    xa[u][ks][rr] = w0;                     // a0 (row g) / a1 (row g+8)
-                    xa[u][ks][2 + rr] = w1;                 // a2 / a3
-                    const float2 f0 = __half22float2(*reinterpret_cast<const __half2 *>(&w0));
+                    const float2 f0 = __half22float2(*reinterpret_cast<const __half2 *>(&xa[u][ks][rr]));
                     nn += f0.x * f0.x + f0.y * f0.y;
                     if (D_SUB >= 16) {
-                        const float2 f1 = __half22float2(*reinterpret_cast<const __half2 *>(&w1));
+                        const float2 f1 = __half22float2(*reinterpret_cast<const __half2 *>(&xa[u][ks][2 + rr]));
                         nn += f1.x * f1.x + f1.y * f1.y;
                     }
                 }
