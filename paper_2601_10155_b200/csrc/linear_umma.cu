@@ -13,13 +13,19 @@
 // tensor memory and returns.
 //
 // linear_skinny_kernel (M <= 32: one decode step of the whole batch): the product is bound by reading W once, and at
-// these sizes by latency.  A CTA owns 16 output columns; each of its 8 warps streams 8 rows of w_t over a quarter of K
-// with 16-byte loads straight into mma.sync.m16n8k16 B fragments (the k order inside a 32-wide block is permuted the
-// same way for both operands, so no shuffle is needed); two 16-row tiles cover the batch; the quarters meet in shared
-// memory.
+// these sizes by latency.  A CTA owns 8 or 32 output columns and a slice of K; its 4 warps stream rows of w_t over
+// quarters of the slice with 16-byte loads straight into mma.sync.m16n8k16 B fragments (the k order inside a 32-wide
+// block is permuted the same way for both operands, so no shuffle is needed); two 16-row tiles cover the batch; the
+// quarters meet in shared memory, the slices in the shared memory of the first CTA of a thread-block cluster.
 #include <cuda.h>           // CUtensorMap and its enums only; the driver entry point is looked up at run time
 
+#include <cooperative_groups.h>
+
+#include <cstring>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace lookat {
 
@@ -248,11 +254,14 @@ linear_umma_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// One decode step's products: M <= 32 rows, bound by reading w_t once, and small enough that latency decides.  A CTA of
-// 8 warps owns 16 output columns: warp (cw, ks) takes columns n0 + 8 cw .. +7 and the ks-th quarter of K, so 4 x as many
-// warps stream the weights as there are 8-column groups; the four partial sums meet in shared memory.  x is read from
-// global memory as it is needed (it is at most 192 KB and stays in L1/L2).
-constexpr int kSkThreads = 256, kSkCols = 16, kSkSplits = 4;
+// One decode step's products: M <= 32 rows, bound by reading w_t once, and small enough that latency decides: what
+// counts is how many 16-byte loads are in flight over the whole GPU.  A CTA of 4 warps owns 8 NT output columns and one
+// slice of K (about 384 wide); a thread-block cluster of up to 8 CTAs covers K.  Warp w takes a quarter of the slice --
+// three 32-wide k-blocks, unrolled, so all its loads are requested before the first MMA -- the quarters meet in shared
+// memory, and the slices meet in the shared memory of the cluster's first CTA (read through distributed shared
+// memory), which applies bias, activation and residual and stores.  x is read from global memory as it is needed (at
+// most 192 KB, resident in L2); NT = 4 for wide outputs, where re-reading x per 8 columns would cost more than w_t.
+constexpr int kSkThreads = 128, kSkWarps = 4, kSkSlice = 384, kSkMaxCluster = 8;
 
 __device__ __forceinline__ void sk_mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
 {
@@ -278,53 +287,68 @@ __device__ __forceinline__ uint4 sk_x8(const void *x, int r, int M, int K, int k
     return *reinterpret_cast<const uint4 *>(static_cast<const __half *>(x) + (size_t)r * K + k);
 }
 
-template <bool X_FP32>
-__global__ void __launch_bounds__(kSkThreads) linear_skinny_kernel(const void *__restrict__ x, const __half *__restrict__ w_t, LinearArgs p)
+// grid (column groups, K slices); the CTAs of one column group form a cluster (gridDim.y of them)
+template <bool X_FP32, int NT>
+__global__ void __launch_bounds__(kSkThreads) linear_skinny_kernel(const void *__restrict__ x, const __half *__restrict__ w_t, LinearArgs p,
+                                                                   int slice)
 {
-    __shared__ float part[kSkSplits][2][2][4][32];              // [k quarter][column warp][row tile][accumulator][lane]
+    constexpr int kVals = NT * 2 * 4 * 32;                      // partial sums of a CTA: [n-tile][row tile][accumulator][lane]
+    __shared__ float part[kSkWarps][kVals];
+    __shared__ float mine[kVals];                               // this CTA's slice, summed over its warps
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const int cw = warp & 1, ks = warp >> 1;
-    const int n0 = blockIdx.x * kSkCols + cw * 8;               // this warp's 8 output columns
+    const int n0 = blockIdx.x * (8 * NT);
     const int M = (int)p.M, K = p.K;
-    // this warp's share of K: whole 32-wide blocks
-    const int blocks = (K + 31) / 32, per = (blocks + kSkSplits - 1) / kSkSplits;
-    const int k_lo = min(K, ks * per * 32), k_hi = min(K, (ks + 1) * per * 32);
-    float acc[2][4] = {};
-    // lane (g, t) streams row n0 + g of w_t, 8 halfs at k = kk + 8 t of every 32-wide block (columns beyond N read row N - 1).
+    // this warp's share of the CTA's slice: whole 32-wide blocks
+    const int per = ((slice >> 5) + kSkWarps - 1) / kSkWarps;
+    const int k_end = min(K, ((int)blockIdx.y + 1) * slice);
+    const int k_lo = min(k_end, (int)blockIdx.y * slice + warp * per * 32), k_hi = min(k_end, k_lo + per * 32);
+    float acc[NT][2][4] = {};
+    // lane (g, t) streams row n0 + 8 nt + g of w_t, 8 halfs at k = kk + 8 t of every 32-wide block (columns beyond N read row N - 1).
     // Inside such a block the MMA's k index is a relabelling of the true one: the lane with t supplies true k = 8 t .. 8 t + 7
     // -- (8t, 8t+1 | 8t+2, 8t+3) to the first MMA, (8t+4, 8t+5 | 8t+6, 8t+7) to the second -- for both operands alike.
-    const __half *wrow = w_t + (size_t)min(n0 + g, p.N - 1) * K;
-#pragma unroll 4
+    const __half *wrow[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) wrow[nt] = w_t + (size_t)min(n0 + nt * 8 + g, p.N - 1) * K;
+#pragma unroll 3
     for (int kk = k_lo; kk < k_hi; kk += 32) {
         const int k = kk + 8 * t;
-        uint4 wv = make_uint4(0u, 0u, 0u, 0u), xa[2][2];
+        uint4 wv[NT], xa[2][2];
         const bool in = k < K;                                  // K is a multiple of 8
-        if (in) wv = __ldg(reinterpret_cast<const uint4 *>(wrow + k));
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) wv[nt] = in ? __ldg(reinterpret_cast<const uint4 *>(wrow[nt] + k)) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
             xa[mt][0] = in ? sk_x8<X_FP32>(x, mt * 16 + g, M, K, k) : make_uint4(0u, 0u, 0u, 0u);
             xa[mt][1] = in ? sk_x8<X_FP32>(x, mt * 16 + g + 8, M, K, k) : make_uint4(0u, 0u, 0u, 0u);
         }
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-            sk_mma(acc[mt], xa[mt][0].x, xa[mt][1].x, xa[mt][0].y, xa[mt][1].y, wv.x, wv.y);
-            sk_mma(acc[mt], xa[mt][0].z, xa[mt][1].z, xa[mt][0].w, xa[mt][1].w, wv.z, wv.w);
-        }
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+                sk_mma(acc[nt][mt], xa[mt][0].x, xa[mt][1].x, xa[mt][0].y, xa[mt][1].y, wv[nt].x, wv[nt].y);
+                sk_mma(acc[nt][mt], xa[mt][0].z, xa[mt][1].z, xa[mt][0].w, xa[mt][1].w, wv[nt].z, wv[nt].w);
+            }
     }
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
+    for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) part[ks][cw][mt][i][lane] = acc[mt][i];
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) part[warp][((nt * 2 + mt) * 4 + i) * 32 + lane] = acc[nt][mt][i];
     __syncthreads();
-    if (ks != 0) return;
-    // accumulator (mt, i): row mt * 16 + g + 8 * (i >> 1), column n0 + 2 t + (i & 1)
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int row = mt * 16 + g + 8 * (i >> 1), col = n0 + 2 * t + (i & 1);
+    for (int e = tid; e < kVals; e += kSkThreads) mine[e] = part[0][e] + part[1][e] + part[2][e] + part[3][e];
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster.sync();                                             // every slice of the column group is summed and visible
+    if (blockIdx.y == 0) {
+        const unsigned n_slices = gridDim.y;
+        // value e: n-tile e >> 8, row tile (e >> 7) & 1, accumulator (e >> 5) & 3 of lane e & 31:
+        // row mt * 16 + g + 8 * (i >> 1), column n0 + 8 nt + 2 t + (i & 1)
+        for (int e = tid; e < kVals; e += kSkThreads) {
+            const int ln = e & 31, i = (e >> 5) & 3, mt = (e >> 7) & 1, nt = e >> 8;
+            const int row = mt * 16 + (ln >> 2) + 8 * (i >> 1), col = n0 + nt * 8 + 2 * (ln & 3) + (i & 1);
+            float v = mine[e];
+            for (unsigned r = 1; r < n_slices; ++r) v += cluster.map_shared_rank(mine, r)[e];
             if (row >= M || col >= p.N) continue;
-            float v = part[0][cw][mt][i][lane] + part[1][cw][mt][i][lane] + part[2][cw][mt][i][lane] + part[3][cw][mt][i][lane];
             v += p.bias ? __half2float(p.bias[col]) : 0.f;
             if (p.gelu) v = gelu_tanh(v);
             if (p.qkv) {
@@ -339,6 +363,8 @@ __global__ void __launch_bounds__(kSkThreads) linear_skinny_kernel(const void *_
                 else static_cast<float *>(p.out)[at] = v;
             }
         }
+    }
+    cluster.sync();                                             // the other CTAs' shared memory stays until it has been read
 }
 
 typedef CUresult (*tensor_map_encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
@@ -394,9 +420,34 @@ lookat_status launch_linear(Ctx *ctx, const void *x, int x_fp32, const __half *w
 {
     p.timeout_flag = ctx->timeout_flag;
     if (p.M <= 32) {
-        const unsigned grid = (unsigned)((p.N + kSkCols - 1) / kSkCols);
-        if (x_fp32) linear_skinny_kernel<true><<<grid, kSkThreads, 0, ctx->stream>>>(x, w_t, p);
-        else linear_skinny_kernel<false><<<grid, kSkThreads, 0, ctx->stream>>>(x, w_t, p);
+        // K in slices of about kSkSlice, at most kSkMaxCluster of them (one cluster per column group), whole 32-wide blocks
+        int slices = (p.K + kSkSlice - 1) / kSkSlice;
+        if (slices > kSkMaxCluster) slices = kSkMaxCluster;
+        if (slices < 1) slices = 1;
+        const int slice = ((p.K + slices - 1) / slices + 31) / 32 * 32;
+        slices = (p.K + slice - 1) / slice;
+        // 32 columns per CTA where that still fills the GPU twice over, else 8
+        const bool wide = (long long)((p.N + 31) / 32) * slices >= 2ll * ctx->sm_count;
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3((unsigned)((p.N + (wide ? 31 : 7)) / (wide ? 32 : 8)), (unsigned)slices, 1);
+        cfg.blockDim = dim3(kSkThreads, 1, 1);
+        cfg.stream = ctx->stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 1;
+        attr.val.clusterDim.y = (unsigned)slices;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        cudaError_t err;
+        if (wide)
+            err = x_fp32 ? cudaLaunchKernelEx(&cfg, linear_skinny_kernel<true, 4>, x, w_t, p, slice)
+                         : cudaLaunchKernelEx(&cfg, linear_skinny_kernel<false, 4>, x, w_t, p, slice);
+        else
+            err = x_fp32 ? cudaLaunchKernelEx(&cfg, linear_skinny_kernel<true, 1>, x, w_t, p, slice)
+                         : cudaLaunchKernelEx(&cfg, linear_skinny_kernel<false, 1>, x, w_t, p, slice);
+        (void)err;                                              // picked up by check_launch
         return check_launch(ctx, "linear_skinny_kernel");
     }
     if (x_fp32) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "linear: fp32 input is taken for M <= 32 only");
