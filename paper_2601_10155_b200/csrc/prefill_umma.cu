@@ -27,6 +27,8 @@
 // lets the CTA drain and free its tensor memory.
 #include <cuda.h>           // CUtensorMap and its enums only; the driver entry point is looked up at run time
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace lookat {
@@ -354,25 +356,26 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
                                  : "memory");
         };
         // key rows of chunk c into key buffer c & 1: one 16-byte item of the codebook image per (token, 8-dim group, plane)
-        auto rebuild_keys = [&](int c) {
+        auto rebuild_keys_as = [&](auto pair_c, int c) {
+            constexpr bool PAIR = decltype(pair_c)::value;
             const int buf = c & 1;
             const bool whole = (long long)(c + 1) * kUmChunk <= t_end;   // every token of the chunk is visible to the CTA
             const uint8_t *cs = codes_s + buf * 1024 + my_j;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {             // in two batches: all loads of a batch before its stores
-                uint32_t code[Lay::kItems / 2], code_b[Lay::kItems / 2];
+                uint32_t code[Lay::kItems / 2], code_b[PAIR ? Lay::kItems / 2 : 1];
                 uint4 item[Lay::kItems / 2];
 #pragma unroll
                 for (int i = 0; i < Lay::kItems / 2; ++i) {
                     const uint8_t *ct = cs + (tl0 + (half * (Lay::kItems / 2) + i) * kTokStep) * a.m;
                     code[i] = ct[0];
-                    code_b[i] = pair ? ct[1] : 0u;
+                    if constexpr (PAIR) code_b[i] = ct[1];
                 }
 #pragma unroll
                 for (int i = 0; i < Lay::kItems / 2; ++i) {
                     item[i] = make_uint4(0u, 0u, 0u, 0u);
                     if (whole || (long long)c * kUmChunk + tl0 + (half * (Lay::kItems / 2) + i) * kTokStep < t_end) {
-                        if (!pair) {
+                        if constexpr (!PAIR) {
                             item[i] = *reinterpret_cast<const uint4 *>(my_src + code[i] * 128);
                         } else {
                             // sub-vectors of 4 dims: the group's first half from the centroid of subspace 2 gi, its second
@@ -391,6 +394,15 @@ attend_prefill_umma_kernel(PrefillArgs a, const __half *__restrict__ images, int
             }
             um_fence_async_smem();                             // generic-proxy writes before the MMA's reads
             um_bar_arrive(bar_k + 8 * buf);
+        };
+        auto rebuild_keys = [&](int c) {
+            if constexpr (D_K == 64) {                         // (16 subspaces at most: sub-vectors of 4 dims only on 64-dim heads)
+                if (pair) {
+                    rebuild_keys_as(std::true_type{}, c);
+                    return;
+                }
+            }
+            rebuild_keys_as(std::false_type{}, c);
         };
         fetch_codes(0);
         if (n_chunks > 1) fetch_codes(1);
