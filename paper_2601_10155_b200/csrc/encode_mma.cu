@@ -94,7 +94,7 @@ __device__ __noinline__ int exact_code_warp(const __half *x, const float *book, 
 
 // KMEANS: the assignment step of Lloyd's iteration (cluster sums, counts, distortion) on top of the codes
 template <int D_SUB, bool KMEANS>
-__global__ void __launch_bounds__(kMmaThreads, KMEANS ? 2 : 3)
+__global__ void __launch_bounds__(kMmaThreads, 2)
 encode_mma_kernel(EncodeArgs a, int H_kv, int d_k, int m, int K, int steps_per_cta)
 {
     using S = MmaShape<D_SUB>;

@@ -447,7 +447,7 @@ lookat_status launch_linear(Ctx *ctx, const void *x, int x_fp32, const __half *w
         else
             err = x_fp32 ? cudaLaunchKernelEx(&cfg, linear_skinny_kernel<true, 1>, x, w_t, p, slice)
                          : cudaLaunchKernelEx(&cfg, linear_skinny_kernel<false, 1>, x, w_t, p, slice);
-        (void)err;                                              // picked up by check_launch
+        if (err != cudaSuccess) return check_launch(ctx, "linear_skinny_kernel (cluster launch)");
         return check_launch(ctx, "linear_skinny_kernel");
     }
     if (x_fp32) return set_error(ctx, LOOKAT_ERR_UNSUPPORTED, "linear: fp32 input is taken for M <= 32 only");
