@@ -250,6 +250,60 @@ def test_attend_is_independent_of_the_split_count_and_handles_ragged_rows(shape)
         check_attend(w, lk, q, books, codes, v, seq_lens=[L_row] * w.B, n_splits=3)
 
 
+# Rows above 8192 tokens take the long-row kernel (attend_stream_kernel: bulk-copy ring, one table set, ranges cut
+# from the flat tile sequence); shapes chosen so that ranges lie inside a unit, cross one border, or span several units.
+LONG_SHAPES = [
+    dict(B=1, n_q_heads=4, n_kv_heads=1, d_k=64, d_v=64, m=4, K=64, L=8300),         # one unit over all CTAs: 3-4 tiles each
+    dict(B=3, n_q_heads=6, n_kv_heads=2, d_k=128, d_v=128, m=8, K=256, L=8500),      # g = 3; six units, ragged rows below
+    dict(B=2, n_q_heads=16, n_kv_heads=2, d_k=64, d_v=128, m=16, K=255, L=8209),     # g = 8: two head groups; m = 16; odd L
+    dict(B=2, n_q_heads=2, n_kv_heads=2, d_k=32, d_v=64, m=1, K=16, L=12000),        # m = 1, g = 1
+    dict(B=40, n_q_heads=8, n_kv_heads=4, d_k=32, d_v=64, m=2, K=32, L=8224),        # 160 units: every range spans two borders
+]
+
+
+@pytest.mark.parametrize("shape", LONG_SHAPES)
+def test_attend_on_long_rows_matches_oracle(shape):
+    w = synth.small_workload(**shape)
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.3)
+    books = random_books(w, 6)
+    codes = oracle.encode_keys(keys, books)
+    lk = ctx_for(w)
+    check_attend(w, lk, q, books, codes, v)
+    # ragged rows: empty, full, one token into the last tile, and (larger batches) lengths all over the place
+    rng = np.random.default_rng(w.L)
+    seq_lens = ([0, w.L, w.L - 15] * w.B)[:w.B] if w.B <= 3 else list(rng.integers(0, w.L + 1, w.B))
+    check_attend(w, lk, q, books, codes, v, seq_lens=seq_lens)
+    if w.B <= 3:
+        for n_splits in (1, 5, 64):
+            check_attend(w, lk, q, books, codes, v, seq_lens=seq_lens, n_splits=n_splits)
+
+
+@pytest.mark.parametrize("shape", LONG_SHAPES[:4])
+@pytest.mark.parametrize("pos_from_end", [1, 16, 50])
+def test_decode_step_on_long_rows(shape, pos_from_end):
+    """The append inside the long-row kernel, with the cache filled to the end of its rows or a little short of it.  Where
+    one unit is cut among all CTAs the new token's tile is among the first tiles its CTA copies (encoded before the ring
+    is primed); elsewhere it lies far down a range (encoded while the first tiles are in flight)."""
+    w = synth.small_workload(**shape)
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.4)
+    books = random_books(w, 8)
+    pos = w.L - pos_from_end
+    ref_codes, gap = oracle.encode_keys(keys[:, :, :pos + 1], books, want_gap=True)
+    assert not ((gap[:, :, pos] > 0) & (gap[:, :, pos] < 1e-6)).any()
+    cache = np.zeros((w.B, w.n_kv_heads, w.L, w.m), np.uint8)
+    cache[:, :, :pos] = ref_codes[:, :, :pos]
+    cache[:, :, pos:] = 201 % w.K                      # stale codes where the new key goes and beyond
+    lk = ctx_for(w)
+    codes_dev = dev(cache)
+    out = lk.lookat_decode_step(dev(q), dev(np.ascontiguousarray(keys[:, :, pos])), dev(books), codes_dev, dev(v), pos)
+    torch.cuda.synchronize()
+    got = codes_dev.cpu().numpy()
+    assert np.array_equal(got[:, :, :pos + 1], ref_codes)          # row pos written, bit-exact
+    assert np.all(got[:, :, pos + 1:] == 201 % w.K)                 # nothing beyond it touched
+    ref = oracle.attend(oracle.build_lut(q, books), ref_codes, v[:, :, :pos + 1], d_k=w.d_k)
+    assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
+
+
 def test_attend_with_prebuilt_tables_and_explicit_scale():
     w = synth.small_workload(B=2, n_q_heads=8, n_kv_heads=2, d_k=64, d_v=64, m=4, K=64, L=500)
     keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.5)
