@@ -824,6 +824,10 @@ lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_
             const long long cph = ctas / a.H_kv, tph = (long long)hgroups * a.B * tpu;
             if (a.multi && a.H_kv > 1 && a.tiles_per_cta > tpu && cph >= 1 && cph * a.H_kv * 10 >= ctas * 9) {
                 a.tiles_per_cta = (tph + cph - 1) / cph;
+                // whole units per CTA where that lengthens the longest range by less than 15 %: no unit is shared, so no
+                // partial goes through global memory and no CTA waits on a counter before it may write its rows
+                const long long whole = (a.tiles_per_cta + tpu - 1) / tpu * tpu;
+                if (whole * 100 <= a.tiles_per_cta * 115) a.tiles_per_cta = whole;
                 a.ctas_per_head = (int)((tph + a.tiles_per_cta - 1) / a.tiles_per_cta);
                 a.n_ctas = a.ctas_per_head * a.H_kv;
             }
