@@ -41,7 +41,11 @@ def lk():
 
 
 @pytest.mark.parametrize("M,N,K", [(200, 384, 128), (128, 128, 64), (129, 200, 72), (1000, 768, 768), (333, 3072, 768), (257, 768, 3072),
-                                   (32, 384, 128), (1, 96, 64), (17, 100, 1032), (32, 2304, 768)])
+                                   (32, 384, 128), (1, 96, 64), (17, 100, 1032), (32, 2304, 768),
+                                   (32, 768, 3072),      # one-token product, K in 8 slices over a thread-block cluster
+                                   (32, 9491, 768),      # ... 32 columns per CTA (wide output), ragged last column group
+                                   (5, 20011, 136),      # ... wide, one slice, K not a multiple of 32
+                                   (32, 8, 8)])          # ... the smallest
 @pytest.mark.parametrize("mode", ["plain_fp16", "gelu_fp16", "residual_fp32"])
 def test_linear_matches_oracle(lk, M, N, K, mode):
     rng = np.random.default_rng(M * 31 + N * 7 + K)
