@@ -71,6 +71,10 @@ const char *lookat_last_error(const lookat_ctx *ctx);
 /* 1 in the debug build of the library, 0 otherwise. */
 int32_t lookat_is_debug_build(void);
 
+/* One environment variable is read, for tests: with LOOKAT_NO_TENSOR_MAPS set, the long-row attend kernel fetches its
+ * tiles by 16-byte cp.async pieces instead of tiled bulk copies -- the path it otherwise takes only where the driver has
+ * no tensor-map entry point or the caches have 2^31 rows or more.  Same results, slower. */
+
 /*
  * Section 3.4, Prototype Learning: for every KV head h and subspace j, a
  * K-centroid codebook minimising  sum_k min_c || k^(j) - c ||^2  over the

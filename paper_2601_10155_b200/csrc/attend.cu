@@ -38,6 +38,7 @@
 // (d_v in {64,128}, m in {1,2,4,8,16}, 16-byte aligned rows) do not hold.
 #include <cuda.h>           // CUtensorMap only
 
+#include <cstdlib>
 #include <cstring>
 #include <type_traits>
 
@@ -778,7 +779,9 @@ lookat_status plan_attend(Ctx *ctx, AttendArgs &a, int n_splits, size_t *part_o_
 {
     a.fused_lut = (!a.lut && a.d_k <= 256) ? 1 : 0;    // tables built inside the streaming kernel
     // tiles by the bulk-copy engine where the driver provides tensor maps and the row coordinate fits 32 bits
-    a.bulk = (tile_maps_available() && (long long)a.B * a.H_kv * a.L_max < (1ll << 31)) ? 1 : 0;
+    // (LOOKAT_NO_TENSOR_MAPS in the environment forces the 16-byte cp.async ring, which otherwise runs only where the
+    // driver has no tensor-map entry point or the caches have 2^31 rows or more: a switch for tests of that path)
+    a.bulk = (tile_maps_available() && (long long)a.B * a.H_kv * a.L_max < (1ll << 31) && !getenv("LOOKAT_NO_TENSOR_MAPS")) ? 1 : 0;
     const int stages = stream_shape_ok(ctx, a) ? stream_stages(ctx, a) : 0;
     if (!stages) a.fused_lut = 0;
     if (stages) {

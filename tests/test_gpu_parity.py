@@ -278,6 +278,32 @@ def test_attend_on_long_rows_matches_oracle(shape):
             check_attend(w, lk, q, books, codes, v, seq_lens=seq_lens, n_splits=n_splits)
 
 
+@pytest.mark.parametrize("shape", [LONG_SHAPES[1], LONG_SHAPES[3], LONG_SHAPES[4]])
+def test_long_rows_on_the_cp_async_ring(shape, monkeypatch):
+    """The long-row kernel's other copy path (16-byte cp.async pieces into padded rows; taken where the driver offers no
+    tensor maps or the caches have 2^31 rows or more), forced by the library's environment switch: attention, ragged
+    rows and a decode step against the oracle."""
+    monkeypatch.setenv("LOOKAT_NO_TENSOR_MAPS", "1")
+    w = synth.small_workload(**shape)
+    keys, v, q = synth.make_keys(w), synth.make_values(w), synth.make_queries(w, 0.3)
+    books = random_books(w, 6)
+    codes = oracle.encode_keys(keys, books)
+    lk = ctx_for(w)
+    check_attend(w, lk, q, books, codes, v)
+    rng = np.random.default_rng(w.L + 1)
+    seq_lens = ([0, w.L, w.L - 15] * w.B)[:w.B] if w.B <= 3 else list(rng.integers(0, w.L + 1, w.B))
+    check_attend(w, lk, q, books, codes, v, seq_lens=seq_lens)
+    pos = w.L - 1
+    cache = codes.copy()
+    cache[:, :, pos] = 201 % w.K
+    codes_dev = dev(cache)
+    out = lk.lookat_decode_step(dev(q), dev(np.ascontiguousarray(keys[:, :, pos])), dev(books), codes_dev, dev(v), pos)
+    torch.cuda.synchronize()
+    assert np.array_equal(codes_dev.cpu().numpy(), codes)
+    ref = oracle.attend(oracle.build_lut(q, books), codes, v, d_k=w.d_k)
+    assert np.abs(out.cpu().numpy() - ref).max() <= OUT_TOL
+
+
 @pytest.mark.parametrize("shape", LONG_SHAPES[:4])
 @pytest.mark.parametrize("pos_from_end", [1, 16, 50])
 def test_decode_step_on_long_rows(shape, pos_from_end):
