@@ -378,6 +378,9 @@ def test_gpt2_shapes_end_to_end_with_handoff():
     dict(B=3, n_q_heads=8, n_kv_heads=2, d_k=64, d_v=64, m=4, K=64, L=300),        # streaming kernel, fused append
     dict(B=2, n_q_heads=16, n_kv_heads=2, d_k=128, d_v=128, m=8, K=256, L=2000),   # g = 8: two head groups per KV head
     dict(B=2, n_q_heads=4, n_kv_heads=2, d_k=32, d_v=8, m=4, K=16, L=100),         # generic kernel: separate encode
+    dict(B=2, n_q_heads=4, n_kv_heads=2, d_k=64, d_v=64, m=2, K=200, L=200),       # g = 2, sub-vectors of 32 dims, K < 256
+    dict(B=1, n_q_heads=12, n_kv_heads=12, d_k=64, d_v=64, m=8, K=256, L=900),     # g = 1, m = 8: distances do not fit beside the partials
+    dict(B=40, n_q_heads=4, n_kv_heads=2, d_k=64, d_v=128, m=4, K=256, L=1500),    # several units per round (separate append pass)
 ])
 @pytest.mark.parametrize("pos_from_end", [1, 2, 17])
 def test_decode_step_on_device_appends_then_attends(shape, pos_from_end):
