@@ -224,6 +224,39 @@ def test_full_size_prefill_on_sampled_rows(prefill_4k, form):
             assert np.abs(out[b, h, i] - ref[0, 0, 0]).max() <= OUT_TOL, (form, b, h, i)
 
 
+def test_prefill_with_16_subspaces_on_64_dim_heads_at_a_gpt2_prompt_size():
+    """The paper's 16-subspace setting on GPT-2 heads (d_k 64, sub-vectors of 4 dims) over a prompt of 1024 tokens, batch 8,
+    12 heads, in the contraction form (two centroids per 8-dim group of a rebuilt key row): sampled (row, head, query)
+    triples against the oracle, every first query against its closed form, and the two forms against each other."""
+    w = synth.small_workload(B=8, n_q_heads=12, n_kv_heads=12, d_k=64, d_v=64, m=16, K=256, L=1024, rank=16)
+    keys, v = synth.make_keys(w), synth.make_values(w)
+    q = synth.make_prefill_queries(w, w.L)
+    books, _ = oracle.fit_codebooks(keys[:, :, :512], w.m, w.K, iters=2, seed=11)
+    lk = Lookat(w.n_q_heads, w.n_kv_heads, w.d_k, w.d_v, w.m, w.K)
+    codes_d = lk.lookat_encode_keys(dev(keys), dev(books))
+    heads = [(0, 0), (3, 7), (7, 11)]
+    for b, h in heads:
+        ref_codes, gap = oracle.encode_keys(keys[b:b + 1, h:h + 1], books[h:h + 1], want_gap=True)
+        got = codes_d[b, h].cpu().numpy()
+        near = (gap[0, 0] > 0) & (gap[0, 0] < 1e-6)
+        assert not ((got != ref_codes[0, 0]) & ~near).any()
+        codes_d[b, h] = dev(ref_codes[0, 0])
+    outs = {}
+    for form in ("contraction", "tables"):
+        lk.lookat_set_prefill_form(form)
+        outs[form] = lk.lookat_attend_prefill(dev(q), dev(books), codes_d, dev(v)).cpu().numpy()
+    lk.lookat_set_prefill_form("auto")
+    out = outs["contraction"]
+    assert np.isfinite(out).all()
+    assert np.abs(out[:, :, 0] - v[:, :, 0].astype(np.float32)).max() <= 1e-3
+    assert np.abs(out - outs["tables"]).max() <= 2 * OUT_TOL
+    for b, h in heads:
+        codes_row = codes_d[b, h].cpu().numpy()[None, None]
+        for i in (0, 1, 63, 64, 127, 128, 255, 256, 700, 1023):
+            ref = oracle.attend_prefill(q[b:b + 1, h:h + 1, i:i + 1], books[h:h + 1], codes_row, v[b:b + 1, h:h + 1], q_pos0=i)
+            assert np.abs(out[b, h, i] - ref[0, 0, 0]).max() <= OUT_TOL, (b, h, i)
+
+
 # ------------------------------------------------------------------ k-means at the sizes the benchmark fits
 def _fit_against_oracle(w, keys, lk, iters, head, subspaces, seed):
     """GPU k-means on the whole problem, the oracle's on `subspaces` (consecutive, starting at 0) of KV head `head`
